@@ -1,0 +1,393 @@
+"""Pins for the CPU oracle: it is checked against what the paper and the mathematics fix,
+never against itself.  Every test names the passage it pins.  CPU only."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.fft
+
+from paper_2510_26771_b200 import inputs as gen
+
+T_ID, T_HAAR, T_DCT = 0, 1, 2
+
+
+# --------------------------------------------------------------------------------------
+# Transform matrices (Theorem 1 premise: L orthogonal; Sec. "Efficient Energy Concentration")
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("transform,n,levels", [
+    (T_HAAR, 2, 0), (T_HAAR, 8, 0), (T_HAAR, 8, 1), (T_HAAR, 64, 3), (T_HAAR, 256, 0), (T_HAAR, 1024, 6),
+    (T_DCT, 2, 0), (T_DCT, 8, 0), (T_DCT, 256, 0), (T_DCT, 96, 0),
+])
+def test_orthonormal(oracle, transform, n, levels):
+    Lm = oracle.transform_matrix(transform, n, levels)
+    assert np.max(np.abs(Lm @ Lm.T - np.eye(n))) <= 1e-12
+    assert np.max(np.abs(Lm.T @ Lm - np.eye(n))) <= 1e-12
+
+
+def test_haar_n2_hand_case(oracle):
+    r = 1.0 / math.sqrt(2.0)
+    Lm = oracle.transform_matrix(T_HAAR, 2, 0)
+    assert np.allclose(Lm, [[r, r], [r, -r]], rtol=0, atol=1e-15)
+
+
+def _haar_closed_form(n, levels):
+    """Rows written from the closed form: a_l[i] = 2^(-l/2) on [i 2^l, (i+1) 2^l);
+    d_j[i] = 2^(-j/2) (+ on the first half, - on the second half of [i 2^j, (i+1) 2^j));
+    row order [a_l | d_l | d_(l-1) | ... | d_1]."""
+    M = np.zeros((n, n))
+    na = n >> levels
+    for i in range(na):
+        M[i, i << levels:(i + 1) << levels] = 2.0 ** (-levels / 2)
+    for j in range(levels, 0, -1):
+        base = n >> j
+        for i in range(n >> j):
+            lo, mid, hi = i << j, (i << j) + (1 << (j - 1)), (i + 1) << j
+            M[base + i, lo:mid] = 2.0 ** (-j / 2)
+            M[base + i, mid:hi] = -(2.0 ** (-j / 2))
+    return M
+
+
+@pytest.mark.parametrize("n,levels", [(4, 1), (4, 2), (16, 3), (64, 3), (64, 6), (512, 9), (2048, 11)])
+def test_haar_closed_form_rows(oracle, n, levels):
+    Lm = oracle.transform_matrix(T_HAAR, n, levels)
+    assert np.max(np.abs(Lm - _haar_closed_form(n, levels))) <= 1e-14
+
+
+def test_haar_full_depth_is_levels_zero(oracle):
+    assert np.array_equal(oracle.transform_matrix(T_HAAR, 64, 0), oracle.transform_matrix(T_HAAR, 64, 6))
+
+
+def test_haar_each_level_halves_the_lowpass_band(oracle):
+    """Each DWT step concentrates a constant (fully correlated) signal into the first half:
+    constant input c => every detail row is 0 and the l-level approximation is c 2^(l/2)."""
+    n, K = 64, 3
+    X = np.full((1, n, K), 1.75)
+    for levels in (1, 2, 3, 6):
+        T = oracle.apply_dense(oracle.transform_matrix(T_HAAR, n, levels), X)[0]
+        na = n >> levels
+        assert np.allclose(T[:na], 1.75 * 2 ** (levels / 2), rtol=1e-14)
+        assert np.max(np.abs(T[na:])) <= 1e-14
+
+
+def test_impulse_gives_matrix_column(oracle):
+    n = 32
+    for transform, levels in ((T_HAAR, 0), (T_HAAR, 2), (T_DCT, 0)):
+        Lm = oracle.transform_matrix(transform, n, levels)
+        for t in (0, 5, 31):
+            X = np.zeros((1, n, 1))
+            X[0, t, 0] = 1.0
+            assert np.array_equal(oracle.apply_dense(Lm, X)[0, :, 0], Lm[:, t])
+
+
+@pytest.mark.parametrize("n", [2, 16, 256])
+def test_dct_matches_scipy_ortho_dct2(oracle, n):
+    """Special case that reduces to a library routine: the DCT matrix applied to data equals
+    SciPy's orthonormal DCT-II along the token axis."""
+    rng = np.random.default_rng(11)
+    X = rng.standard_normal((1, n, 5))
+    T = oracle.apply_dense(oracle.transform_matrix(T_DCT, n), X)
+    ref = scipy.fft.dct(X, type=2, norm="ortho", axis=1)
+    assert np.max(np.abs(T - ref)) <= 1e-12 * np.max(np.abs(ref))
+    # row 0 is the DC row: low frequencies come first
+    assert np.allclose(oracle.transform_matrix(T_DCT, n)[0], 1 / math.sqrt(n))
+
+
+def test_block_diagonal_application(oracle):
+    """A blockwise transform acts on each block of n tokens and each batch item separately."""
+    rng = np.random.default_rng(5)
+    n, B, L, K = 8, 2, 32, 3
+    X = rng.standard_normal((B, L, K))
+    Lm = oracle.transform_matrix(T_DCT, n)
+    T = oracle.apply_dense(Lm, X)
+    for b in range(B):
+        for blk in range(L // n):
+            assert np.allclose(T[b, blk * n:(blk + 1) * n], Lm @ X[b, blk * n:(blk + 1) * n], atol=1e-13)
+
+
+@pytest.mark.parametrize("transform,n,levels", [(T_HAAR, 128, 0), (T_HAAR, 128, 3), (T_DCT, 64, 0)])
+def test_energy_and_reconstruction(oracle, transform, n, levels):
+    """Sequence transforms do not alter the total energy (remark after Theorem 1) and
+    L^T (L X) = X."""
+    rng = np.random.default_rng(3)
+    X = rng.standard_normal((2, 2 * n, 7)) * np.array([1, 10, 0.1, 3, 1, 1, 50])
+    Lm = oracle.transform_matrix(transform, n, levels)
+    T = oracle.apply_dense(Lm, X)
+    assert abs(np.sum(T * T) - np.sum(X * X)) <= 1e-12 * np.sum(X * X)
+    back = oracle.apply_dense(Lm, T, transpose=True)
+    assert np.max(np.abs(back - X)) <= 1e-12 * np.max(np.abs(X))
+
+
+def test_csr_equals_dense(oracle):
+    rng = np.random.default_rng(8)
+    for n, levels in ((64, 0), (256, 5), (1024, 0)):
+        X = rng.standard_normal((1, 2 * n, 4)).astype(np.float32)
+        Lm = oracle.transform_matrix(T_HAAR, n, levels)
+        csr = oracle.haar_matrix_csr(n, levels)
+        T_d = oracle.apply_dense(Lm, X.astype(np.float64))
+        T_s = oracle.apply_csr(csr, n, X)
+        assert np.max(np.abs(T_d - T_s)) <= 1e-13 * np.max(np.abs(T_d))
+        Y_d = oracle.apply_dense(Lm, T_d, transpose=True)
+        Y_s = oracle.apply_csr_transpose(csr, n, T_d)
+        assert np.max(np.abs(Y_d - Y_s)) <= 1e-13 * np.max(np.abs(Y_d))
+        # CSR holds exactly the non-zeros of the dense matrix
+        rp, col, val = csr
+        D = np.zeros((n, n))
+        for i in range(n):
+            D[i, col[rp[i]:rp[i + 1]]] = val[rp[i]:rp[i + 1]]
+        assert np.array_equal(D, Lm)
+
+
+def test_bias_projection_closed_form(oracle):
+    """l = L 1 (Method, second equation): Haar l-level => 2^(l/2) on the first n/2^l rows,
+    0 elsewhere; DCT => (sqrt n, 0, ..., 0); and L^T (Y_t + l b^T) = L^T Y_t + 1 b^T."""
+    n = 64
+    ones = np.ones((1, n, 1))
+    for levels in (1, 3, 6):
+        l = oracle.apply_dense(oracle.transform_matrix(T_HAAR, n, levels), ones)[0, :, 0]
+        na = n >> levels
+        assert np.allclose(l[:na], 2 ** (levels / 2), rtol=1e-14)
+        assert np.max(np.abs(l[na:])) <= 1e-14
+    l = oracle.apply_dense(oracle.transform_matrix(T_DCT, n), ones)[0, :, 0]
+    assert abs(l[0] - math.sqrt(n)) <= 1e-13 and np.max(np.abs(l[1:])) <= 1e-13
+    rng = np.random.default_rng(1)
+    Yt = rng.standard_normal((1, n, 5))
+    beta = rng.standard_normal(5)
+    Lm = oracle.transform_matrix(T_HAAR, n, 3)
+    lvec = (Lm @ np.ones(n))[:, None]
+    lhs = oracle.apply_dense(Lm, Yt + lvec * beta[None, :], transpose=True)
+    rhs = oracle.apply_dense(Lm, Yt, transpose=True) + beta
+    assert np.max(np.abs(lhs - rhs)) <= 1e-12
+
+
+# --------------------------------------------------------------------------------------
+# Quantizer (Sec. 2.1, first equation and the range bound that follows it)
+# --------------------------------------------------------------------------------------
+
+def test_quantizer_properties(oracle):
+    rng = np.random.default_rng(2)
+    rows, K = 40, 96
+    T = rng.standard_normal((rows, K)) * rng.lognormal(0, 2, size=(rows, 1))
+    bits = np.where(np.arange(rows) < 8, 8, 4).astype(np.int32)
+    q, s = oracle.quantize_rows(T, bits)
+    qmax = (2 ** (bits - 1) - 1)[:, None]
+    assert q.dtype == np.int8 and s.dtype == np.float32
+    assert np.all(np.abs(q.astype(int)) <= qmax)                  # restricted symmetric range
+    am = np.argmax(np.abs(T), axis=1)
+    assert np.all(np.abs(q[np.arange(rows), am].astype(int)) == qmax[:, 0])   # absmax -> +-qmax
+    assert np.allclose(s, (np.max(np.abs(T), axis=1).astype(np.float32) / qmax[:, 0].astype(np.float32)))
+    sd = s.astype(np.float64)[:, None]
+    err = T - sd * q
+    assert np.all(np.abs(err) <= sd / 2 * (1 + 1e-6))             # no clipping: rounding error only
+    # per-token bound: ||Q(t) - t||^2 <= K s^2 / 4 <= K ||t||^2 / (4 qmax^2)
+    e2 = np.sum(err * err, axis=1)
+    assert np.all(e2 <= K * sd[:, 0] ** 2 / 4 * (1 + 1e-6))
+    assert np.all(e2 <= K * np.sum(T * T, axis=1) / (4 * qmax[:, 0] ** 2) * (1 + 1e-6))
+    # re-quantizing the de-quantized row is idempotent
+    q2, s2 = oracle.quantize_rows(sd * q, bits)
+    assert np.array_equal(q2, q)
+    assert np.allclose(s2, s, rtol=1e-6)
+
+
+def test_quantizer_round_half_to_even_and_zero_row(oracle):
+    # scale = 7/7 = 1 exactly, so the values are their own pre-rounding codes
+    T = np.array([[7.0, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.49, -3.51],
+                  [0, 0, 0, 0, 0, 0, 0, 0, 0]])
+    q, s = oracle.quantize_rows(T, np.array([4, 4], dtype=np.int32))
+    assert s[0] == 1.0 and s[1] == 1.0                                # zero row: scale 1, codes 0
+    assert q[0].tolist() == [7, 0, 2, 2, 0, -2, -2, 3, -4]
+    assert not q[1].any()
+    # 8-bit row
+    T = np.array([[127.0, -126.5, 0.49999, 63.5]])
+    q, s = oracle.quantize_rows(T, np.array([8], dtype=np.int32))
+    assert s[0] == 1.0 and q[0].tolist() == [127, -126, 0, 64]
+
+
+def test_bit_map_reproduces_printed_effective_bits(oracle):
+    """Golden values printed in the paper (tests/golden/effective_bits.txt)."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "effective_bits.txt")
+    rows = [ln.split("#")[0].split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 2
+    for k, L, bh, bl, eff in rows:
+        bits = oracle.bit_map(int(L), int(L), int(k), int(bh), int(bl))
+        assert bits.mean() == float(eff)
+        assert np.all(bits[:int(k)] == int(bh)) and np.all(bits[int(k):] == int(bl))
+    # blockwise: the first k_hi rows OF EACH BLOCK are the 8-bit ones
+    bits = oracle.bit_map(1024, 256, 16)
+    assert bits.mean() == 4.25
+    assert set(np.nonzero(bits == 8)[0] % 256) == set(range(16))
+
+
+def test_error_invariance_under_orthogonal_transform(oracle):
+    """First step of the proof of Theorem 1: ||L^T Q(LX) - X||_F = ||Q(LX) - LX||_F."""
+    cfg = gen.scaled(gen.config_tiny(), L=128, K=64)
+    X = gen.make_activation(cfg).astype(np.float64)
+    for transform, levels in ((T_HAAR, 0), (T_HAAR, 3), (T_DCT, 0)):
+        Lm = oracle.transform_matrix(transform, cfg.L, levels)
+        T = oracle.apply_dense(Lm, X)
+        q, s = oracle.quantize_rows(T[0], oracle.bit_map(cfg.L, cfg.L, 8))
+        Tq = (q * s.astype(np.float64)[:, None])[None]
+        lhs = np.linalg.norm(oracle.apply_dense(Lm, Tq, transpose=True) - X)
+        rhs = np.linalg.norm(Tq - T)
+        assert abs(lhs - rhs) <= 1e-12 * rhs
+
+
+# --------------------------------------------------------------------------------------
+# Integer GEMM and the whole layer
+# --------------------------------------------------------------------------------------
+
+def test_gemm_brute_force(oracle):
+    rng = np.random.default_rng(4)
+    M, N, K = 37, 19, 256
+    q = rng.integers(-127, 128, size=(M, K), dtype=np.int8)
+    wq = rng.integers(-7, 8, size=(N, K), dtype=np.int8)
+    acc = oracle.gemm_i32(q, wq)
+    ref = q.astype(np.int64) @ wq.astype(np.int64).T
+    assert acc.shape == (M, N) and np.array_equal(acc.astype(np.int64), ref)
+    assert np.max(np.abs(acc)) <= 127 * 7 * K
+    # extreme codes reach the bound exactly
+    acc = oracle.gemm_i32(np.full((2, K), 127, np.int8), np.full((3, K), -7, np.int8))
+    assert np.all(acc == -127 * 7 * K)
+
+
+def test_unquantized_pipeline_is_plain_matmul(oracle):
+    """(L^-1 (L X)) W^T = L^-1 ((L X) W^T) = X W^T  (Method, second equation)."""
+    rng = np.random.default_rng(6)
+    B, L, K, N = 2, 64, 48, 24
+    X = rng.standard_normal((B, L, K)).astype(np.float32)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    ref = oracle.matmul_f64(X.reshape(-1, K), W).reshape(B, L, N)
+    assert np.max(np.abs(ref - X.astype(np.float64) @ W.astype(np.float64).T)) <= 1e-12
+    for transform, n, levels in ((T_HAAR, 64, 0), (T_HAAR, 32, 2), (T_DCT, 16, 0)):
+        Lm = oracle.transform_matrix(transform, n, levels)
+        T = oracle.apply_dense(Lm, X.astype(np.float64))
+        Yt = (T.reshape(-1, K) @ W.astype(np.float64).T).reshape(B, L, N)
+        Y = oracle.apply_dense(Lm, Yt, transpose=True)
+        assert np.max(np.abs(Y - ref)) <= 1e-12 * np.max(np.abs(ref))
+
+
+def test_layer_exact_when_codes_are_exact(oracle):
+    """Inputs built so that every transformed row is an integer multiple of a power-of-two
+    scale with the extreme code present: quantization is then lossless and the STaMP layer
+    must return the textbook X W^T (+ bias)."""
+    rng = np.random.default_rng(9)
+    nblk, K, N = 6, 32, 10
+    # block of 4 tokens [u, u, v, v] with 2-level Haar: a_2 = u + v, d_2 = u - v, d_1 = 0
+    P = rng.integers(-127, 128, size=(nblk, K)); P[:, 0] = 127      # 8-bit row (k_hi = 1)
+    Q = rng.integers(-7, 8, size=(nblk, K)); Q[:, 1] = -7           # 4-bit row
+    u, v = (P + Q) / 2.0, (P - Q) / 2.0
+    X = np.stack([u, u, v, v], axis=1).reshape(1, 4 * nblk, K).astype(np.float32)
+    Wi = rng.integers(-7, 8, size=(N, K)); Wi[:, 2] = 7
+    W = (Wi * 2.0 ** -3).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    out = oracle.stamp_linear(X, W, bias, transform=T_HAAR, block=4, levels=2, k_hi=1)
+    q = out["q"].reshape(nblk, 4, K)
+    assert np.array_equal(q[:, 0], P) and np.array_equal(q[:, 1], Q) and not q[:, 2:].any()
+    assert np.array_equal(out["wq"], Wi)
+    assert np.all(out["x_scale"].reshape(nblk, 4) == 1.0) and np.all(out["w_scale"] == 2.0 ** -3)
+    ref = X[0].astype(np.float64) @ W.astype(np.float64).T + bias.astype(np.float64)
+    assert np.max(np.abs(out["Y"] - ref)) <= 1e-12 * np.max(np.abs(ref))
+
+
+def _python_loop_layer(X, W, bias, n, levels, k_hi):
+    """The Algorithm written out with Python floats and loops (tiny sizes only)."""
+    L, K = len(X), len(X[0])
+    N = len(W)
+    r = 1.0 / math.sqrt(2.0)
+    T = [[0.0] * K for _ in range(L)]
+    for b0 in range(0, L, n):
+        for j in range(K):
+            v = [X[b0 + t][j] for t in range(n)]
+            length = n
+            for _ in range(levels):
+                a = [(v[2 * i] + v[2 * i + 1]) * r for i in range(length // 2)]
+                d = [(v[2 * i] - v[2 * i + 1]) * r for i in range(length // 2)]
+                v[:length] = a + d
+                length //= 2
+            for t in range(n):
+                T[b0 + t][j] = v[t]
+
+    def quant(row, qmax):
+        amax = max(abs(x) for x in row)
+        s = float(np.float32(amax) / np.float32(qmax)) if amax > 0 else 1.0
+        return [max(-qmax, min(qmax, int(round(x / s)))) for x in row], s   # round(): half to even
+
+    qs = [quant(T[i], 127 if (i % n) < k_hi else 7) for i in range(L)]
+    ws = [quant(W[c], 7) for c in range(N)]
+    Yt = [[sum(qs[i][0][k] * ws[c][0][k] for k in range(K)) * qs[i][1] * ws[c][1] for c in range(N)]
+          for i in range(L)]
+    Y = [[0.0] * N for _ in range(L)]
+    for b0 in range(0, L, n):
+        for c in range(N):
+            v = [Yt[b0 + t][c] for t in range(n)]
+            length = n >> levels
+            for _ in range(levels):
+                a, d = v[:length], v[length:2 * length]
+                rec = []
+                for i in range(length):
+                    rec += [(a[i] + d[i]) * r, (a[i] - d[i]) * r]
+                v[:2 * length] = rec
+                length *= 2
+            for t in range(n):
+                Y[b0 + t][c] = v[t] + bias[c]
+    return np.array(Y), np.array([x[0] for x in qs]), np.array([x[1] for x in qs])
+
+
+def test_layer_vs_python_loops(oracle):
+    """Brute force on tiny inputs: an independent, loop-by-loop statement of the Algorithm
+    (fast in-place Haar instead of the explicit matrix)."""
+    rng = np.random.default_rng(12)
+    L, K, N, n, levels, k_hi = 16, 6, 5, 8, 3, 2
+    X = rng.standard_normal((L, K)).astype(np.float32)
+    X[:, 1] *= 20
+    W = (rng.standard_normal((N, K)) * 0.1).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    out = oracle.stamp_linear(X[None], W, bias, transform=T_HAAR, block=n, levels=levels, k_hi=k_hi)
+    Y, q, s = _python_loop_layer(X.astype(float).tolist(), W.astype(float).tolist(), bias.astype(float).tolist(),
+                                 n, levels, k_hi)
+    assert np.array_equal(out["q"], q)
+    assert np.allclose(out["x_scale"], s, rtol=1e-7)
+    assert np.max(np.abs(out["Y"] - Y)) <= 1e-12 * np.max(np.abs(Y))
+
+
+def test_layer_stages_compose(oracle):
+    """The one-call layer equals its exported steps chained in the Algorithm's order."""
+    cfg = gen.scaled(gen.config_tiny(), L=64, K=128, N=32)
+    X, W = gen.make_activation(cfg), gen.make_weight(cfg)
+    out = oracle.stamp_linear(X, W, None, transform=T_DCT, block=32, k_hi=4)
+    Lm = oracle.transform_matrix(T_DCT, 32)
+    T = oracle.apply_dense(Lm, X.astype(np.float64))
+    assert np.array_equal(out["T"], T.reshape(-1, cfg.K))
+    q, s = oracle.quantize_rows(T.reshape(-1, cfg.K), oracle.bit_map(cfg.L, 32, 4))
+    wq, sw = oracle.quantize_weights(W)
+    assert np.array_equal(out["q"], q) and np.array_equal(out["wq"], wq)
+    acc = oracle.gemm_i32(q, wq)
+    assert np.array_equal(out["acc"], acc)
+    Yt = oracle.dequant(acc, s, sw)
+    assert np.array_equal(out["Yt"], Yt)
+    assert np.array_equal(out["Y"], oracle.apply_dense(Lm, Yt.reshape(1, cfg.L, -1), transpose=True).reshape(cfg.L, -1))
+
+
+# --------------------------------------------------------------------------------------
+# Qualitative claims on the synthetic stand-ins (sanity, not parity criteria)
+# --------------------------------------------------------------------------------------
+
+def _sqnr(ref, x):
+    return 10 * math.log10(np.sum(ref * ref) / np.sum((ref - x) ** 2))
+
+
+def test_energy_concentrates_and_stamp_beats_uniform_4bit(oracle):
+    cfg = gen.scaled(gen.config_sweep(512, 2048), K=256, N=64)
+    X, W = gen.make_activation(cfg), gen.make_weight(cfg)
+    ref = oracle.matmul_f64(X[0], W)
+    stamp = oracle.stamp_linear(X, W, None, transform=T_HAAR, k_hi=cfg.k_hi, want=("T", "Y"))
+    e = np.sum(stamp["T"] ** 2, axis=1)
+    L = cfg.L
+    # AR(1) with rho = 0.9 decorrelates over ~10 tokens: every level up to 2^5 tokens gains energy
+    # over the finer one, and the 8-bit rows (coarsest bands) carry far more energy per token
+    band_mean = [e[L >> j:L >> (j - 1)].mean() for j in range(5, 0, -1)]
+    assert all(a > b for a, b in zip(band_mean, band_mean[1:]))
+    assert e[:cfg.k_hi].mean() > 10 * e[cfg.k_hi:].mean()
+    uniform = oracle.stamp_linear(X, W, None, transform=T_ID, k_hi=0, want=("Y",))
+    assert _sqnr(ref, stamp["Y"]) > _sqnr(ref, uniform["Y"])
