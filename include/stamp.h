@@ -1,0 +1,175 @@
+/*
+ * stamp.h -- C ABI of the B200 (sm_100a) STaMP-quantized linear layer.
+ *
+ * STaMP (Sequence Transformation and Mixed Precision, arXiv 2510.26771) mixes an activation
+ * X [L tokens x K features] along the TOKEN axis with an orthonormal sequence transform L
+ * (multi-level Haar DWT or DCT-II), quantizes each transformed token with its own scale --
+ * the first k_hi tokens of each transform block at bits_hi (8), the others at bits_lo (4) --
+ * multiplies the integer codes with per-output-channel quantized weights, de-quantizes, and
+ * applies the inverse sequence transform to the output:
+ *
+ *        Y = L^-1 ( Q(L X) Q(W)^T ) + 1 bias^T            (Algorithm "STaMP Linear";
+ *                                                          Method section, second equation)
+ *
+ * Conventions common to every call
+ *   - All tensor pointers are DEVICE pointers owned by the caller; tensors are dense,
+ *     row-major.  X: [B, L, K];  W: [N, K];  Y, Yt: [B, L, N].  B independent sequences.
+ *   - Scratch space is the caller's `ws` buffer of at least stamp_workspace_bytes() bytes,
+ *     256-byte aligned.  Calls that share a workspace must be ordered on one stream.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work; they never synchronize the stream.
+ *   - Every function returns a stamp_status.  Argument problems are detected on the host
+ *     before anything is launched.  Device-side problems (a bounded wait inside a kernel that
+ *     ran out) are recorded in a device status word read by stamp_last_device_status().
+ *   - Shape rules: K % 128 == 0, N % 8 == 0, the transform block length (cfg.block, or L when
+ *     0) is a power of two that divides L, Haar levels <= log2(block).  Anything else returns
+ *     STAMP_ERR_UNSUPPORTED.
+ *   - Transformed-token ("logical") order inside a block of n tokens:
+ *       Haar, l levels: [a_l (n/2^l rows) | d_l | d_(l-1) | ... | d_1 (n/2 rows)], with
+ *         a[i] = (x[2i] + x[2i+1]) / sqrt2,  d[i] = (x[2i] - x[2i+1]) / sqrt2  per level;
+ *       DCT-II (orthonormal): row u = frequency u, row 0 = DC.
+ *     The 8-bit tokens are the rows {i : i mod n < k_hi} ("the first 64 tokens are kept at
+ *     8 bits", Sec. "Optimal bit allocation").
+ *   - Quantizer (Sec. 2.1, first equation, symmetric form): scale = absmax / qmax,
+ *     code = clamp(round_half_even(t / scale), -qmax, +qmax), qmax = 2^(bits-1) - 1; a zero
+ *     row gets scale 1.  Nothing clips (min-max range setting of Sec. 2.1).
+ */
+#ifndef STAMP_H_
+#define STAMP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  STAMP_OK = 0,
+  STAMP_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad enum value            */
+  STAMP_ERR_UNSUPPORTED = 2, /* valid request outside the shape / transform rules above    */
+  STAMP_ERR_WORKSPACE = 3,   /* ws is null, misaligned or smaller than required            */
+  STAMP_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, tensor map)   */
+  STAMP_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (device status only)    */
+} stamp_status;
+
+typedef enum { STAMP_F32 = 0, STAMP_BF16 = 1 } stamp_dtype;
+
+typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2 } stamp_transform;
+
+typedef enum { STAMP_G_PER_TOKEN = 0, STAMP_G_PER_CHANNEL = 1 } stamp_granularity;
+
+/* Weight operand formats accepted by the GEMM entry points. */
+typedef enum {
+  STAMP_W_PACKED4 = 0, /* [N, K/2] two's-complement nibbles, low nibble = even k (the output of
+                          stamp_quantize_weights); expanded into the workspace on every call  */
+  STAMP_W_INT8 = 1     /* [N, K] one 4-bit code per int8 (the output of stamp_prepare_weights):
+                          the tensor-core operand format, made once for static weights        */
+} stamp_weight_format;
+
+/* The knobs of the paper's problem statement. */
+typedef struct {
+  int32_t transform; /* stamp_transform: the sequence transform L                              */
+  int32_t block;     /* tokens per transform block; 0 => the whole sequence (L tokens)         */
+  int32_t levels;    /* Haar: number of levels, 1..log2(block); 0 => full depth. DCT: ignored  */
+  int32_t k_hi;      /* the first k_hi transformed tokens OF EACH BLOCK use bits_hi            */
+  int32_t bits_hi;   /* 8                                                                      */
+  int32_t bits_lo;   /* 4                                                                      */
+  int32_t bits_w;    /* 4 (weights, per output channel)                                        */
+  int32_t act_gran;  /* STAMP_G_PER_TOKEN   (scales shared across features, Sec. 2.1)          */
+  int32_t w_gran;    /* STAMP_G_PER_CHANNEL (one scale per output channel, Sec. "Set-up")      */
+  int32_t reserved;  /* must be 0                                                              */
+} stamp_config;
+
+/* Bytes of scratch any call below may need for this problem size (the maximum over the calls). */
+int stamp_workspace_bytes(const stamp_config* cfg, int B, int L, int K, int N, size_t* out_bytes);
+
+/*
+ * Weight quantization (offline; weights are untouched by the sequence transform, Method
+ * section): per output channel n, w_scale[n] = max_k |W[n,k]| / 7 and
+ * wq[n,k] = clamp(rne(W[n,k] / w_scale[n]), -7, 7).
+ *   W        [N, K]   w_dtype (STAMP_F32 or STAMP_BF16)      in
+ *   wq       [N, K/2] packed 4-bit codes (STAMP_W_PACKED4)    out
+ *   w_scale  [N]      float                                   out
+ */
+int stamp_quantize_weights(const stamp_config* cfg, const void* W, int w_dtype, int N, int K, void* wq,
+                           float* w_scale, void* stream);
+
+/* Expand packed weight codes into the tensor-core operand format (STAMP_W_INT8), once per
+ * weight matrix.  wq_packed [N, K/2] in; w_int8 [N, K] out.  No counterpart in the paper: it
+ * is a storage choice of this implementation (the int8 MMA consumes one code per byte). */
+int stamp_prepare_weights(const stamp_config* cfg, const void* wq_packed, int N, int K, void* w_int8,
+                          void* stream);
+
+/*
+ * Algorithm lines "X <- L X" and "x_i <- Q(x_i; b_i)": sequence transform + per-token
+ * mixed-precision quantization of one activation tensor.
+ *   X        [B, L, K]   x_dtype                                                    in
+ *   q_hi     [B * n_hi, K]        int8, the 8-bit tokens in logical order, where
+ *            n_hi = k_hi * (L / block); row (b, blk, i) at index (b*(L/block)+blk)*k_hi + i   out
+ *   q_lo     [B * (L-n_hi), K/2]  packed 4-bit codes of the remaining tokens in logical
+ *            order (low nibble = even k)                                             out
+ *   x_scale  [B, L]      float, per transformed token (logical order)                out
+ */
+int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, void* q_hi,
+                   void* q_lo, float* x_scale, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Algorithm line "Y <- X W^T" on the integer codes plus de-quantization (Sec. 2.1):
+ *   Yt[m, n] = (sum_k q[m,k] * wq[n,k]) * x_scale[m] * w_scale[n],   int32 accumulation on the
+ * tensor cores.  Output stays in the transformed token domain.
+ *   q_hi, q_lo, x_scale : as written by stamp_quantize                               in
+ *   w, w_format, w_scale: weight codes (stamp_weight_format) and per-channel scales  in
+ *   Yt       [B, L, N]   float                                                       out
+ */
+int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, const float* x_scale,
+                 const void* w, int w_format, const float* w_scale, int B, int L, int K, int N, float* Yt,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Algorithm lines "Y <- L^-1 Y" and "Y <- Y + bias": inverse sequence transform along tokens
+ * (L^-1 = L^T, L orthonormal: Theorem 1's premise) and optional bias.
+ *   Yt       [B, L, N]   float                                                       in
+ *   bias     [N] float or NULL                                                       in
+ *   Y        [B, L, N]   y_dtype (STAMP_F32 or STAMP_BF16)                           out
+ */
+int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
+                  int y_dtype, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The whole Algorithm in one call: Y = L^-1( Q(L X) Q(W)^T ) + bias.  Intermediates (codes,
+ * scales, transformed-domain output) live in the workspace only.
+ */
+int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, const void* w, int w_format,
+                       const float* w_scale, const float* bias, int B, int L, int K, int N, void* Y,
+                       int y_dtype, void* ws, size_t ws_bytes, void* stream);
+
+/* ---- parity / debug exports: the intermediate stages, judged separately against the oracle ---- */
+
+/* T = L X in fp32, logical token order.  T [B, L, K] float out. */
+int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, float* T,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/* Codes written by stamp_quantize, one per int8, logical order.  codes [B, L, K] int8 out. */
+int stamp_debug_unpack_codes(const stamp_config* cfg, const void* q_hi, const void* q_lo, int B, int L, int K,
+                             int8_t* codes, void* stream);
+
+/* Raw int32 accumulators of the tensor-core GEMM.  acc [B*L, N] int32 out. */
+int stamp_debug_gemm_i32(const stamp_config* cfg, const void* q_hi, const void* q_lo, const void* w,
+                         int w_format, int B, int L, int K, int N, int32_t* acc, void* ws, size_t ws_bytes,
+                         void* stream);
+
+/* Synchronizes `stream`, then reads and clears the device status word of the current device.
+ * *status is STAMP_OK or STAMP_ERR_TIMEOUT (a bounded wait inside a kernel expired; outputs of
+ * the calls since the last read are then invalid). */
+int stamp_last_device_status(void* stream, int* status);
+
+/* How many kernels of this library the calling thread's last API call launched. */
+int stamp_last_launch_count(void);
+
+const char* stamp_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STAMP_H_ */

@@ -1,0 +1,203 @@
+"""Thin ctypes binding of libstamp.so: same names as the C ABI (include/stamp.h), argument
+marshalling only.  Tensors are torch CUDA tensors used as plain device buffers; every step of the
+layer runs inside the CUDA library.  There is no CPU fallback: if the library is missing or a
+call fails, an exception is raised."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from .build import LIB_PATH
+
+STAMP_OK = 0
+F32, BF16 = 0, 1
+T_IDENTITY, T_HAAR, T_DCT2 = 0, 1, 2
+G_PER_TOKEN, G_PER_CHANNEL = 0, 1
+W_PACKED4, W_INT8 = 0, 1
+
+EXPORTS = (
+    "stamp_workspace_bytes", "stamp_quantize_weights", "stamp_prepare_weights", "stamp_quantize",
+    "stamp_linear", "stamp_inverse", "stamp_linear_fused", "stamp_debug_transform",
+    "stamp_debug_unpack_codes", "stamp_debug_gemm_i32", "stamp_last_device_status",
+    "stamp_last_launch_count", "stamp_status_string",
+)
+
+
+class StampConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("transform", "block", "levels", "k_hi", "bits_hi", "bits_lo",
+                                              "bits_w", "act_gran", "w_gran", "reserved")]
+
+
+def make_config(transform: int, block: int = 0, levels: int = 0, k_hi: int = 64, bits_hi: int = 8,
+                bits_lo: int = 4, bits_w: int = 4) -> StampConfig:
+    return StampConfig(transform, block, levels, k_hi, bits_hi, bits_lo, bits_w, G_PER_TOKEN, G_PER_CHANNEL, 0)
+
+
+class StampError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built in-tree by paper_2510_26771_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"CUDA library not built: {LIB_PATH} is missing "
+                               "(run `python -m paper_2510_26771_b200.build`); there is no fallback path")
+        _lib = ctypes.CDLL(LIB_PATH)
+        _lib.stamp_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            getattr(_lib, name)
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().stamp_status_string(int(status)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise ValueError(f"unsupported dtype {t.dtype}")
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != STAMP_OK:
+        raise StampError(rc, what)
+
+
+def _ws_args(ws: torch.Tensor):
+    return _ptr(ws), ctypes.c_size_t(ws.numel() * ws.element_size())
+
+
+def stamp_workspace_bytes(cfg: StampConfig, B: int, L: int, K: int, N: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().stamp_workspace_bytes(ctypes.byref(cfg), B, L, K, N, ctypes.byref(out)), "stamp_workspace_bytes")
+    return int(out.value)
+
+
+def alloc_workspace(cfg: StampConfig, B: int, L: int, K: int, N: int, device="cuda") -> torch.Tensor:
+    return torch.empty(stamp_workspace_bytes(cfg, B, L, K, N), dtype=torch.uint8, device=device)
+
+
+def stamp_quantize_weights(cfg: StampConfig, W: torch.Tensor):
+    N, K = W.shape
+    wq = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    w_scale = torch.empty((N,), dtype=torch.float32, device=W.device)
+    _check(lib().stamp_quantize_weights(ctypes.byref(cfg), _ptr(W), _dtype_code(W), N, K, _ptr(wq), _ptr(w_scale),
+                                        _stream()), "stamp_quantize_weights")
+    return wq, w_scale
+
+
+def stamp_prepare_weights(cfg: StampConfig, wq: torch.Tensor) -> torch.Tensor:
+    N, K2 = wq.shape
+    w8 = torch.empty((N, 2 * K2), dtype=torch.int8, device=wq.device)
+    _check(lib().stamp_prepare_weights(ctypes.byref(cfg), _ptr(wq), N, 2 * K2, _ptr(w8), _stream()),
+           "stamp_prepare_weights")
+    return w8
+
+
+def n_hi_rows(cfg: StampConfig, B: int, L: int) -> int:
+    n = cfg.block if cfg.block else L
+    return B * (L // n) * cfg.k_hi
+
+
+def stamp_quantize(cfg: StampConfig, X: torch.Tensor, ws: torch.Tensor):
+    B, L, K = X.shape
+    nh = n_hi_rows(cfg, B, L)
+    q_hi = torch.empty((max(nh, 1), K), dtype=torch.int8, device=X.device)
+    q_lo = torch.empty((max(B * L - nh, 1), K // 2), dtype=torch.uint8, device=X.device)
+    x_scale = torch.empty((B, L), dtype=torch.float32, device=X.device)
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_quantize(ctypes.byref(cfg), _ptr(X), _dtype_code(X), B, L, K, _ptr(q_hi), _ptr(q_lo),
+                                _ptr(x_scale), wp, wb, _stream()), "stamp_quantize")
+    return q_hi, q_lo, x_scale
+
+
+def stamp_linear(cfg: StampConfig, q_hi, q_lo, x_scale, w, w_format: int, w_scale, B: int, L: int, K: int, N: int,
+                 ws: torch.Tensor) -> torch.Tensor:
+    Yt = torch.empty((B, L, N), dtype=torch.float32, device=x_scale.device)
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_linear(ctypes.byref(cfg), _ptr(q_hi), _ptr(q_lo), _ptr(x_scale), _ptr(w), int(w_format),
+                              _ptr(w_scale), B, L, K, N, _ptr(Yt), wp, wb, _stream()), "stamp_linear")
+    return Yt
+
+
+def stamp_inverse(cfg: StampConfig, Yt: torch.Tensor, bias: Optional[torch.Tensor], ws: torch.Tensor,
+                  out_dtype=torch.float32, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    B, L, N = Yt.shape
+    Y = out if out is not None else torch.empty((B, L, N), dtype=out_dtype, device=Yt.device)
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_inverse(ctypes.byref(cfg), _ptr(Yt), _ptr(bias), B, L, N, _ptr(Y), _dtype_code(Y), wp, wb,
+                               _stream()), "stamp_inverse")
+    return Y
+
+
+def stamp_linear_fused(cfg: StampConfig, X: torch.Tensor, w: torch.Tensor, w_format: int, w_scale: torch.Tensor,
+                       bias: Optional[torch.Tensor], ws: torch.Tensor, out_dtype=torch.float32,
+                       out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    B, L, K = X.shape
+    N = w.shape[0]
+    Y = out if out is not None else torch.empty((B, L, N), dtype=out_dtype, device=X.device)
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_linear_fused(ctypes.byref(cfg), _ptr(X), _dtype_code(X), _ptr(w), int(w_format),
+                                    _ptr(w_scale), _ptr(bias), B, L, K, N, _ptr(Y), _dtype_code(Y), wp, wb,
+                                    _stream()), "stamp_linear_fused")
+    return Y
+
+
+def stamp_debug_transform(cfg: StampConfig, X: torch.Tensor, ws: torch.Tensor) -> torch.Tensor:
+    B, L, K = X.shape
+    T = torch.empty((B, L, K), dtype=torch.float32, device=X.device)
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_debug_transform(ctypes.byref(cfg), _ptr(X), _dtype_code(X), B, L, K, _ptr(T), wp, wb,
+                                       _stream()), "stamp_debug_transform")
+    return T
+
+
+def stamp_debug_unpack_codes(cfg: StampConfig, q_hi, q_lo, B: int, L: int, K: int) -> torch.Tensor:
+    codes = torch.empty((B, L, K), dtype=torch.int8, device=q_lo.device)
+    _check(lib().stamp_debug_unpack_codes(ctypes.byref(cfg), _ptr(q_hi), _ptr(q_lo), B, L, K, _ptr(codes), _stream()),
+           "stamp_debug_unpack_codes")
+    return codes
+
+
+def stamp_debug_gemm_i32(cfg: StampConfig, q_hi, q_lo, w, w_format: int, B: int, L: int, K: int, N: int,
+                         ws: torch.Tensor) -> torch.Tensor:
+    acc = torch.empty((B * L, N), dtype=torch.int32, device=w.device)
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_debug_gemm_i32(ctypes.byref(cfg), _ptr(q_hi), _ptr(q_lo), _ptr(w), int(w_format), B, L, K, N,
+                                      _ptr(acc), wp, wb, _stream()), "stamp_debug_gemm_i32")
+    return acc
+
+
+def stamp_last_device_status() -> int:
+    st = ctypes.c_int(0)
+    _check(lib().stamp_last_device_status(_stream(), ctypes.byref(st)), "stamp_last_device_status")
+    return int(st.value)
+
+
+def stamp_last_launch_count() -> int:
+    return int(lib().stamp_last_launch_count())

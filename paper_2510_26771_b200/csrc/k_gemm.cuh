@@ -1,0 +1,261 @@
+// Integer GEMM of the STaMP linear layer on the 5th-generation tensor cores (Algorithm line
+// "Y <- X W^T" evaluated on the integer codes, followed by the de-quantization of Sec. 2.1).
+//
+//   acc[tok, ch] = sum_k a8[tok, k] * w8[ch, k]            int8 x int8 -> int32
+//
+// Operand roles are swapped with respect to the usual activation-major GEMM: the weight tile
+// (128 output channels) is the MMA "A" operand and the token tile (BN tokens) is the MMA "B"
+// operand, so an accumulator lives in TMEM with lane = output channel and column = token.
+// An epilogue thread therefore owns one output channel and reads runs of consecutive tokens
+// into registers -- the axis along which the inverse sequence transform acts -- while a warp's
+// 32 lanes cover 32 consecutive channels of one token, i.e. one coalesced 128-byte store.
+//
+// Structure: persistent CTAs (one per SM), warp-specialised.
+//   warp 0     TMA producer: 128-byte-swizzled K-major tiles of both operands into a
+//              STAGES-deep shared-memory ring (one mbarrier pair per stage)
+//   warp 1     allocates TMEM; one elected thread issues tcgen05.mma kind::i8 (128 x BN x 32
+//              per instruction, four per 128-byte K block) into one of two accumulators
+//   warps 2-5  epilogue: tcgen05.ld the finished accumulator (the other one is being filled),
+//              de-quantize with per-token x per-channel scales, store
+// Every mbarrier wait is bounded; when one expires the CTA raises the device status word,
+// drains its outstanding copies, frees TMEM and returns.
+#pragma once
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace stamp {
+
+enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1 };
+
+struct GemmParams {
+  int n_out;               // output channels (MMA M extent)
+  int m_tok;               // tokens (MMA N extent)
+  int k;                   // reduction length, multiple of 128
+  const float* x_scale;    // [m_tok]
+  const float* w_scale;    // [n_out]
+  void* out;               // [m_tok, n_out] float (EPI_DEQUANT_F32) or int32 (EPI_RAW_I32)
+  int group;               // channel tiles per raster band
+};
+
+constexpr int GEMM_BM = 128;           // output channels per tile
+constexpr int GEMM_BK = 128;           // int8 per K block = one 128-byte swizzle row
+constexpr int GEMM_THREADS = 192;
+constexpr long long GEMM_WAIT_LIMIT = 4000000000LL;  // SM clocks (~2 s) before a wait gives up
+
+template <int BN, int STAGES>
+struct GemmSmem {
+  static constexpr int W_BYTES = GEMM_BM * GEMM_BK;
+  static constexpr int X_BYTES = BN * GEMM_BK;
+  static constexpr int STAGE_BYTES = W_BYTES + X_BYTES;
+  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  // full[STAGES], empty[STAGES], tfull[2], tempty[2], then tmem base + abort word
+  static constexpr int NUM_BARS = 2 * STAGES + 4;
+  static constexpr int TOTAL = BAR_OFFSET + NUM_BARS * 8 + 16;
+  static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for 1024-byte alignment of the ring
+};
+
+__device__ __forceinline__ void tile_coords(int tile, int ch_tiles, int tok_tiles, int group, int& ch_t, int& tok_t) {
+  // bands of `group` channel tiles; inside a band, channel tiles vary fastest so that CTAs
+  // running at the same time share token tiles and the band's weight tiles stay in L2
+  const int per_band = group * tok_tiles;
+  const int band = tile / per_band;
+  const int rem = tile - band * per_band;
+  const int first = band * group;
+  const int height = min(group, ch_tiles - first);
+  tok_t = rem / height;
+  ch_t = first + (rem - tok_t * height);
+}
+
+template <int BN, int STAGES, int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+    k_gemm_i8(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, GemmParams p) {
+  using SM = GemmSmem<BN, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFFSET);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tfull = empty + STAGES;
+  uint64_t* tempty = tfull + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  volatile uint32_t* abort_word = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int ch_tiles = (p.n_out + GEMM_BM - 1) / GEMM_BM;
+  const int tok_tiles = (p.m_tok + BN - 1) / BN;
+  const int num_tiles = ch_tiles * tok_tiles;
+  const int num_kb = p.k / GEMM_BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&tfull[a], 1);
+      ptx::mbar_init(&tempty[a], 128);
+    }
+    *abort_word = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&tmap_w);
+    ptx::prefetch_tensormap(&tmap_x);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, 2 * BN);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (ptx::elect_one()) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t armed = 0, armed_parity = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int ch_t, tok_t;
+        tile_coords(tile, ch_tiles, tok_tiles, p.group, ch_t, tok_t);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!ptx::mbar_wait_bounded(&empty[stage], phase ^ 1u, abort_word, GEMM_WAIT_LIMIT)) {
+            ok = false;
+            break;
+          }
+          uint8_t* ws = smem + stage * SM::STAGE_BYTES;
+          ptx::mbar_arrive_expect_tx(&full[stage], SM::STAGE_BYTES);
+          ptx::tma_load_2d(ws, &tmap_w, &full[stage], kb * GEMM_BK, ch_t * GEMM_BM);
+          ptx::tma_load_2d(ws + SM::W_BYTES, &tmap_x, &full[stage], kb * GEMM_BK, tok_t * BN);
+          armed |= 1u << stage;
+          armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+          if (++stage == STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      if (!ok) {
+        *abort_word = 1;
+        raise_device_status(STAMP_ERR_TIMEOUT);
+        // let the copies already in flight land before the CTA gives its shared memory back
+        for (int s = 0; s < STAGES; ++s)
+          if (armed & (1u << s)) {
+            const long long t0 = clock64();
+            while (!ptx::mbar_try_wait(&full[s], (armed_parity >> s) & 1u) && clock64() - t0 < 2000000LL) {
+            }
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (ptx::elect_one()) {
+      constexpr uint32_t idesc = ptx::make_i8_idesc(GEMM_BM, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        const int a = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1u;
+        if (!ptx::mbar_wait_bounded(&tempty[a], acc_phase ^ 1u, abort_word, GEMM_WAIT_LIMIT)) {
+          ok = false;
+          break;
+        }
+        ptx::tc_fence_after();
+        const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(a * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!ptx::mbar_wait_bounded(&full[stage], phase, abort_word, GEMM_WAIT_LIMIT)) {
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after();
+          const uint32_t wa = ptx::smem_u32(smem + stage * SM::STAGE_BYTES);
+          const uint32_t xa = wa + SM::W_BYTES;
+#pragma unroll
+          for (int k = 0; k < GEMM_BK / 32; ++k) {
+            const uint64_t adesc = ptx::make_kmajor_sw128_desc(wa + k * 32);
+            const uint64_t bdesc = ptx::make_kmajor_sw128_desc(xa + k * 32);
+            ptx::mma_i8_ss(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          ptx::tc_commit(&empty[stage]);  // frees the stage once these MMAs have read it
+          if (++stage == STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (ok) ptx::tc_commit(&tfull[a]);  // accumulator complete
+      }
+      if (!ok) {
+        *abort_word = 1;
+        raise_device_status(STAMP_ERR_TIMEOUT);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32 * (warp % 4) ...
+    const int row = quarter * 32 + lane;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      int ch_t, tok_t;
+      tile_coords(tile, ch_tiles, tok_tiles, p.group, ch_t, tok_t);
+      const int a = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1u;
+      const int ch = ch_t * GEMM_BM + row;
+      const int tok0 = tok_t * BN;
+      const bool ch_ok = ch < p.n_out;
+      float sw = 0.f;
+      if (EPI == EPI_DEQUANT_F32 && ch_ok) sw = __ldg(p.w_scale + ch);
+      // the TMEM loads below are warp-collective: the whole warp continues or the whole warp stops
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&tfull[a], acc_phase, abort_word, GEMM_WAIT_LIMIT))) {
+        ok = false;
+        break;
+      }
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(a * BN);
+#pragma unroll 1
+      for (int chunk = 0; chunk < BN / 32; ++chunk) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32b_x32(taddr + chunk * 32, r);
+        ptx::tmem_ld_wait();
+        const int tbase = tok0 + chunk * 32;
+        if (EPI == EPI_DEQUANT_F32) {
+          float* out = static_cast<float*>(p.out);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int tok = tbase + j;
+            if (tok < p.m_tok) {
+              const float sx = __ldg(p.x_scale + tok);
+              const float v = static_cast<float>(static_cast<int>(r[j])) * sx * sw;
+              if (ch_ok) out[(long)tok * p.n_out + ch] = v;
+            }
+          }
+        } else {
+          int* out = static_cast<int*>(p.out);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int tok = tbase + j;
+            if (tok < p.m_tok && ch_ok) out[(long)tok * p.n_out + ch] = static_cast<int>(r[j]);
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&tempty[a]);
+    }
+    if (!ok) {
+      *abort_word = 1;
+      raise_device_status(STAMP_ERR_TIMEOUT);
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+}  // namespace stamp

@@ -1,0 +1,257 @@
+// General-shape kernels: multi-pass Haar analysis / synthesis along the token axis with the
+// transformed activations materialised in fp32, the row quantizer that reads them, code
+// (un)packing and the offline weight quantizer.  These serve the debug exports, every shape the
+// specialised kernels do not cover, and the unfused API calls.
+#pragma once
+#include "common.cuh"
+
+namespace stamp {
+
+// ------------------------------------------------------------------------------------------
+// Haar analysis, P levels per pass (Sec. "Efficient Energy Concentration": each DWT step moves
+// the averages to the first half and the differences to the second half of the tokens).
+//
+// One thread owns two adjacent channels of one group of G = 2^P consecutive input tokens and
+// runs the butterflies in registers on UNNORMALISED sums; a coefficient of global level j is
+// multiplied once by 2^(-j/2) when it is written.  Detail rows go to their logical row of T,
+// [a | d_levels | ... | d_1]; the group's running sum goes to `aout` for the next pass, or, in
+// the last pass, to the approximation rows of T.
+//   in      [nseq, Lin, K]      TIn (first pass: X; later passes: unnormalised sums, float)
+//   T       [nseq * n, K]       float
+//   aout    [nseq, Lin >> P, K] float, or nullptr in the last pass
+//   rowmax  [nseq * n]          uint bit patterns of per-row |T| maxima (atomicMax), or nullptr
+// ------------------------------------------------------------------------------------------
+template <int P, typename TIn>
+__global__ void __launch_bounds__(128) k_haar_fwd_pass(const TIn* __restrict__ in, int Lin, long ngroups, int K,
+                                                       float* __restrict__ T, int n, int lvl0,
+                                                       float* __restrict__ aout, unsigned* __restrict__ rowmax) {
+  constexpr int G = 1 << P;
+  const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
+  if (c >= K) return;  // whole warps only: K/2 is a multiple of 32
+  const int gps = Lin >> P;  // groups per transform block
+  for (long grp = blockIdx.y; grp < ngroups; grp += gridDim.y) {
+    const long s = grp / gps;
+    const int g = static_cast<int>(grp - s * gps);
+    float a0[G], a1[G];
+    const TIn* src = in + ((s * Lin + (long)g * G) * K + c);
+#pragma unroll
+    for (int t = 0; t < G; ++t) {
+      const float2 v = load2(src + (long)t * K);
+      a0[t] = v.x;
+      a1[t] = v.y;
+    }
+    float* Tseq = T + (s * n) * (long)K + c;
+    unsigned* rm = rowmax ? rowmax + s * n : nullptr;
+#pragma unroll
+    for (int l = 1; l <= P; ++l) {
+      const int half = G >> l;
+      const int j = lvl0 + l;
+      const float nrm = haar_norm(j);
+      const int row0 = (n >> j) + g * half;
+#pragma unroll
+      for (int i = 0; i < half; ++i) {
+        const float d0 = (a0[2 * i] - a0[2 * i + 1]) * nrm;
+        const float d1 = (a1[2 * i] - a1[2 * i + 1]) * nrm;
+        const float s0 = a0[2 * i] + a0[2 * i + 1];
+        const float s1 = a1[2 * i] + a1[2 * i + 1];
+        a0[i] = s0;
+        a1[i] = s1;
+        store2(Tseq + (long)(row0 + i) * K, d0, d1);
+        if (rm) {
+          const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(d0), absbits(d1)));
+          if ((threadIdx.x & 31) == 0) atomicMax(rm + row0 + i, m);
+        }
+      }
+    }
+    if (aout) {
+      store2(aout + ((s * gps + g) * (long)K + c), a0[0], a1[0]);
+    } else {
+      const float nrm = haar_norm(lvl0 + P);
+      const float v0 = a0[0] * nrm, v1 = a1[0] * nrm;
+      store2(Tseq + (long)g * K, v0, v1);
+      if (rm) {
+        const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(v0), absbits(v1)));
+        if ((threadIdx.x & 31) == 0) atomicMax(rm + g, m);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Haar synthesis (L^-1 = L^T), P levels per pass, coarse to fine.  A thread owns two adjacent
+// output channels of one group: it starts from the group's coarse value, already carrying all
+// coarser contributions, and per level adds / subtracts the detail coefficient pre-multiplied
+// by 2^(-j/2):  v[2i] = v[i] + d'_j[i],  v[2i+1] = v[i] - d'_j[i].
+//   Yt    [nseq * n, N]            float, transformed domain (logical row order)
+//   ain   [nseq, n >> (jlo+P), N]  float partial sums from the coarser pass; nullptr in the
+//                                  first pass (the approximation rows of Yt are read instead)
+//   out   jlo > 0 : [nseq, n >> jlo, N] float partial sums for the next pass
+//         jlo == 0: Y [nseq * n, N] TOut, bias added
+// ------------------------------------------------------------------------------------------
+template <int P, typename TOut>
+__global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__ Yt, const float* __restrict__ ain,
+                                                       int n, int jlo, long ngroups, int N,
+                                                       const float* __restrict__ bias, void* __restrict__ out_) {
+  constexpr int G = 1 << P;
+  const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
+  if (c >= N) return;
+  const int gps = n >> (jlo + P);
+  float b0 = 0.f, b1 = 0.f;
+  if (jlo == 0 && bias != nullptr) {
+    b0 = bias[c];
+    b1 = bias[c + 1];
+  }
+  for (long grp = blockIdx.y; grp < ngroups; grp += gridDim.y) {
+    const long s = grp / gps;
+    const int g = static_cast<int>(grp - s * gps);
+    const float* Yseq = Yt + (s * n) * (long)N + c;
+    float v0[G], v1[G];
+    if (ain) {
+      const float2 a = load2(ain + ((s * gps + g) * (long)N + c));
+      v0[0] = a.x;
+      v1[0] = a.y;
+    } else {
+      const float nrm = haar_norm(jlo + P);
+      const float2 a = load2(Yseq + (long)g * N);
+      v0[0] = a.x * nrm;
+      v1[0] = a.y * nrm;
+    }
+#pragma unroll
+    for (int l = P; l >= 1; --l) {
+      const int cur = 1 << (P - l);
+      const int j = jlo + l;
+      const float nrm = haar_norm(j);
+      const int row0 = (n >> j) + g * cur;
+#pragma unroll
+      for (int i = cur - 1; i >= 0; --i) {
+        const float2 d = load2(Yseq + (long)(row0 + i) * N);
+        const float d0 = d.x * nrm, d1 = d.y * nrm;
+        const float p0 = v0[i], p1 = v1[i];
+        v0[2 * i] = p0 + d0;
+        v0[2 * i + 1] = p0 - d0;
+        v1[2 * i] = p1 + d1;
+        v1[2 * i + 1] = p1 - d1;
+      }
+    }
+    if (jlo == 0) {
+      TOut* dst = static_cast<TOut*>(out_) + ((s * n + (long)g * G) * N + c);
+#pragma unroll
+      for (int t = 0; t < G; ++t) store2(dst + (long)t * N, v0[t] + b0, v1[t] + b1);
+    } else {
+      float* dst = static_cast<float*>(out_) + ((s * (long)(n >> jlo) + (long)g * G) * N + c);
+#pragma unroll
+      for (int t = 0; t < G; ++t) store2(dst + (long)t * N, v0[t], v1[t]);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Row quantizer (Sec. 2.1, first equation, symmetric form) reading materialised T.
+// One CTA per transformed token: scale = absmax / qmax (IEEE fp32 division), codes =
+// clamp(rne(t * (1 / scale))).  Writes any of: the int8 operand row for the GEMM (a8), the
+// public packed outputs (q_hi rows as int8, q_lo rows as nibble pairs), the scale.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_quant_rows(const float* __restrict__ T, const unsigned* __restrict__ rowmax,
+                                                    int K, int n, int k_hi, int qmax_hi, int qmax_lo,
+                                                    int8_t* __restrict__ a8, int8_t* __restrict__ q_hi,
+                                                    uint8_t* __restrict__ q_lo, float* __restrict__ x_scale) {
+  const long r = blockIdx.x;
+  const long s = r / n;
+  const int i = static_cast<int>(r - s * n);
+  const bool hi = i < k_hi;
+  const float qmax = static_cast<float>(hi ? qmax_hi : qmax_lo);
+  const float amax = __uint_as_float(rowmax[r]);
+  const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
+  const float inv = __fdiv_rn(1.0f, scale);
+  if (threadIdx.x == 0) x_scale[r] = scale;
+  const float4* src = reinterpret_cast<const float4*>(T + r * (long)K);
+  char4* dst8 = a8 ? reinterpret_cast<char4*>(a8 + r * (long)K) : nullptr;
+  char4* dsth = (q_hi && hi) ? reinterpret_cast<char4*>(q_hi + (s * k_hi + i) * (long)K) : nullptr;
+  uint16_t* dstl =
+      (q_lo && !hi) ? reinterpret_cast<uint16_t*>(q_lo + (s * (n - k_hi) + (i - k_hi)) * (long)(K / 2)) : nullptr;
+  for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) {
+    const float4 t = src[k4];
+    int q0 = __float2int_rn(t.x * inv), q1 = __float2int_rn(t.y * inv);
+    int q2 = __float2int_rn(t.z * inv), q3 = __float2int_rn(t.w * inv);
+    const int qm = static_cast<int>(qmax);
+    q0 = max(-qm, min(qm, q0));
+    q1 = max(-qm, min(qm, q1));
+    q2 = max(-qm, min(qm, q2));
+    q3 = max(-qm, min(qm, q3));
+    const char4 c = make_char4((signed char)q0, (signed char)q1, (signed char)q2, (signed char)q3);
+    if (dst8) dst8[k4] = c;
+    if (dsth) dsth[k4] = c;
+    if (dstl)
+      dstl[k4] = static_cast<uint16_t>((q0 & 0xF) | ((q1 & 0xF) << 4) | ((q2 & 0xF) << 8) | ((q3 & 0xF) << 12));
+  }
+}
+
+// Sign-extend the two nibbles of a byte.
+__device__ __forceinline__ int nib_lo(uint32_t b) { return (static_cast<int>(b << 28)) >> 28; }
+__device__ __forceinline__ int nib_hi(uint32_t b) { return (static_cast<int>(b << 24)) >> 28; }
+
+// Public code format -> one int8 per code, logical token order.  One CTA per token.
+__global__ void __launch_bounds__(256) k_unpack_codes(const int8_t* __restrict__ q_hi, const uint8_t* __restrict__ q_lo,
+                                                      int K, int n, int k_hi, int8_t* __restrict__ out) {
+  const long r = blockIdx.x;
+  const long s = r / n;
+  const int i = static_cast<int>(r - s * n);
+  char4* dst = reinterpret_cast<char4*>(out + r * (long)K);
+  if (i < k_hi) {
+    const char4* src = reinterpret_cast<const char4*>(q_hi + (s * k_hi + i) * (long)K);
+    for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) dst[k4] = src[k4];
+  } else {
+    const uint16_t* src = reinterpret_cast<const uint16_t*>(q_lo + (s * (n - k_hi) + (i - k_hi)) * (long)(K / 2));
+    for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) {
+      const uint32_t u = src[k4];
+      dst[k4] = make_char4((signed char)nib_lo(u), (signed char)nib_hi(u), (signed char)nib_lo(u >> 8),
+                           (signed char)nib_hi(u >> 8));
+    }
+  }
+}
+
+// Packed 4-bit rows -> int8 rows (weights). One CTA per row.
+__global__ void __launch_bounds__(256) k_unpack_rows4(const uint8_t* __restrict__ packed, int K, int8_t* __restrict__ out) {
+  const long r = blockIdx.x;
+  const uint16_t* src = reinterpret_cast<const uint16_t*>(packed + r * (long)(K / 2));
+  char4* dst = reinterpret_cast<char4*>(out + r * (long)K);
+  for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) {
+    const uint32_t u = src[k4];
+    dst[k4] = make_char4((signed char)nib_lo(u), (signed char)nib_hi(u), (signed char)nib_lo(u >> 8),
+                         (signed char)nib_hi(u >> 8));
+  }
+}
+
+// Offline weight quantizer: per output channel absmax / qmax, round to nearest, packed nibbles.
+template <typename TW>
+__global__ void __launch_bounds__(256) k_quant_weights(const TW* __restrict__ W, int K, int qmax_w,
+                                                       uint8_t* __restrict__ wq, float* __restrict__ w_scale) {
+  __shared__ unsigned red[8];
+  const long r = blockIdx.x;
+  const TW* src = W + r * (long)K;
+  unsigned m = 0;
+  for (int k2 = threadIdx.x; k2 < K / 2; k2 += blockDim.x) {
+    const float2 v = load2(src + 2 * k2);
+    m = max(m, max(absbits(v.x), absbits(v.y)));
+  }
+  m = __reduce_max_sync(0xffffffffu, m);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = red[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) m = max(m, red[w]);
+  const float amax = __uint_as_float(m);
+  const float qmax = static_cast<float>(qmax_w);
+  const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
+  if (threadIdx.x == 0) w_scale[r] = scale;
+  uint8_t* dst = wq + r * (long)(K / 2);
+  for (int k2 = threadIdx.x; k2 < K / 2; k2 += blockDim.x) {
+    const float2 v = load2(src + 2 * k2);
+    // offline path: a true division keeps the codes identical to a plain w / scale
+    int q0 = max(-qmax_w, min(qmax_w, __float2int_rn(__fdiv_rn(v.x, scale))));
+    int q1 = max(-qmax_w, min(qmax_w, __float2int_rn(__fdiv_rn(v.y, scale))));
+    dst[k2] = static_cast<uint8_t>((q0 & 0xF) | ((q1 & 0xF) << 4));
+  }
+}
+
+}  // namespace stamp

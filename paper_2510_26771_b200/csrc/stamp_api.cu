@@ -1,0 +1,544 @@
+// Host layer of the STaMP CUDA library: argument validation, workspace layout, tensor maps,
+// kernel selection and launch.  Every extern "C" entry point of include/stamp.h is defined here.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+#include <unordered_map>
+
+#include "common.cuh"
+#include "k_gemm.cuh"
+#include "k_generic.cuh"
+#include "stamp.h"
+
+namespace stamp {
+
+static thread_local int t_launches = 0;
+
+#define STAMP_CHECK_LAUNCH()                                   \
+  do {                                                         \
+    ++t_launches;                                              \
+    if (cudaGetLastError() != cudaSuccess) return STAMP_ERR_CUDA; \
+  } while (0)
+
+static inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+static inline int ilog2(int v) {
+  int l = 0;
+  while ((1 << l) < v) ++l;
+  return l;
+}
+static inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+
+// ------------------------------------------------------------------------------------------
+// Validation: stamp_config + sizes -> Problem
+// ------------------------------------------------------------------------------------------
+static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool need_n, Problem* out) {
+  if (!cfg || !out) return STAMP_ERR_INVALID_ARG;
+  if (B <= 0 || L <= 0 || K <= 0 || (need_n && N <= 0)) return STAMP_ERR_INVALID_ARG;
+  if (cfg->transform < STAMP_T_IDENTITY || cfg->transform > STAMP_T_DCT2) return STAMP_ERR_INVALID_ARG;
+  if (cfg->block < 0 || cfg->levels < 0 || cfg->k_hi < 0 || cfg->reserved != 0) return STAMP_ERR_INVALID_ARG;
+  if (cfg->bits_hi != 8 || cfg->bits_lo != 4 || cfg->bits_w != 4) return STAMP_ERR_UNSUPPORTED;
+  if (cfg->act_gran != STAMP_G_PER_TOKEN || cfg->w_gran != STAMP_G_PER_CHANNEL) return STAMP_ERR_UNSUPPORTED;
+  const int n = cfg->block ? cfg->block : L;
+  if (!is_pow2(n) || L % n != 0) return STAMP_ERR_UNSUPPORTED;
+  if (cfg->k_hi > n) return STAMP_ERR_INVALID_ARG;
+  if (K % 128 != 0) return STAMP_ERR_UNSUPPORTED;
+  if (need_n && N % 8 != 0) return STAMP_ERR_UNSUPPORTED;
+  if ((long)B * L > (1L << 30)) return STAMP_ERR_UNSUPPORTED;
+  int levels = 0;
+  if (cfg->transform == STAMP_T_HAAR) {
+    const int full = ilog2(n);
+    levels = cfg->levels ? cfg->levels : full;
+    if (levels > full) return STAMP_ERR_UNSUPPORTED;
+  }
+  out->B = B;
+  out->L = L;
+  out->K = K;
+  out->N = need_n ? N : 0;
+  out->transform = cfg->transform;
+  out->n = n;
+  out->levels = levels;
+  out->k_hi = cfg->k_hi;
+  out->nseq = B * (L / n);
+  out->M = (long)B * L;
+  out->qmax_hi = (1 << (cfg->bits_hi - 1)) - 1;
+  out->qmax_lo = (1 << (cfg->bits_lo - 1)) - 1;
+  out->qmax_w = (1 << (cfg->bits_w - 1)) - 1;
+  return STAMP_OK;
+}
+
+static bool dtype_ok(int d) { return d == STAMP_F32 || d == STAMP_BF16; }
+
+// ------------------------------------------------------------------------------------------
+// Multi-pass plan for the Haar kernels: up to 5 levels per pass, finest first.
+// ------------------------------------------------------------------------------------------
+struct PassPlan {
+  int npass;
+  int p[8];
+};
+static PassPlan make_plan(int levels) {
+  PassPlan pl{};
+  int rem = levels;
+  if (rem == 0) {
+    pl.npass = 1;
+    pl.p[0] = 0;
+    return pl;
+  }
+  while (rem > 0) {
+    const int p = rem > 5 ? 5 : rem;
+    pl.p[pl.npass++] = p;
+    rem -= p;
+  }
+  return pl;
+}
+
+// ------------------------------------------------------------------------------------------
+// Workspace layout (one layout for all calls of a problem size).
+// ------------------------------------------------------------------------------------------
+struct Workspace {
+  size_t rowmax, xscale, T, ping, pong, a8, w8, yt, total;
+};
+static Workspace layout(const Problem& pb) {
+  Workspace w{};
+  const size_t M = (size_t)pb.M;
+  const size_t KN = (size_t)(pb.K > pb.N ? pb.K : pb.N);
+  const PassPlan pl = make_plan(pb.levels);
+  const size_t ping_rows = pl.npass > 1 ? (M >> pl.p[0]) : 0;
+  const size_t pong_rows = pl.npass > 2 ? (M >> (pl.p[0] + pl.p[1])) : 0;
+  size_t off = 0;
+  w.rowmax = off; off += align256(M * 4);
+  w.xscale = off; off += align256(M * 4);
+  w.T = off;      off += align256(M * (size_t)pb.K * 4);
+  w.ping = off;   off += align256(ping_rows * KN * 4);
+  w.pong = off;   off += align256(pong_rows * KN * 4);
+  w.a8 = off;     off += align256(M * (size_t)pb.K);
+  w.w8 = off;     off += align256((size_t)pb.N * pb.K);
+  w.yt = off;     off += align256(M * (size_t)pb.N * 4);
+  w.total = off;
+  return w;
+}
+static int check_ws(const Workspace& w, const void* ws, size_t ws_bytes) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < w.total) return STAMP_ERR_WORKSPACE;
+  return STAMP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Tensor maps (driver entry point fetched through the runtime; no link against libcuda).
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// int8 matrix [rows, K] row-major; box = 128 bytes of K x box_rows rows, 128-byte swizzle.
+static int make_tmap_i8(const void* base, long rows, int K, int box_rows, CUtensorMap* out) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return STAMP_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) != 0) return STAMP_ERR_INVALID_ARG;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K};
+  cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? STAMP_OK : STAMP_ERR_CUDA;
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+// ------------------------------------------------------------------------------------------
+// Launchers
+// ------------------------------------------------------------------------------------------
+template <int BN, int STAGES, int EPI>
+static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const GemmParams& gp, cudaStream_t st) {
+  using SM = GemmSmem<BN, STAGES>;
+  auto kern = k_gemm_i8<BN, STAGES, EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::DYN_BYTES) != cudaSuccess)
+      return STAMP_ERR_CUDA;
+    attr_set = true;
+  }
+  const int ch_tiles = (gp.n_out + GEMM_BM - 1) / GEMM_BM;
+  const int tok_tiles = (gp.m_tok + BN - 1) / BN;
+  const int tiles = ch_tiles * tok_tiles;
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  kern<<<grid, GEMM_THREADS, SM::DYN_BYTES, st>>>(tw, tx, gp);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// acc/out[tok, ch] from int8 operands a8 [M, K], w8 [N, K].
+static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K, const float* x_scale,
+                       const float* w_scale, void* out, int epi, cudaStream_t st) {
+  GemmParams gp{};
+  gp.n_out = N;
+  gp.m_tok = (int)M;
+  gp.k = K;
+  gp.x_scale = x_scale;
+  gp.w_scale = w_scale;
+  gp.out = out;
+  gp.group = 16;
+  CUtensorMap tw, tx;
+  int rc = make_tmap_i8(w8, N, K, GEMM_BM, &tw);
+  if (rc) return rc;
+  const bool wide = M >= 256;
+  rc = make_tmap_i8(a8, M, K, wide ? 256 : 128, &tx);
+  if (rc) return rc;
+  if (wide) {
+    if (epi == EPI_DEQUANT_F32) return launch_gemm_t<256, 4, EPI_DEQUANT_F32>(tw, tx, gp, st);
+    return launch_gemm_t<256, 4, EPI_RAW_I32>(tw, tx, gp, st);
+  }
+  if (epi == EPI_DEQUANT_F32) return launch_gemm_t<128, 6, EPI_DEQUANT_F32>(tw, tx, gp, st);
+  return launch_gemm_t<128, 6, EPI_RAW_I32>(tw, tx, gp, st);
+}
+
+template <typename TIn>
+static int launch_fwd_pass(int P, const TIn* in, int Lin, long ngroups, int K, float* T, int n, int lvl0, float* aout,
+                           unsigned* rowmax, cudaStream_t st) {
+  dim3 grid((K / 2 + 127) / 128, (unsigned)(ngroups < 32768 ? ngroups : 32768));
+  switch (P) {
+    case 0: k_haar_fwd_pass<0, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
+    case 1: k_haar_fwd_pass<1, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
+    case 2: k_haar_fwd_pass<2, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
+    case 3: k_haar_fwd_pass<3, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
+    case 4: k_haar_fwd_pass<4, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
+    default: k_haar_fwd_pass<5, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
+  }
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// T = L X (Haar or identity), fp32, logical order; optionally the per-row |T| maxima.
+static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, float* T, unsigned* rowmax,
+                                 float* ping, float* pong, cudaStream_t st) {
+  if (pb.transform == STAMP_T_DCT2) return STAMP_ERR_UNSUPPORTED;
+  if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+  const PassPlan pl = make_plan(pb.levels);
+  int lvl0 = 0;
+  int Lin = pb.n;
+  const float* cur = nullptr;
+  float* bufs[2] = {ping, pong};
+  for (int i = 0; i < pl.npass; ++i) {
+    const int P = pl.p[i];
+    const bool last = (i == pl.npass - 1);
+    float* aout = last ? nullptr : bufs[i & 1];
+    const long ngroups = (long)pb.nseq * (Lin >> P);
+    int rc;
+    if (i == 0) {
+      rc = (x_dtype == STAMP_BF16)
+               ? launch_fwd_pass<__nv_bfloat16>(P, static_cast<const __nv_bfloat16*>(X), Lin, ngroups, pb.K, T, pb.n,
+                                                lvl0, aout, rowmax, st)
+               : launch_fwd_pass<float>(P, static_cast<const float*>(X), Lin, ngroups, pb.K, T, pb.n, lvl0, aout,
+                                        rowmax, st);
+    } else {
+      rc = launch_fwd_pass<float>(P, cur, Lin, ngroups, pb.K, T, pb.n, lvl0, aout, rowmax, st);
+    }
+    if (rc) return rc;
+    cur = aout;
+    lvl0 += P;
+    Lin >>= P;
+  }
+  return STAMP_OK;
+}
+
+template <typename TOut>
+static int launch_inv_pass(int P, const float* Yt, const float* ain, int n, int jlo, long ngroups, int N,
+                           const float* bias, void* out, cudaStream_t st) {
+  dim3 grid((N / 2 + 127) / 128, (unsigned)(ngroups < 32768 ? ngroups : 32768));
+  switch (P) {
+    case 0: k_haar_inv_pass<0, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 1: k_haar_inv_pass<1, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 2: k_haar_inv_pass<2, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 3: k_haar_inv_pass<3, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 4: k_haar_inv_pass<4, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    default: k_haar_inv_pass<5, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
+  }
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// Y = L^T Yt + bias (Haar or identity), coarse passes first.
+static int run_inverse_generic(const Problem& pb, const float* Yt, const float* bias, void* Y, int y_dtype,
+                               float* ping, float* pong, cudaStream_t st) {
+  if (pb.transform == STAMP_T_DCT2) return STAMP_ERR_UNSUPPORTED;
+  const PassPlan pl = make_plan(pb.levels);
+  // forward pass i covered levels (sum p[0..i-1], sum p[0..i]]; run them in reverse
+  int jlo_of[8];
+  int acc = 0;
+  for (int i = 0; i < pl.npass; ++i) {
+    jlo_of[i] = acc;
+    acc += pl.p[i];
+  }
+  const float* ain = nullptr;
+  float* bufs[2] = {ping, pong};
+  for (int i = pl.npass - 1; i >= 0; --i) {
+    const int P = pl.p[i];
+    const int jlo = jlo_of[i];
+    const long ngroups = (long)pb.nseq * (pb.n >> (jlo + P));
+    int rc;
+    if (i == 0) {
+      rc = (y_dtype == STAMP_BF16)
+               ? launch_inv_pass<__nv_bfloat16>(P, Yt, ain, pb.n, jlo, ngroups, pb.N, bias, Y, st)
+               : launch_inv_pass<float>(P, Yt, ain, pb.n, jlo, ngroups, pb.N, bias, Y, st);
+    } else {
+      // partial sums of level jlo have (M >> jlo) rows: the buffer sized for forward pass i-1's output
+      float* aout = bufs[(i - 1) & 1];
+      rc = launch_inv_pass<float>(P, Yt, ain, pb.n, jlo, ngroups, pb.N, nullptr, aout, st);
+      if (rc) return rc;
+      ain = aout;
+      continue;
+    }
+    if (rc) return rc;
+  }
+  return STAMP_OK;
+}
+
+static int run_quant_rows(const Problem& pb, const float* T, const unsigned* rowmax, int8_t* a8, void* q_hi,
+                          void* q_lo, float* x_scale, cudaStream_t st) {
+  k_quant_rows<<<(unsigned)pb.M, 256, 0, st>>>(T, rowmax, pb.K, pb.n, pb.k_hi, pb.qmax_hi, pb.qmax_lo, a8,
+                                                static_cast<int8_t*>(q_hi), static_cast<uint8_t*>(q_lo), x_scale);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+static int run_unpack_codes(const Problem& pb, const void* q_hi, const void* q_lo, int8_t* out, cudaStream_t st) {
+  k_unpack_codes<<<(unsigned)pb.M, 256, 0, st>>>(static_cast<const int8_t*>(q_hi), static_cast<const uint8_t*>(q_lo),
+                                                  pb.K, pb.n, pb.k_hi, out);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// Resolve the weight operand to int8 [N, K]: either the caller's prepared copy or an expansion
+// of the packed codes into the workspace.
+static int weights_as_int8(const Problem& pb, const void* w, int w_format, int8_t* w8_ws, const int8_t** out,
+                           cudaStream_t st) {
+  if (w_format == STAMP_W_INT8) {
+    *out = static_cast<const int8_t*>(w);
+    return STAMP_OK;
+  }
+  if (w_format != STAMP_W_PACKED4) return STAMP_ERR_INVALID_ARG;
+  k_unpack_rows4<<<(unsigned)pb.N, 256, 0, st>>>(static_cast<const uint8_t*>(w), pb.K, w8_ws);
+  STAMP_CHECK_LAUNCH();
+  *out = w8_ws;
+  return STAMP_OK;
+}
+
+}  // namespace stamp
+
+// ============================================================================================
+// C ABI
+// ============================================================================================
+using namespace stamp;
+
+extern "C" {
+
+int stamp_workspace_bytes(const stamp_config* cfg, int B, int L, int K, int N, size_t* out_bytes) {
+  if (!out_bytes) return STAMP_ERR_INVALID_ARG;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, N, true, &pb);
+  if (rc) return rc;
+  *out_bytes = layout(pb).total;
+  return STAMP_OK;
+}
+
+int stamp_quantize_weights(const stamp_config* cfg, const void* W, int w_dtype, int N, int K, void* wq,
+                           float* w_scale, void* stream) {
+  t_launches = 0;
+  if (!cfg || !W || !wq || !w_scale || N <= 0 || K <= 0 || !dtype_ok(w_dtype)) return STAMP_ERR_INVALID_ARG;
+  if (cfg->bits_w != 4 || cfg->w_gran != STAMP_G_PER_CHANNEL || K % 128 != 0) return STAMP_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (w_dtype == STAMP_BF16)
+    k_quant_weights<__nv_bfloat16><<<N, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W), K, 7,
+                                                      static_cast<uint8_t*>(wq), w_scale);
+  else
+    k_quant_weights<float><<<N, 256, 0, st>>>(static_cast<const float*>(W), K, 7, static_cast<uint8_t*>(wq), w_scale);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+int stamp_prepare_weights(const stamp_config* cfg, const void* wq_packed, int N, int K, void* w_int8, void* stream) {
+  t_launches = 0;
+  if (!cfg || !wq_packed || !w_int8 || N <= 0 || K <= 0) return STAMP_ERR_INVALID_ARG;
+  if (cfg->bits_w != 4 || K % 128 != 0) return STAMP_ERR_UNSUPPORTED;
+  k_unpack_rows4<<<N, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t*>(wq_packed), K,
+                                                                    static_cast<int8_t*>(w_int8));
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, void* q_hi, void* q_lo,
+                   float* x_scale, void* ws, size_t ws_bytes, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, 0, false, &pb);
+  if (rc) return rc;
+  if (!X || !x_scale || !dtype_ok(x_dtype)) return STAMP_ERR_INVALID_ARG;
+  if ((pb.n_hi_rows() > 0 && !q_hi) || (pb.n_lo_rows() > 0 && !q_lo)) return STAMP_ERR_INVALID_ARG;
+  const Workspace w = layout(pb);
+  if ((rc = check_ws(w, ws, ws_bytes))) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* T = reinterpret_cast<float*>(base + w.T);
+  unsigned* rowmax = reinterpret_cast<unsigned*>(base + w.rowmax);
+  rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
+                             reinterpret_cast<float*>(base + w.pong), st);
+  if (rc) return rc;
+  return run_quant_rows(pb, T, rowmax, nullptr, q_hi, q_lo, x_scale, st);
+}
+
+int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, const float* x_scale, const void* w,
+                 int w_format, const float* w_scale, int B, int L, int K, int N, float* Yt, void* ws, size_t ws_bytes,
+                 void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, N, true, &pb);
+  if (rc) return rc;
+  if (!x_scale || !w || !w_scale || !Yt) return STAMP_ERR_INVALID_ARG;
+  if ((pb.n_hi_rows() > 0 && !q_hi) || (pb.n_lo_rows() > 0 && !q_lo)) return STAMP_ERR_INVALID_ARG;
+  const Workspace wl = layout(pb);
+  if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
+  if ((rc = run_unpack_codes(pb, q_hi, q_lo, a8, st))) return rc;
+  const int8_t* w8 = nullptr;
+  if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
+  return launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, Yt, EPI_DEQUANT_F32, st);
+}
+
+int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
+                  int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  // the inverse does not touch K: validate with a stand-in that satisfies the K rule
+  int rc = resolve(cfg, B, L, 128, N, true, &pb);
+  if (rc) return rc;
+  if (!Yt || !Y || !dtype_ok(y_dtype)) return STAMP_ERR_INVALID_ARG;
+  const Workspace wl = layout(pb);
+  if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  return run_inverse_generic(pb, Yt, bias, Y, y_dtype, reinterpret_cast<float*>(base + wl.ping),
+                             reinterpret_cast<float*>(base + wl.pong), static_cast<cudaStream_t>(stream));
+}
+
+int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, const void* w, int w_format,
+                       const float* w_scale, const float* bias, int B, int L, int K, int N, void* Y, int y_dtype,
+                       void* ws, size_t ws_bytes, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, N, true, &pb);
+  if (rc) return rc;
+  if (!X || !w || !w_scale || !Y || !dtype_ok(x_dtype) || !dtype_ok(y_dtype)) return STAMP_ERR_INVALID_ARG;
+  const Workspace wl = layout(pb);
+  if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* T = reinterpret_cast<float*>(base + wl.T);
+  unsigned* rowmax = reinterpret_cast<unsigned*>(base + wl.rowmax);
+  float* ping = reinterpret_cast<float*>(base + wl.ping);
+  float* pong = reinterpret_cast<float*>(base + wl.pong);
+  int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
+  float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
+  float* yt = reinterpret_cast<float*>(base + wl.yt);
+  if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, st))) return rc;
+  if ((rc = run_quant_rows(pb, T, rowmax, a8, nullptr, nullptr, x_scale, st))) return rc;
+  const int8_t* w8 = nullptr;
+  if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
+  if ((rc = launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_F32, st))) return rc;
+  return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, st);
+}
+
+int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, float* T, void* ws,
+                          size_t ws_bytes, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, 0, false, &pb);
+  if (rc) return rc;
+  if (!X || !T || !dtype_ok(x_dtype)) return STAMP_ERR_INVALID_ARG;
+  const Workspace wl = layout(pb);
+  if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  return run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + wl.ping),
+                               reinterpret_cast<float*>(base + wl.pong), static_cast<cudaStream_t>(stream));
+}
+
+int stamp_debug_unpack_codes(const stamp_config* cfg, const void* q_hi, const void* q_lo, int B, int L, int K,
+                             int8_t* codes, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, 0, false, &pb);
+  if (rc) return rc;
+  if (!codes) return STAMP_ERR_INVALID_ARG;
+  if ((pb.n_hi_rows() > 0 && !q_hi) || (pb.n_lo_rows() > 0 && !q_lo)) return STAMP_ERR_INVALID_ARG;
+  return run_unpack_codes(pb, q_hi, q_lo, codes, static_cast<cudaStream_t>(stream));
+}
+
+int stamp_debug_gemm_i32(const stamp_config* cfg, const void* q_hi, const void* q_lo, const void* w, int w_format,
+                         int B, int L, int K, int N, int32_t* acc, void* ws, size_t ws_bytes, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, N, true, &pb);
+  if (rc) return rc;
+  if (!w || !acc) return STAMP_ERR_INVALID_ARG;
+  if ((pb.n_hi_rows() > 0 && !q_hi) || (pb.n_lo_rows() > 0 && !q_lo)) return STAMP_ERR_INVALID_ARG;
+  const Workspace wl = layout(pb);
+  if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
+  if ((rc = run_unpack_codes(pb, q_hi, q_lo, a8, st))) return rc;
+  const int8_t* w8 = nullptr;
+  if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
+  return launch_gemm(a8, w8, pb.M, N, K, nullptr, nullptr, acc, EPI_RAW_I32, st);
+}
+
+int stamp_last_device_status(void* stream, int* status) {
+  if (!status) return STAMP_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return STAMP_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)) != cudaSuccess) return STAMP_ERR_CUDA;
+  if (v != 0) {
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return STAMP_ERR_CUDA;
+  }
+  *status = v;
+  return STAMP_OK;
+}
+
+int stamp_last_launch_count(void) { return t_launches; }
+
+const char* stamp_status_string(int status) {
+  switch (status) {
+    case STAMP_OK: return "ok";
+    case STAMP_ERR_INVALID_ARG: return "invalid argument";
+    case STAMP_ERR_UNSUPPORTED: return "unsupported shape or configuration";
+    case STAMP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case STAMP_ERR_CUDA: return "CUDA call failed";
+    case STAMP_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,162 @@
+"""Parity of the CUDA path against the CPU oracle, stage by stage, through the C ABI.
+Tolerances: T within 1e-5 relative; codes bit-exact except at most 1e-5 of them off by +-1
+(ties at rounding boundaries); int32 accumulators bit-exact given identical codes; final fp32
+output within 1e-3 relative Frobenius error of the fp64 oracle."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2510_26771_b200 import inputs as gen
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+T_TOL = 1e-5
+CODE_FRAC = 1e-5
+Y_TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def st():
+    import torch
+    from paper_2510_26771_b200 import binding
+    assert torch.cuda.is_available()
+    binding.lib()
+    return binding
+
+
+def _cfg_struct(st, cfg):
+    return st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi)
+
+
+def _oracle_all(oracle, cfg, X, W, bias=None, want=("T", "x_scale", "q", "w_scale", "wq", "acc", "Yt", "Y")):
+    return oracle.stamp_linear(X, W, bias, transform=cfg.transform, block=cfg.block, levels=cfg.levels,
+                               k_hi=cfg.k_hi, want=want)
+
+
+def _allowed(count):
+    return int(math.floor(CODE_FRAC * count))
+
+
+CASES = {
+    "tiny": gen.config_tiny(),
+    # several channel and token tiles with ragged tails (N not a multiple of 128, 3 K blocks)
+    "ragged": gen.scaled(gen.config_llm_up(), B=2, L=512, K=384, N=392, k_hi=16),
+    # fixed-depth Haar on a 2-D-grid-like input, block smaller than the sequence
+    "blocked": gen.scaled(gen.config_dit_proj(), B=1, L=1024, K=256, N=136, grid=32, block=256, levels=6, k_hi=4),
+    # one-level transform and the identity (pure mixed-precision quantization)
+    "one_level": gen.scaled(gen.config_sweep(512, 2048), L=256, K=128, N=64, levels=1, k_hi=128),
+    "identity": gen.scaled(gen.config_sweep(512, 2048), L=192 + 64, K=256, N=128, transform=gen.T_IDENTITY, k_hi=8),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_stagewise_parity(st, oracle, name):
+    import torch
+    cfg = CASES[name]
+    c = _cfg_struct(st, cfg)
+    X, W, bias = gen.make_activation(cfg), gen.make_weight(cfg), gen.make_bias(cfg)
+    ref = _oracle_all(oracle, cfg, X, W, bias)
+    B, L, K, N = cfg.B, cfg.L, cfg.K, cfg.N
+    Xd, Wd = H.to_device(X, cfg.dtype), H.to_device(W, cfg.dtype)
+    bd = torch.from_numpy(bias).cuda()
+    ws = st.alloc_workspace(c, B, L, K, N)
+
+    # a1: transform
+    T = st.stamp_debug_transform(c, Xd, ws).cpu().numpy().reshape(-1, K).astype(np.float64)
+    row_max = np.abs(ref["T"]).max(axis=1, keepdims=True)
+    assert np.all(np.abs(T - ref["T"]) <= T_TOL * np.maximum(row_max, 1e-30))
+    assert H.rel_fro(T, ref["T"]) <= T_TOL
+
+    # a2-a3: scales and codes
+    q_hi, q_lo, xs = st.stamp_quantize(c, Xd, ws)
+    codes = st.stamp_debug_unpack_codes(c, q_hi, q_lo, B, L, K).cpu().numpy().reshape(-1, K)
+    assert np.allclose(xs.cpu().numpy().reshape(-1), ref["x_scale"], rtol=1e-6, atol=0)
+    bad, worst = H.code_mismatch(codes, ref["q"])
+    assert worst <= 1 and bad <= _allowed(codes.size), (bad, worst, codes.size)
+
+    # a4: weights
+    wq, wsc = st.stamp_quantize_weights(c, Wd)
+    w8 = st.stamp_prepare_weights(c, wq)
+    assert np.array_equal(wsc.cpu().numpy(), ref["w_scale"])
+    bad, worst = H.code_mismatch(w8.cpu().numpy(), ref["wq"])
+    assert worst <= 1 and bad <= _allowed(w8.numel()), (bad, worst)
+    assert np.array_equal(wq.cpu().numpy(), H.pack_nibbles(w8.cpu().numpy()))
+
+    # a5: integer GEMM, fed the ORACLE's codes: accumulators must be bit-identical
+    oq_hi, oq_lo = H.pack_codes(ref["q"], cfg.block_len, cfg.k_hi)
+    owq = torch.from_numpy(H.pack_nibbles(ref["wq"])).cuda()
+    oqh, oql = torch.from_numpy(oq_hi).cuda(), torch.from_numpy(oq_lo).cuda()
+    acc = st.stamp_debug_gemm_i32(c, oqh, oql, owq, st.W_PACKED4, B, L, K, N, ws).cpu().numpy()
+    assert np.array_equal(acc, ref["acc"])
+    ow8 = torch.from_numpy(ref["wq"]).cuda()
+    acc = st.stamp_debug_gemm_i32(c, oqh, oql, ow8, st.W_INT8, B, L, K, N, ws).cpu().numpy()
+    assert np.array_equal(acc, ref["acc"])
+
+    # a6: de-quantized transformed-domain output from the oracle's codes and scales
+    oxs = torch.from_numpy(ref["x_scale"]).cuda()
+    ows = torch.from_numpy(ref["w_scale"]).cuda()
+    Yt = st.stamp_linear(c, oqh, oql, oxs, owq, st.W_PACKED4, ows, B, L, K, N, ws).cpu().numpy().reshape(-1, N)
+    assert H.rel_fro(Yt, ref["Yt"]) <= 1e-6
+
+    # a7-a8: inverse transform + bias from the oracle's Yt
+    Ytd = torch.from_numpy(ref["Yt"].astype(np.float32)).cuda().reshape(B, L, N)
+    Y = st.stamp_inverse(c, Ytd, bd, ws).cpu().numpy().reshape(-1, N)
+    assert H.rel_fro(Y, ref["Y"]) <= 1e-6
+    Yb = st.stamp_inverse(c, Ytd, bd, ws, out_dtype=torch.bfloat16).float().cpu().numpy().reshape(-1, N)
+    ref_bf16 = gen.round_to_bf16(ref["Y"].astype(np.float32))
+    # bf16 output: compare with the oracle's output rounded to bf16, within one bf16 ulp
+    assert np.all(np.abs(Yb - ref_bf16) <= np.abs(ref_bf16) * 2.0 ** -7 + 1e-30)
+
+    # whole layer, chained calls and the fused call
+    Yt2 = st.stamp_linear(c, q_hi, q_lo, xs, wq, st.W_PACKED4, wsc, B, L, K, N, ws)
+    Y2 = st.stamp_inverse(c, Yt2, bd, ws).cpu().numpy().reshape(-1, N)
+    assert H.rel_fro(Y2, ref["Y"]) <= Y_TOL
+    for wfmt, wbuf in ((st.W_PACKED4, wq), (st.W_INT8, w8)):
+        Y3 = st.stamp_linear_fused(c, Xd, wbuf, wfmt, wsc, bd, ws).cpu().numpy().reshape(-1, N)
+        assert H.rel_fro(Y3, ref["Y"]) <= Y_TOL
+    assert st.stamp_last_launch_count() > 0
+    assert st.stamp_last_device_status() == 0
+
+
+def test_transform_then_inverse_is_identity(st):
+    """Quantizers off: L^T (L X) = X on the device (uses the activation as its own 'output')."""
+    import torch
+    cfg = gen.scaled(gen.config_llm_up(), B=1, L=2048, K=256, N=256)
+    c = _cfg_struct(st, cfg)
+    X = gen.make_activation(cfg)
+    ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+    T = st.stamp_debug_transform(c, H.to_device(X, cfg.dtype), ws)
+    back = st.stamp_inverse(c, T, None, ws).cpu().numpy()
+    assert np.max(np.abs(back - X)) <= 2e-6 * np.max(np.abs(X))
+    # energy preservation on the device result
+    e_t = float((T.double() ** 2).sum())
+    e_x = float((X.astype(np.float64) ** 2).sum())
+    assert abs(e_t - e_x) <= 1e-6 * e_x
+
+
+def test_edge_cases(st, oracle):
+    """Zero activations (scale 1, codes 0), k_hi = 0 and k_hi = block."""
+    import torch
+    base = gen.scaled(gen.config_tiny(), L=128, K=128, N=64, levels=0)
+    for k_hi in (0, 128):
+        cfg = gen.scaled(base, k_hi=k_hi)
+        c = _cfg_struct(st, cfg)
+        X, W = gen.make_activation(cfg), gen.make_weight(cfg)
+        ref = _oracle_all(oracle, cfg, X, W, want=("q", "Y"))
+        ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+        Xd, Wd = H.to_device(X, cfg.dtype), H.to_device(W, cfg.dtype)
+        q_hi, q_lo, xs = st.stamp_quantize(c, Xd, ws)
+        codes = st.stamp_debug_unpack_codes(c, q_hi, q_lo, cfg.B, cfg.L, cfg.K).cpu().numpy().reshape(-1, cfg.K)
+        bad, worst = H.code_mismatch(codes, ref["q"])
+        assert worst <= 1 and bad <= 1
+        wq, wsc = st.stamp_quantize_weights(c, Wd)
+        Y = st.stamp_linear_fused(c, Xd, wq, st.W_PACKED4, wsc, None, ws).cpu().numpy().reshape(-1, cfg.N)
+        assert H.rel_fro(Y, ref["Y"]) <= Y_TOL
+    cfg = base
+    c = _cfg_struct(st, cfg)
+    ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+    Xz = torch.zeros((1, cfg.L, cfg.K), device="cuda")
+    q_hi, q_lo, xs = st.stamp_quantize(c, Xz, ws)
+    assert torch.all(xs == 1.0) and not q_hi.any() and not q_lo.any()
