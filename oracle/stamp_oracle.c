@@ -304,8 +304,13 @@ int oracle_bit_map(int L, int n, int k_hi, int bits_hi, int bits_lo, int32_t* bi
  *   amax  = max_j |t_j|                        (fp64)
  *   scale = (float)amax / (float)qmax          (evaluated in fp32: the scale is an fp32
  *                                               output of the method); amax == 0 -> scale 1
- *   q_j   = clamp(rne(t_j / scale), -qmax, qmax),   qmax = 2^(bits-1) - 1
- * rne = round half to even (rint in the default rounding mode).
+ *   q_j   = clamp(rne((float)t_j / scale), -qmax, qmax),   qmax = 2^(bits-1) - 1
+ * rne = round half to even (rintf in the default rounding mode).
+ * The rounding decision is taken in fp32: the transformed value is rounded to fp32 and
+ * divided by the fp32 scale with an IEEE fp32 division.  The paper fixes no precision for this
+ * step; low-precision inputs (bf16 activations and weights) land EXACTLY on rounding
+ * boundaries often (whenever absmax has a mantissa divisible by qmax), so the precision in
+ * which the tie is seen decides the code, and fp32 is the precision of the scale itself.
  * bits_per_row has `period` entries and row r uses bits_per_row[r % period].
  * ------------------------------------------------------------------------------------------ */
 int oracle_quantize_rows(const double* T, long rows, int K, const int32_t* bits_per_row, int period,
@@ -324,11 +329,10 @@ int oracle_quantize_rows(const double* T, long rows, int K, const int32_t* bits_
     float s = (amax > 0.0) ? ((float)amax / qmaxf) : 1.0f;
     if (!(s > 0.0f)) s = 1.0f; /* amax so small that the fp32 scale underflowed */
     scale[r] = s;
-    double sd = (double)s, qmax = (double)qmaxf;
     for (int j = 0; j < K; ++j) {
-      double q = rint(t[j] / sd);
-      if (q > qmax) q = qmax;
-      if (q < -qmax) q = -qmax;
+      float q = rintf((float)t[j] / s);
+      if (q > qmaxf) q = qmaxf;
+      if (q < -qmaxf) q = -qmaxf;
       codes[(size_t)r * K + j] = (int8_t)q;
     }
   }
@@ -350,11 +354,10 @@ int oracle_quantize_rows_f32in(const float* W, long rows, int K, int bits, float
     float s = (amax > 0.0) ? ((float)amax / qmaxf) : 1.0f;
     if (!(s > 0.0f)) s = 1.0f;
     scale[r] = s;
-    double sd = (double)s, qmax = (double)qmaxf;
     for (int j = 0; j < K; ++j) {
-      double q = rint((double)t[j] / sd);
-      if (q > qmax) q = qmax;
-      if (q < -qmax) q = -qmax;
+      float q = rintf(t[j] / s);
+      if (q > qmaxf) q = qmaxf;
+      if (q < -qmaxf) q = -qmaxf;
       codes[(size_t)r * K + j] = (int8_t)q;
     }
   }

@@ -29,17 +29,26 @@ struct Problem {
   long n_lo_rows() const { return M - n_hi_rows(); }
 };
 
-// 2^(-j/2) in fp32: an exact power of two for even j, float(1/sqrt 2) scaled exactly for odd j.
-__host__ __device__ __forceinline__ float haar_norm(int j) {
-  const float base = (j & 1) ? 0.70710678118654752440f : 1.0f;
-#ifdef __CUDA_ARCH__
-  return __int_as_float(__float_as_int(base) - ((j >> 1) << 23));
-#else
-  float r = base;
-  for (int i = 0; i < (j >> 1); ++i) r *= 0.5f;
-  return r;
-#endif
+// Multiplication by 2^(-j/2).  Even j: an exact power of two.  Odd j: 1/sqrt(2) is split into
+// an fp32 head and tail, v * head + v * tail in one FMA, so the product is rounded once (to within
+// a hair of the correctly rounded v / sqrt 2) instead of inheriting the constant's rounding error.
+struct HaarNorm {
+  float hi, lo;
+};
+__host__ __device__ __forceinline__ HaarNorm haar_norm(int j) {
+  HaarNorm h;
+  float p = 1.0f;
+  for (int i = 0; i < (j >> 1); ++i) p *= 0.5f;  // unrolled / folded where j is a constant
+  if (j & 1) {
+    h.hi = 0.707106769084930419921875f * p;       // fp32(1/sqrt 2)
+    h.lo = 1.2101617101e-8f * p;                  // 1/sqrt 2 - fp32(1/sqrt 2)
+  } else {
+    h.hi = p;
+    h.lo = 0.0f;
+  }
+  return h;
 }
+__device__ __forceinline__ float mul_norm(float v, const HaarNorm& h) { return fmaf(v, h.hi, v * h.lo); }
 
 // Two adjacent channels of one token as floats.
 __device__ __forceinline__ float2 load2(const float* p) { return *reinterpret_cast<const float2*>(p); }

@@ -46,12 +46,12 @@ __global__ void __launch_bounds__(128) k_haar_fwd_pass(const TIn* __restrict__ i
     for (int l = 1; l <= P; ++l) {
       const int half = G >> l;
       const int j = lvl0 + l;
-      const float nrm = haar_norm(j);
+      const HaarNorm nrm = haar_norm(j);
       const int row0 = (n >> j) + g * half;
 #pragma unroll
       for (int i = 0; i < half; ++i) {
-        const float d0 = (a0[2 * i] - a0[2 * i + 1]) * nrm;
-        const float d1 = (a1[2 * i] - a1[2 * i + 1]) * nrm;
+        const float d0 = mul_norm(a0[2 * i] - a0[2 * i + 1], nrm);
+        const float d1 = mul_norm(a1[2 * i] - a1[2 * i + 1], nrm);
         const float s0 = a0[2 * i] + a0[2 * i + 1];
         const float s1 = a1[2 * i] + a1[2 * i + 1];
         a0[i] = s0;
@@ -66,8 +66,8 @@ __global__ void __launch_bounds__(128) k_haar_fwd_pass(const TIn* __restrict__ i
     if (aout) {
       store2(aout + ((s * gps + g) * (long)K + c), a0[0], a1[0]);
     } else {
-      const float nrm = haar_norm(lvl0 + P);
-      const float v0 = a0[0] * nrm, v1 = a1[0] * nrm;
+      const HaarNorm nrm = haar_norm(lvl0 + P);
+      const float v0 = mul_norm(a0[0], nrm), v1 = mul_norm(a1[0], nrm);
       store2(Tseq + (long)g * K, v0, v1);
       if (rm) {
         const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(v0), absbits(v1)));
@@ -111,21 +111,21 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
       v0[0] = a.x;
       v1[0] = a.y;
     } else {
-      const float nrm = haar_norm(jlo + P);
+      const HaarNorm nrm = haar_norm(jlo + P);
       const float2 a = load2(Yseq + (long)g * N);
-      v0[0] = a.x * nrm;
-      v1[0] = a.y * nrm;
+      v0[0] = mul_norm(a.x, nrm);
+      v1[0] = mul_norm(a.y, nrm);
     }
 #pragma unroll
     for (int l = P; l >= 1; --l) {
       const int cur = 1 << (P - l);
       const int j = jlo + l;
-      const float nrm = haar_norm(j);
+      const HaarNorm nrm = haar_norm(j);
       const int row0 = (n >> j) + g * cur;
 #pragma unroll
       for (int i = cur - 1; i >= 0; --i) {
         const float2 d = load2(Yseq + (long)(row0 + i) * N);
-        const float d0 = d.x * nrm, d1 = d.y * nrm;
+        const float d0 = mul_norm(d.x, nrm), d1 = mul_norm(d.y, nrm);
         const float p0 = v0[i], p1 = v1[i];
         v0[2 * i] = p0 + d0;
         v0[2 * i + 1] = p0 - d0;
@@ -143,6 +143,15 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
       for (int t = 0; t < G; ++t) store2(dst + (long)t * N, v0[t], v1[t]);
     }
   }
+}
+
+// t / scale from a pre-computed reciprocal plus one Newton correction: q0 = t * inv,
+// q0 + (t - q0 * scale) * inv.  Two FMAs instead of a division, and the quotient is the correctly
+// rounded one except in rare half-ulp cases, so codes only differ from a true division when the
+// quotient itself sits within one fp32 ulp of a rounding boundary.
+__device__ __forceinline__ float div_by_scale(float t, float scale, float inv) {
+  const float q0 = t * inv;
+  return fmaf(fmaf(-q0, scale, t), inv, q0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -171,8 +180,8 @@ __global__ void __launch_bounds__(256) k_quant_rows(const float* __restrict__ T,
       (q_lo && !hi) ? reinterpret_cast<uint16_t*>(q_lo + (s * (n - k_hi) + (i - k_hi)) * (long)(K / 2)) : nullptr;
   for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) {
     const float4 t = src[k4];
-    int q0 = __float2int_rn(t.x * inv), q1 = __float2int_rn(t.y * inv);
-    int q2 = __float2int_rn(t.z * inv), q3 = __float2int_rn(t.w * inv);
+    int q0 = __float2int_rn(div_by_scale(t.x, scale, inv)), q1 = __float2int_rn(div_by_scale(t.y, scale, inv));
+    int q2 = __float2int_rn(div_by_scale(t.z, scale, inv)), q3 = __float2int_rn(div_by_scale(t.w, scale, inv));
     const int qm = static_cast<int>(qmax);
     q0 = max(-qm, min(qm, q0));
     q1 = max(-qm, min(qm, q1));

@@ -311,7 +311,8 @@ def _python_loop_layer(X, W, bias, n, levels, k_hi):
     def quant(row, qmax):
         amax = max(abs(x) for x in row)
         s = float(np.float32(amax) / np.float32(qmax)) if amax > 0 else 1.0
-        return [max(-qmax, min(qmax, int(round(x / s)))) for x in row], s   # round(): half to even
+        # the rounding decision is taken in fp32 (np.rint: half to even)
+        return [max(-qmax, min(qmax, int(np.rint(np.float32(x) / np.float32(s))))) for x in row], s
 
     qs = [quant(T[i], 127 if (i % n) < k_hi else 7) for i in range(L)]
     ws = [quant(W[c], 7) for c in range(N)]
