@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the STaMP-quantized linear layer on B200.
+
+A step is one pass of the whole hot path -- sequence transform, per-token mixed-precision
+quantization, int8 tensor-core GEMM, de-quantization, inverse transform, bias -- over one
+synthetic activation batch, through the C ABI (stamp_linear_fused).  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference] [--workload NAME]
+
+N > 1 (launched by torch.distributed.run) runs N independent replicas, one per GPU: the layer
+has no cross-GPU exchange, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_26771_b200 import inputs as gen  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_I8_OVER_BF16 = 2.0      # dense tensor peaks: 4.5 POPS int8 vs 2.25 PFLOPS bf16
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None until
+# a capture of that workload exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def workloads():
+    w = dict(gen.named_configs())
+    for L in gen.SWEEP_L:
+        for D in gen.SWEEP_D:
+            c = gen.config_sweep(L, D)
+            w[c.name] = c
+    return w
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_burst": float(p["bf16_tflops"]),
+                "bf16_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_burst": FALLBACK_BF16_TFLOPS, "bf16_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the GPU is under load."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.tmp,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            # samples under load = the upper half of the observed clocks (idle samples sit at the floor)
+            out["sm_mhz"] = statistics.median(sorted(sm)[len(sm) // 2:])
+            out["sm_max_mhz"] = max(smax)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def cpu_oracle_sample(cfg, seconds_target=15.0):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: all tokens and
+    features, a subset of output channels chosen so that the run takes roughly seconds_target."""
+    from oracle import stamp_oracle as orc
+    orc.build()
+    X = gen.make_activation(cfg)
+    def run(ncol):
+        Wc = gen.make_weight(cfg, np.arange(ncol))
+        t0 = time.perf_counter()
+        orc.stamp_linear(X, Wc, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi,
+                         want=("Y",))
+        return time.perf_counter() - t0
+    # two probes separate the fixed cost (transform + quantizer) from the per-channel cost (GEMM, inverse)
+    c1, c2 = min(cfg.N, 8), min(cfg.N, 64)
+    t1, t2 = run(c1), run(c2)
+    per_col = max((t2 - t1) / max(c2 - c1, 1), 1e-6)
+    fixed = max(t1 - per_col * c1, 0.0)
+    ncols = int(min(cfg.N, max(c2, (seconds_target - fixed) / per_col)))
+    ncols = max(8, (ncols // 8) * 8)
+    W = gen.make_weight(cfg, np.arange(ncols))
+    t0 = time.perf_counter()
+    orc.stamp_linear(X, W, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi,
+                     want=("Y",))
+    dt = time.perf_counter() - t0
+    tops = 2.0 * cfg.M * ncols * cfg.K / dt / 1e12
+    return {"value": tops, "unit": "TOPS", "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"all {cfg.M} tokens x {cfg.K} features, {ncols} of {cfg.N} output channels, "
+                      f"{dt:.1f} s of oracle time"}, (X, W, ncols)
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import stamp_oracle as orc
+    base, (X, W, ncols) = cpu_oracle_sample(cfg, seconds_target=8.0)
+
+    def step():
+        orc.stamp_linear(X, W, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi,
+                         want=("Y",))
+    for _ in range(min(args.warmup, 1)):
+        step()
+    steps = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    tops = 2.0 * cfg.M * ncols * cfg.K / dt / 1e12
+    line = {"impl": "reference", "metric": "stamp_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "K": cfg.K, "N": cfg.N,
+                       "sample_output_channels": ncols},
+            "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": base["cores"], "kind": "oracle",
+                             "sample": f"all {cfg.M} tokens x {cfg.K} features, {ncols} of {cfg.N} output channels "
+                                       "per step"},
+            "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="native", choices=("native", "reference"))
+    ap.add_argument("--workload", default="llm_mlp_up")
+    ap.add_argument("--out-dtype", default="bf16", choices=("bf16", "f32"))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="timed region only (no side measurements, no CPU baseline): for profiler captures")
+    args = ap.parse_args()
+    cfg = workloads()[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2510_26771_b200 import binding as st
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    st.lib()  # fails loudly if the CUDA library is missing
+    warmup = max(args.warmup, 3)
+    steps = max(args.steps, 1)
+    peaks = measured_peaks()
+
+    # ---- inputs: generated on the host, resident in HBM before the timed region ----
+    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi)
+    B, L, K, N, M = cfg.B, cfg.L, cfg.K, cfg.N, cfg.M
+    x_t = torch.bfloat16 if cfg.dtype == gen.BF16 else torch.float32
+    y_t = torch.bfloat16 if args.out_dtype == "bf16" else torch.float32
+    X_host = torch.from_numpy(gen.make_activation(cfg)).to(x_t).pin_memory()
+    W_dev = torch.from_numpy(gen.make_weight(cfg)).cuda().to(x_t)
+    bias = torch.from_numpy(gen.make_bias(cfg)).cuda()
+    wq, w_scale = st.stamp_quantize_weights(c, W_dev)       # offline: weights are static
+    w8 = st.stamp_prepare_weights(c, wq)
+    del W_dev
+    x_bytes = X_host.numel() * X_host.element_size()
+    y_bytes = M * N * (2 if y_t == torch.bfloat16 else 4)
+    # rotate over enough distinct copies that consecutive steps never find their inputs in L2
+    n_x = max(2, -(-2 * L2_BYTES // x_bytes))
+    n_w = max(2, -(-2 * L2_BYTES // w8.numel()))
+    Xs = [X_host.cuda() for _ in range(n_x)]
+    Ws = [w8.clone() for _ in range(n_w)]
+    Y = torch.empty((B, L, N), dtype=y_t, device="cuda")
+    ws = st.alloc_workspace(c, B, L, K, N)
+
+    def step(i):
+        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], st.W_INT8, w_scale, bias, ws, out=Y)
+
+    for i in range(warmup):
+        step(i)
+    launches_per_step = st.stamp_last_launch_count()
+    torch.cuda.synchronize()
+    if st.stamp_last_device_status() != 0:
+        raise RuntimeError("device status word raised during warm-up")
+
+    # ---- timed region: exactly `steps` steps, CUDA events, GEMM bracketed by its own events ----
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    n_ev = min(steps, 200)
+    g0 = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev)]
+    g1 = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev)]
+    for e in g0 + g1:
+        e.record()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0.record()
+    for i in range(steps):
+        if i < n_ev:
+            st.stamp_profile_gemm_events(g0[i], g1[i])
+        elif i == n_ev:
+            st.stamp_profile_gemm_events(None, None)
+        step(i)
+    ev1.record()
+    st.stamp_profile_gemm_events(None, None)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / steps
+    gemm_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(g0, g1))
+    status = st.stamp_last_device_status()
+
+    # keep the GPU under the same load a little longer if the timed region was too short to sample clocks
+    clocks = None
+    if sampler is not None:
+        t_end = time.time() + (0.0 if args.quick else max(0.0, 1.0 - total_ms / 1e3))
+        i = 0
+        while time.time() < t_end:
+            step(i)
+            i += 1
+            if i % 64 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+
+    ops = 2.0 * M * N * K
+    value = world * ops / (ms_per_step * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    if args.quick:
+        gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
+        print(json.dumps({"metric": "stamp_linear_tops", "value": value, "unit": "TOPS", "n_gpus": world,
+                          "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "quick": True,
+                          "config": {"workload": cfg.name}, "extra": {"gemm_ms": gemm_ms, "gemm_tops": gemm_tops},
+                          "gpu_launches": launches_per_step * steps, "clocks": clocks}), flush=True)
+        return
+
+    # ---- the bandwidth-bound passes, timed alone (L2 defeated by the same rotation) ----
+    def time_loop(fn, iters):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(iters):
+            fn(i)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters
+
+    iters = max(10, min(steps, 200))
+    nh = st.n_hi_rows(c, B, L)
+    quant_bytes = x_bytes + nh * K + (M - nh) * K // 2 + 4 * M
+    q_ms = time_loop(lambda i: st.stamp_quantize(c, Xs[i % n_x], ws), iters)
+    n_yt = max(2, -(-2 * L2_BYTES // (M * N * 4)))
+    Yts = [torch.randn((B, L, N), device="cuda") for _ in range(n_yt)]
+    inv_bytes = M * N * 4 + y_bytes
+    i_ms = time_loop(lambda i: st.stamp_inverse(c, Yts[i % n_yt], bias, ws, out=Y), iters)
+    del Yts
+
+    # ---- int8 GEMM throughput of the vendor library on this machine, for context ----
+    int_mm_tops = None
+    try:
+        a = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda")
+        b = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda").t()
+        mm_ms = time_loop(lambda i: torch._int_mm(a, b), 20)
+        int_mm_tops = 2.0 * 8192 ** 3 / (mm_ms * 1e-3) / 1e12
+        del a, b
+    except Exception:
+        pass
+
+    # ---- end to end: host buffers, copies inside the timed region, through the C ABI ----
+    ws_h = torch.empty(st.stamp_workspace_bytes_host(c, B, L, K, N, st._dtype_code(X_host), 1 if y_t == torch.bfloat16 else 0),
+                       dtype=torch.uint8, device="cuda")
+    Y_host = torch.empty((B, L, N), dtype=y_t).pin_memory()
+    e2e_steps = max(5, min(steps, 100))
+
+    def e2e_step(i):
+        st.stamp_linear_fused_host(c, X_host, Ws[i % n_w], st.W_INT8, w_scale, bias, Y_host, ws_h)
+    e2e_ms = time_loop(e2e_step, e2e_steps)
+    e2e = {"value": ops / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": x_bytes,
+           "d2h_bytes_per_step": y_bytes, "ms_per_step": e2e_ms}
+
+    i8_peak = peaks["bf16_sustained"] * NOMINAL_I8_OVER_BF16
+    gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "k_gemm_i8", "achieved": gemm_tops, "peak": i8_peak, "unit": "TFLOP/s",
+                "frac": gemm_tops / i8_peak, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                "note": f"int8 ops; peak = {peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s x 2 "
+                        "(nominal int8:bf16 ratio); kernel timed inside the long step loop"}
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu_baseline, _ = cpu_oracle_sample(cfg)
+
+    line = {
+        "metric": "stamp_linear_tops", "value": value, "unit": "TOPS", "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": B, "L": L, "K": K, "N": N, "transform": int(cfg.transform),
+                   "block": cfg.block, "levels": cfg.levels, "k_hi": cfg.k_hi, "x_dtype": str(x_t).split(".")[-1],
+                   "y_dtype": str(y_t).split(".")[-1], "weights": "int4 codes, one per int8, prepared offline",
+                   "l2": f"inputs rotate over {n_x} activation and {n_w} weight copies (> 2x L2)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * steps, "roofline": roofline,
+        "cpu_baseline": cpu_baseline,
+        "extra": {"gemm_ms": gemm_ms, "gemm_tops": gemm_tops, "frac_of_nominal_4500": gemm_tops / 4500.0,
+                  "layer_frac_of_i8_peak": value / world / i8_peak,
+                  "quant_ms": q_ms, "quant_gbs": quant_bytes / (q_ms * 1e-3) / 1e9,
+                  "quant_frac_hbm": quant_bytes / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                  "inverse_ms": i_ms, "inverse_gbs": inv_bytes / (i_ms * 1e-3) / 1e9,
+                  "inverse_frac_hbm": inv_bytes / (i_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                  "torch_int_mm_8192_tops": int_mm_tops, "launches_per_step": launches_per_step,
+                  "device_status": status, "peaks": peaks},
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

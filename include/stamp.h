@@ -144,6 +144,19 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
                        const float* w_scale, const float* bias, int B, int L, int K, int N, void* Y,
                        int y_dtype, void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * The same call for callers whose activation and output live in HOST memory (ideally pinned):
+ * copies X host->device, runs the layer, copies Y device->host, all enqueued on `stream`.  The
+ * weight operand, scales and bias are device pointers as above.  `ws` must hold at least
+ * stamp_workspace_bytes_host() bytes (the device workspace plus staging for X and Y).
+ * No counterpart in the paper: a convenience for end-to-end measurement and host-side callers.
+ */
+int stamp_workspace_bytes_host(const stamp_config* cfg, int B, int L, int K, int N, int x_dtype, int y_dtype,
+                               size_t* out_bytes);
+int stamp_linear_fused_host(const stamp_config* cfg, const void* X_host, int x_dtype, const void* w, int w_format,
+                            const float* w_scale, const float* bias, int B, int L, int K, int N, void* Y_host,
+                            int y_dtype, void* ws, size_t ws_bytes, void* stream);
+
 /* ---- parity / debug exports: the intermediate stages, judged separately against the oracle ---- */
 
 /* T = L X in fp32, logical token order.  T [B, L, K] float out. */
@@ -163,6 +176,11 @@ int stamp_debug_gemm_i32(const stamp_config* cfg, const void* q_hi, const void* 
  * *status is STAMP_OK or STAMP_ERR_TIMEOUT (a bounded wait inside a kernel expired; outputs of
  * the calls since the last read are then invalid). */
 int stamp_last_device_status(void* stream, int* status);
+
+/* Measurement hook: while both events are non-NULL, every tensor-core GEMM launched by the
+ * calling thread is bracketed by cudaEventRecord(start) / cudaEventRecord(stop) on its stream
+ * (each launch re-records the pair).  Pass NULLs to switch it off.  Events are cudaEvent_t. */
+int stamp_profile_gemm_events(void* start_event, void* stop_event);
 
 /* How many kernels of this library the calling thread's last API call launched. */
 int stamp_last_launch_count(void);

@@ -20,7 +20,8 @@ W_PACKED4, W_INT8 = 0, 1
 
 EXPORTS = (
     "stamp_workspace_bytes", "stamp_quantize_weights", "stamp_prepare_weights", "stamp_quantize",
-    "stamp_linear", "stamp_inverse", "stamp_linear_fused", "stamp_debug_transform",
+    "stamp_linear", "stamp_inverse", "stamp_linear_fused", "stamp_workspace_bytes_host",
+    "stamp_linear_fused_host", "stamp_profile_gemm_events", "stamp_debug_transform",
     "stamp_debug_unpack_codes", "stamp_debug_gemm_i32", "stamp_last_device_status",
     "stamp_last_launch_count", "stamp_status_string",
 )
@@ -166,6 +167,36 @@ def stamp_linear_fused(cfg: StampConfig, X: torch.Tensor, w: torch.Tensor, w_for
                                     _ptr(w_scale), _ptr(bias), B, L, K, N, _ptr(Y), _dtype_code(Y), wp, wb,
                                     _stream()), "stamp_linear_fused")
     return Y
+
+
+def stamp_workspace_bytes_host(cfg: StampConfig, B: int, L: int, K: int, N: int, x_dtype: int, y_dtype: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().stamp_workspace_bytes_host(ctypes.byref(cfg), B, L, K, N, x_dtype, y_dtype, ctypes.byref(out)),
+           "stamp_workspace_bytes_host")
+    return int(out.value)
+
+
+def stamp_linear_fused_host(cfg: StampConfig, X_host: torch.Tensor, w: torch.Tensor, w_format: int,
+                            w_scale: torch.Tensor, bias: Optional[torch.Tensor], Y_host: torch.Tensor,
+                            ws: torch.Tensor) -> torch.Tensor:
+    """X_host / Y_host are CPU tensors (pinned for asynchronous copies); everything else is on the device."""
+    B, L, K = X_host.shape
+    N = w.shape[0]
+    if X_host.is_cuda or Y_host.is_cuda or not X_host.is_contiguous() or not Y_host.is_contiguous():
+        raise ValueError("expected contiguous host tensors")
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_linear_fused_host(ctypes.byref(cfg), ctypes.c_void_p(X_host.data_ptr()), _dtype_code(X_host),
+                                         _ptr(w), int(w_format), _ptr(w_scale), _ptr(bias), B, L, K, N,
+                                         ctypes.c_void_p(Y_host.data_ptr()), _dtype_code(Y_host), wp, wb, _stream()),
+           "stamp_linear_fused_host")
+    return Y_host
+
+
+def stamp_profile_gemm_events(start: Optional["torch.cuda.Event"], stop: Optional["torch.cuda.Event"]) -> None:
+    """Bracket every GEMM launch of this thread with the two (already created) CUDA events."""
+    s = ctypes.c_void_p(start.cuda_event) if start is not None else None
+    e = ctypes.c_void_p(stop.cuda_event) if stop is not None else None
+    _check(lib().stamp_profile_gemm_events(s, e), "stamp_profile_gemm_events")
 
 
 def stamp_debug_transform(cfg: StampConfig, X: torch.Tensor, ws: torch.Tensor) -> torch.Tensor:

@@ -14,6 +14,7 @@
 namespace stamp {
 
 static thread_local int t_launches = 0;
+static thread_local cudaEvent_t t_gemm_ev_start = nullptr, t_gemm_ev_stop = nullptr;
 
 #define STAMP_CHECK_LAUNCH()                                   \
   do {                                                         \
@@ -184,7 +185,10 @@ static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const Gem
   const int tok_tiles = (gp.m_tok + BN - 1) / BN;
   const int tiles = ch_tiles * tok_tiles;
   const int grid = tiles < sm_count() ? tiles : sm_count();
+  const bool timed = t_gemm_ev_start && t_gemm_ev_stop;
+  if (timed) cudaEventRecord(t_gemm_ev_start, st);
   kern<<<grid, GEMM_THREADS, SM::DYN_BYTES, st>>>(tw, tx, gp);
+  if (timed) cudaEventRecord(t_gemm_ev_stop, st);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
 }
@@ -470,6 +474,42 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, st);
 }
 
+static size_t dtype_size(int d) { return d == STAMP_BF16 ? 2 : 4; }
+
+int stamp_workspace_bytes_host(const stamp_config* cfg, int B, int L, int K, int N, int x_dtype, int y_dtype,
+                               size_t* out_bytes) {
+  if (!out_bytes || !dtype_ok(x_dtype) || !dtype_ok(y_dtype)) return STAMP_ERR_INVALID_ARG;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, N, true, &pb);
+  if (rc) return rc;
+  *out_bytes = layout(pb).total + align256((size_t)pb.M * K * dtype_size(x_dtype)) +
+               align256((size_t)pb.M * N * dtype_size(y_dtype));
+  return STAMP_OK;
+}
+
+int stamp_linear_fused_host(const stamp_config* cfg, const void* X_host, int x_dtype, const void* w, int w_format,
+                            const float* w_scale, const float* bias, int B, int L, int K, int N, void* Y_host,
+                            int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+  size_t need = 0;
+  int rc = stamp_workspace_bytes_host(cfg, B, L, K, N, x_dtype, y_dtype, &need);
+  if (rc) return rc;
+  if (!X_host || !Y_host) return STAMP_ERR_INVALID_ARG;
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < need) return STAMP_ERR_WORKSPACE;
+  Problem pb;
+  resolve(cfg, B, L, K, N, true, &pb);
+  const size_t dev_ws = layout(pb).total;
+  const size_t xb = (size_t)pb.M * K * dtype_size(x_dtype), yb = (size_t)pb.M * N * dtype_size(y_dtype);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  void* Xd = base + dev_ws;
+  void* Yd = base + dev_ws + align256(xb);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(Xd, X_host, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return STAMP_ERR_CUDA;
+  rc = stamp_linear_fused(cfg, Xd, x_dtype, w, w_format, w_scale, bias, B, L, K, N, Yd, y_dtype, ws, dev_ws, stream);
+  if (rc) return rc;
+  if (cudaMemcpyAsync(Y_host, Yd, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return STAMP_ERR_CUDA;
+  return STAMP_OK;
+}
+
 int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, float* T, void* ws,
                           size_t ws_bytes, void* stream) {
   t_launches = 0;
@@ -524,6 +564,13 @@ int stamp_last_device_status(void* stream, int* status) {
     if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return STAMP_ERR_CUDA;
   }
   *status = v;
+  return STAMP_OK;
+}
+
+int stamp_profile_gemm_events(void* start_event, void* stop_event) {
+  if ((start_event == nullptr) != (stop_event == nullptr)) return STAMP_ERR_INVALID_ARG;
+  t_gemm_ev_start = static_cast<cudaEvent_t>(start_event);
+  t_gemm_ev_stop = static_cast<cudaEvent_t>(stop_event);
   return STAMP_OK;
 }
 
