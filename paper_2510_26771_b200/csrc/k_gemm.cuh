@@ -50,7 +50,8 @@ struct GemmSmem {
   static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
   // full[STAGES], empty[STAGES], tfull[2], tempty[2], then tmem base + abort word
   static constexpr int NUM_BARS = 2 * STAGES + 4;
-  static constexpr int TOTAL = BAR_OFFSET + NUM_BARS * 8 + 16;
+  static constexpr int SX_OFFSET = BAR_OFFSET + NUM_BARS * 8 + 16;  // token scales of the tile being drained
+  static constexpr int TOTAL = SX_OFFSET + 2 * BN * 4;   // one buffer per accumulator
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for 1024-byte alignment of the ring
 };
 
@@ -78,6 +79,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
   uint64_t* tempty = tfull + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile uint32_t* abort_word = tmem_slot + 1;
+  float* sx_stage = reinterpret_cast<float*>(smem + SM::SX_OFFSET);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -196,6 +198,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32 * (warp % 4) ...
     const int row = quarter * 32 + lane;
+    const int ep_tid = threadIdx.x - 64;  // 0..127
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
@@ -206,39 +209,58 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       const int ch = ch_t * GEMM_BM + row;
       const int tok0 = tok_t * BN;
       const bool ch_ok = ch < p.n_out;
+      const bool full_tile = (tok0 + BN <= p.m_tok);
+      float* sxs = sx_stage + a * BN;
       float sw = 0.f;
-      if (EPI == EPI_DEQUANT_F32 && ch_ok) sw = __ldg(p.w_scale + ch);
+      float my_sx[BN / 128];
+      if (EPI == EPI_DEQUANT_F32) {
+        if (ch_ok) sw = __ldg(p.w_scale + ch);
+        // fetch this tile's token scales while the accumulator is still being filled
+#pragma unroll
+        for (int i = 0; i < BN / 128; ++i) {
+          const int tok = tok0 + i * 128 + ep_tid;
+          my_sx[i] = (tok < p.m_tok) ? __ldg(p.x_scale + tok) : 0.f;
+        }
+      }
       // the TMEM loads below are warp-collective: the whole warp continues or the whole warp stops
       if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&tfull[a], acc_phase, abort_word, GEMM_WAIT_LIMIT))) {
         ok = false;
         break;
       }
       ptx::tc_fence_after();
+      if (EPI == EPI_DEQUANT_F32) {
+        // every epilogue thread has finished the previous tile that used accumulator `a` (all 128
+        // arrived on tempty[a] before tfull[a] could complete again), so its staging buffer is free
+#pragma unroll
+        for (int i = 0; i < BN / 128; ++i) sxs[i * 128 + ep_tid] = my_sx[i];
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(a * BN);
-#pragma unroll 1
+      uint32_t r[2][32];
+      ptx::tmem_ld_32x32b_x32(taddr, r[0]);
+#pragma unroll
       for (int chunk = 0; chunk < BN / 32; ++chunk) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32b_x32(taddr + chunk * 32, r);
         ptx::tmem_ld_wait();
+        if (chunk + 1 < BN / 32) ptx::tmem_ld_32x32b_x32(taddr + (chunk + 1) * 32, r[(chunk + 1) & 1]);
+        const uint32_t(&rc)[32] = r[chunk & 1];
         const int tbase = tok0 + chunk * 32;
         if (EPI == EPI_DEQUANT_F32) {
-          float* out = static_cast<float*>(p.out);
+          float* out = static_cast<float*>(p.out) + (long)tbase * p.n_out + ch;
+          if (full_tile && ch_ok) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int tok = tbase + j;
-            if (tok < p.m_tok) {
-              const float sx = __ldg(p.x_scale + tok);
-              const float v = static_cast<float>(static_cast<int>(r[j])) * sx * sw;
-              if (ch_ok) out[(long)tok * p.n_out + ch] = v;
-            }
+            for (int j = 0; j < 32; ++j)
+              out[(long)j * p.n_out] = static_cast<float>(static_cast<int>(rc[j])) * sxs[chunk * 32 + j] * sw;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (tbase + j < p.m_tok && ch_ok)
+                out[(long)j * p.n_out] = static_cast<float>(static_cast<int>(rc[j])) * sxs[chunk * 32 + j] * sw;
           }
         } else {
-          int* out = static_cast<int*>(p.out);
+          int* out = static_cast<int*>(p.out) + (long)tbase * p.n_out + ch;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int tok = tbase + j;
-            if (tok < p.m_tok && ch_ok) out[(long)tok * p.n_out + ch] = static_cast<int>(r[j]);
-          }
+          for (int j = 0; j < 32; ++j)
+            if (tbase + j < p.m_tok && ch_ok) out[(long)j * p.n_out] = static_cast<int>(rc[j]);
         }
       }
       ptx::tc_fence_before();

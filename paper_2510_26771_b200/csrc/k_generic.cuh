@@ -13,7 +13,9 @@ namespace stamp {
 //
 // One thread owns two adjacent channels of one group of G = 2^P consecutive input tokens and
 // runs the butterflies in registers on UNNORMALISED sums; a coefficient of global level j is
-// multiplied once by 2^(-j/2) when it is written.  Detail rows go to their logical row of T,
+// multiplied once by 2^(-(j + norm_off)/2) when it is written (norm_off > 0 when the input rows are
+// themselves sums over 2^norm_off tokens produced by another kernel and T is the compact table of
+// the remaining coarse rows).  Detail rows go to their logical row of T,
 // [a | d_levels | ... | d_1]; the group's running sum goes to `aout` for the next pass, or, in
 // the last pass, to the approximation rows of T.
 //   in      [nseq, Lin, K]      TIn (first pass: X; later passes: unnormalised sums, float)
@@ -23,7 +25,7 @@ namespace stamp {
 // ------------------------------------------------------------------------------------------
 template <int P, typename TIn>
 __global__ void __launch_bounds__(128) k_haar_fwd_pass(const TIn* __restrict__ in, int Lin, long ngroups, int K,
-                                                       float* __restrict__ T, int n, int lvl0,
+                                                       float* __restrict__ T, int n, int lvl0, int norm_off,
                                                        float* __restrict__ aout, unsigned* __restrict__ rowmax) {
   constexpr int G = 1 << P;
   const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
@@ -46,7 +48,7 @@ __global__ void __launch_bounds__(128) k_haar_fwd_pass(const TIn* __restrict__ i
     for (int l = 1; l <= P; ++l) {
       const int half = G >> l;
       const int j = lvl0 + l;
-      const HaarNorm nrm = haar_norm(j);
+      const HaarNorm nrm = haar_norm(j + norm_off);
       const int row0 = (n >> j) + g * half;
 #pragma unroll
       for (int i = 0; i < half; ++i) {
@@ -66,7 +68,7 @@ __global__ void __launch_bounds__(128) k_haar_fwd_pass(const TIn* __restrict__ i
     if (aout) {
       store2(aout + ((s * gps + g) * (long)K + c), a0[0], a1[0]);
     } else {
-      const HaarNorm nrm = haar_norm(lvl0 + P);
+      const HaarNorm nrm = haar_norm(lvl0 + P + norm_off);
       const float v0 = mul_norm(a0[0], nrm), v1 = mul_norm(a1[0], nrm);
       store2(Tseq + (long)g * K, v0, v1);
       if (rm) {
@@ -156,24 +158,26 @@ __device__ __forceinline__ float div_by_scale(float t, float scale, float inv) {
 
 // ------------------------------------------------------------------------------------------
 // Row quantizer (Sec. 2.1, first equation, symmetric form) reading materialised T.
-// One CTA per transformed token: scale = absmax / qmax (IEEE fp32 division), codes =
-// clamp(rne(t * (1 / scale))).  Writes any of: the int8 operand row for the GEMM (a8), the
+// One CTA per materialised row: scale = absmax / qmax (IEEE fp32 division), codes =
+// clamp(rne(t / scale)).  Writes any of: the int8 operand row for the GEMM (a8), the
 // public packed outputs (q_hi rows as int8, q_lo rows as nibble pairs), the scale.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_quant_rows(const float* __restrict__ T, const unsigned* __restrict__ rowmax,
-                                                    int K, int n, int k_hi, int qmax_hi, int qmax_lo,
+                                                    int K, int n_src, int n, int k_hi, int qmax_hi, int qmax_lo,
                                                     int8_t* __restrict__ a8, int8_t* __restrict__ q_hi,
                                                     uint8_t* __restrict__ q_lo, float* __restrict__ x_scale) {
-  const long r = blockIdx.x;
-  const long s = r / n;
-  const int i = static_cast<int>(r - s * n);
+  // T / rowmax hold the first n_src rows of every block of n logical rows
+  const long rs = blockIdx.x;
+  const long s = rs / n_src;
+  const int i = static_cast<int>(rs - s * n_src);
+  const long r = s * n + i;
   const bool hi = i < k_hi;
   const float qmax = static_cast<float>(hi ? qmax_hi : qmax_lo);
-  const float amax = __uint_as_float(rowmax[r]);
+  const float amax = __uint_as_float(rowmax[rs]);
   const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
   const float inv = __fdiv_rn(1.0f, scale);
   if (threadIdx.x == 0) x_scale[r] = scale;
-  const float4* src = reinterpret_cast<const float4*>(T + r * (long)K);
+  const float4* src = reinterpret_cast<const float4*>(T + rs * (long)K);
   char4* dst8 = a8 ? reinterpret_cast<char4*>(a8 + r * (long)K) : nullptr;
   char4* dsth = (q_hi && hi) ? reinterpret_cast<char4*>(q_hi + (s * k_hi + i) * (long)K) : nullptr;
   uint16_t* dstl =

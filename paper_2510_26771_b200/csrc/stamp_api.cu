@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "k_gemm.cuh"
 #include "k_generic.cuh"
+#include "k_haar_tq.cuh"
 #include "stamp.h"
 
 namespace stamp {
@@ -97,7 +98,7 @@ static PassPlan make_plan(int levels) {
 // Workspace layout (one layout for all calls of a problem size).
 // ------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t rowmax, xscale, T, ping, pong, a8, w8, yt, total;
+  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, a8, w8, yt, total;
 };
 static Workspace layout(const Problem& pb) {
   Workspace w{};
@@ -112,6 +113,10 @@ static Workspace layout(const Problem& pb) {
   w.T = off;      off += align256(M * (size_t)pb.K * 4);
   w.ping = off;   off += align256(ping_rows * KN * 4);
   w.pong = off;   off += align256(pong_rows * KN * 4);
+  // level-5-or-coarser sums leaving the fused transform+quantize kernel, and its top passes
+  w.atop = off;     off += align256((M >> 5) * (size_t)pb.K * 4);
+  w.top_ping = off; off += align256((M >> 10) * (size_t)pb.K * 4);
+  w.top_pong = off; off += align256((M >> 15) * (size_t)pb.K * 4);
   w.a8 = off;     off += align256(M * (size_t)pb.K);
   w.w8 = off;     off += align256((size_t)pb.N * pb.K);
   w.yt = off;     off += align256(M * (size_t)pb.N * 4);
@@ -219,18 +224,49 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
 }
 
 template <typename TIn>
-static int launch_fwd_pass(int P, const TIn* in, int Lin, long ngroups, int K, float* T, int n, int lvl0, float* aout,
-                           unsigned* rowmax, cudaStream_t st) {
+static int launch_fwd_pass(int P, const TIn* in, int Lin, long ngroups, int K, float* T, int n, int lvl0, int norm_off,
+                           float* aout, unsigned* rowmax, cudaStream_t st) {
   dim3 grid((K / 2 + 127) / 128, (unsigned)(ngroups < 32768 ? ngroups : 32768));
   switch (P) {
-    case 0: k_haar_fwd_pass<0, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
-    case 1: k_haar_fwd_pass<1, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
-    case 2: k_haar_fwd_pass<2, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
-    case 3: k_haar_fwd_pass<3, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
-    case 4: k_haar_fwd_pass<4, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
-    default: k_haar_fwd_pass<5, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, aout, rowmax); break;
+    case 0: k_haar_fwd_pass<0, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, norm_off, aout, rowmax); break;
+    case 1: k_haar_fwd_pass<1, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, norm_off, aout, rowmax); break;
+    case 2: k_haar_fwd_pass<2, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, norm_off, aout, rowmax); break;
+    case 3: k_haar_fwd_pass<3, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, norm_off, aout, rowmax); break;
+    case 4: k_haar_fwd_pass<4, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, norm_off, aout, rowmax); break;
+    default: k_haar_fwd_pass<5, TIn><<<grid, 128, 0, st>>>(in, Lin, ngroups, K, T, n, lvl0, norm_off, aout, rowmax); break;
   }
   STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// Multi-pass Haar analysis of `levels` levels over nseq sequences of Lin input rows.  The input
+// rows are X itself (norm_off = 0) or un-normalised sums over 2^norm_off tokens.  Coefficients go
+// to T, laid out as blocks of n rows in [a | d_coarse .. d_fine] order where the first level of
+// this call has row-mapping level lvl0 + 1; optionally the per-row |T| maxima (pre-zeroed here).
+static int run_haar_passes(const void* in, bool in_bf16, int nseq, int Lin, int K, int levels, float* T, int n,
+                           int lvl0, int norm_off, unsigned* rowmax, size_t rowmax_rows, float* ping, float* pong,
+                           cudaStream_t st) {
+  if (rowmax && cudaMemsetAsync(rowmax, 0, rowmax_rows * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+  const PassPlan pl = make_plan(levels);
+  const float* cur = nullptr;
+  float* bufs[2] = {ping, pong};
+  for (int i = 0; i < pl.npass; ++i) {
+    const int P = pl.p[i];
+    const bool last = (i == pl.npass - 1);
+    float* aout = last ? nullptr : bufs[i & 1];
+    const long ngroups = (long)nseq * (Lin >> P);
+    int rc;
+    if (i == 0 && in_bf16)
+      rc = launch_fwd_pass<__nv_bfloat16>(P, static_cast<const __nv_bfloat16*>(in), Lin, ngroups, K, T, n, lvl0,
+                                          norm_off, aout, rowmax, st);
+    else
+      rc = launch_fwd_pass<float>(P, i == 0 ? static_cast<const float*>(in) : cur, Lin, ngroups, K, T, n, lvl0,
+                                  norm_off, aout, rowmax, st);
+    if (rc) return rc;
+    cur = aout;
+    lvl0 += P;
+    Lin >>= P;
+  }
   return STAMP_OK;
 }
 
@@ -238,33 +274,8 @@ static int launch_fwd_pass(int P, const TIn* in, int Lin, long ngroups, int K, f
 static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, float* T, unsigned* rowmax,
                                  float* ping, float* pong, cudaStream_t st) {
   if (pb.transform == STAMP_T_DCT2) return STAMP_ERR_UNSUPPORTED;
-  if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
-  const PassPlan pl = make_plan(pb.levels);
-  int lvl0 = 0;
-  int Lin = pb.n;
-  const float* cur = nullptr;
-  float* bufs[2] = {ping, pong};
-  for (int i = 0; i < pl.npass; ++i) {
-    const int P = pl.p[i];
-    const bool last = (i == pl.npass - 1);
-    float* aout = last ? nullptr : bufs[i & 1];
-    const long ngroups = (long)pb.nseq * (Lin >> P);
-    int rc;
-    if (i == 0) {
-      rc = (x_dtype == STAMP_BF16)
-               ? launch_fwd_pass<__nv_bfloat16>(P, static_cast<const __nv_bfloat16*>(X), Lin, ngroups, pb.K, T, pb.n,
-                                                lvl0, aout, rowmax, st)
-               : launch_fwd_pass<float>(P, static_cast<const float*>(X), Lin, ngroups, pb.K, T, pb.n, lvl0, aout,
-                                        rowmax, st);
-    } else {
-      rc = launch_fwd_pass<float>(P, cur, Lin, ngroups, pb.K, T, pb.n, lvl0, aout, rowmax, st);
-    }
-    if (rc) return rc;
-    cur = aout;
-    lvl0 += P;
-    Lin >>= P;
-  }
-  return STAMP_OK;
+  return run_haar_passes(X, x_dtype == STAMP_BF16, pb.nseq, pb.n, pb.K, pb.levels, T, pb.n, 0, 0, rowmax,
+                         (size_t)pb.M, ping, pong, st);
 }
 
 template <typename TOut>
@@ -319,12 +330,112 @@ static int run_inverse_generic(const Problem& pb, const float* Yt, const float* 
   return STAMP_OK;
 }
 
-static int run_quant_rows(const Problem& pb, const float* T, const unsigned* rowmax, int8_t* a8, void* q_hi,
-                          void* q_lo, float* x_scale, cudaStream_t st) {
-  k_quant_rows<<<(unsigned)pb.M, 256, 0, st>>>(T, rowmax, pb.K, pb.n, pb.k_hi, pb.qmax_hi, pb.qmax_lo, a8,
-                                                static_cast<int8_t*>(q_hi), static_cast<uint8_t*>(q_lo), x_scale);
+// Quantize materialised rows: T / rowmax hold the first n_src rows of every block of pb.n rows.
+static int run_quant_rows(const Problem& pb, const float* T, const unsigned* rowmax, int n_src, int8_t* a8,
+                          void* q_hi, void* q_lo, float* x_scale, cudaStream_t st) {
+  const long rows = (long)pb.nseq * n_src;
+  k_quant_rows<<<(unsigned)rows, 256, 0, st>>>(T, rowmax, pb.K, n_src, pb.n, pb.k_hi, pb.qmax_hi, pb.qmax_lo, a8,
+                                               static_cast<int8_t*>(q_hi), static_cast<uint8_t*>(q_lo), x_scale);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Fused Haar transform + quantizer (bf16 input): one cluster kernel for the first D levels, the
+// general passes for the few coarse rows above.
+// ------------------------------------------------------------------------------------------
+struct TqChoice {
+  int G, m, tree, D;
+  size_t smem;
+};
+static bool choose_tq(const Problem& pb, int x_dtype, TqChoice* c) {
+  if (pb.transform != STAMP_T_HAAR || x_dtype != STAMP_BF16 || pb.levels < 2) return false;
+  const int cand[3] = {16, 8, 4};
+  int G = 0;
+  for (int i = 0; i < 3; ++i) {
+    const int g = cand[i], m = ilog2(g);
+    if (m > pb.levels) continue;
+    const size_t slab = (size_t)g * pb.K * 2;
+    if (slab <= 65536 || (g == 4 && slab + (size_t)pb.K * 4 <= 200 * 1024)) {
+      G = g;
+      break;
+    }
+  }
+  if (!G) return false;
+  c->G = G;
+  c->m = ilog2(G);
+  c->tree = pb.levels - c->m < 3 ? pb.levels - c->m : 3;
+  c->D = c->m + c->tree;
+  c->smem = G == 16 ? tq_smem_bytes<16>(pb.K) : G == 8 ? tq_smem_bytes<8>(pb.K) : tq_smem_bytes<4>(pb.K);
+  return true;
+}
+
+template <int G>
+static int launch_tq(const TqParams& tp, const TqChoice& c, long M, cudaStream_t st) {
+  auto kern = k_haar_tq<G>;
+  static size_t attr_smem = 0;
+  if (c.smem > attr_smem) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem) != cudaSuccess)
+      return STAMP_ERR_CUDA;
+    attr_smem = c.smem;
+  }
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3((unsigned)(M / G));
+  lc.blockDim = dim3(TQ_THREADS);
+  lc.dynamicSmemBytes = c.smem;
+  lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 1u << c.tree;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  if (cudaLaunchKernelEx(&lc, kern, tp) != cudaSuccess) {
+    cudaGetLastError();
+    return STAMP_ERR_CUDA;
+  }
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// Transform + quantize through the fused kernel.  Any of a8 / (q_hi, q_lo) / T_out may be null.
+static int run_quantize_fast(const Problem& pb, const TqChoice& c, const void* X, int8_t* a8, void* q_hi, void* q_lo,
+                             float* x_scale, float* T_out, uint8_t* base, const Workspace& wl, cudaStream_t st) {
+  TqParams tp{};
+  tp.X = static_cast<const __nv_bfloat16*>(X);
+  tp.K = pb.K;
+  tp.n = pb.n;
+  tp.levels = pb.levels;
+  tp.k_hi = pb.k_hi;
+  tp.qmax_hi = pb.qmax_hi;
+  tp.qmax_lo = pb.qmax_lo;
+  tp.tree_steps = c.tree;
+  tp.a8 = a8;
+  tp.q_hi = static_cast<int8_t*>(q_hi);
+  tp.q_lo = static_cast<uint8_t*>(q_lo);
+  tp.x_scale = x_scale;
+  tp.T_out = T_out;
+  const bool has_top = pb.levels > c.D;
+  float* atop = reinterpret_cast<float*>(base + wl.atop);
+  tp.atop = has_top ? atop : nullptr;
+  int rc = c.G == 16 ? launch_tq<16>(tp, c, pb.M, st) : c.G == 8 ? launch_tq<8>(tp, c, pb.M, st)
+                                                                 : launch_tq<4>(tp, c, pb.M, st);
+  if (rc || !has_top) return rc;
+  // the remaining levels act on the level-D sums: a short sequence of n >> D rows per block
+  const int n_top = pb.n >> c.D;
+  float* T_top = reinterpret_cast<float*>(base + wl.T);
+  unsigned* rowmax_top = reinterpret_cast<unsigned*>(base + wl.rowmax);
+  float* tping = reinterpret_cast<float*>(base + wl.top_ping);
+  float* tpong = reinterpret_cast<float*>(base + wl.top_pong);
+  rc = run_haar_passes(atop, false, pb.nseq, n_top, pb.K, pb.levels - c.D, T_top, n_top, 0, c.D, rowmax_top,
+                       (size_t)pb.nseq * n_top, tping, tpong, st);
+  if (rc) return rc;
+  if ((rc = run_quant_rows(pb, T_top, rowmax_top, n_top, a8, q_hi, q_lo, x_scale, st))) return rc;
+  if (T_out)  // debug export: the same coarse rows once more, written at their logical place
+    rc = run_haar_passes(atop, false, pb.nseq, n_top, pb.K, pb.levels - c.D, T_out, pb.n, c.D, 0, nullptr, 0, tping,
+                         tpong, st);
+  return rc;
 }
 
 static int run_unpack_codes(const Problem& pb, const void* q_hi, const void* q_lo, int8_t* out, cudaStream_t st) {
@@ -406,10 +517,12 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   uint8_t* base = static_cast<uint8_t*>(ws);
   float* T = reinterpret_cast<float*>(base + w.T);
   unsigned* rowmax = reinterpret_cast<unsigned*>(base + w.rowmax);
+  TqChoice tc;
+  if (choose_tq(pb, x_dtype, &tc)) return run_quantize_fast(pb, tc, X, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
   rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
                              reinterpret_cast<float*>(base + w.pong), st);
   if (rc) return rc;
-  return run_quant_rows(pb, T, rowmax, nullptr, q_hi, q_lo, x_scale, st);
+  return run_quant_rows(pb, T, rowmax, pb.n, nullptr, q_hi, q_lo, x_scale, st);
 }
 
 int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, const float* x_scale, const void* w,
@@ -466,8 +579,13 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
   float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
   float* yt = reinterpret_cast<float*>(base + wl.yt);
-  if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, st))) return rc;
-  if ((rc = run_quant_rows(pb, T, rowmax, a8, nullptr, nullptr, x_scale, st))) return rc;
+  TqChoice tc;
+  if (choose_tq(pb, x_dtype, &tc)) {
+    if ((rc = run_quantize_fast(pb, tc, X, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
+  } else {
+    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, st))) return rc;
+    if ((rc = run_quant_rows(pb, T, rowmax, pb.n, a8, nullptr, nullptr, x_scale, st))) return rc;
+  }
   const int8_t* w8 = nullptr;
   if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
   if ((rc = launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_F32, st))) return rc;
@@ -520,6 +638,10 @@ int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, i
   const Workspace wl = layout(pb);
   if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
   uint8_t* base = static_cast<uint8_t*>(ws);
+  TqChoice tc;
+  if (choose_tq(pb, x_dtype, &tc))  // same kernels as the product path, with the fp32 export switched on
+    return run_quantize_fast(pb, tc, X, nullptr, nullptr, nullptr, reinterpret_cast<float*>(base + wl.xscale), T, base,
+                             wl, static_cast<cudaStream_t>(stream));
   return run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + wl.ping),
                                reinterpret_cast<float*>(base + wl.pong), static_cast<cudaStream_t>(stream));
 }

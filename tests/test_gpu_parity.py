@@ -49,6 +49,11 @@ CASES = {
     # one-level transform and the identity (pure mixed-precision quantization)
     "one_level": gen.scaled(gen.config_sweep(512, 2048), L=256, K=128, N=64, levels=1, k_hi=128),
     "identity": gen.scaled(gen.config_sweep(512, 2048), L=192 + 64, K=256, N=128, transform=gen.T_IDENTITY, k_hi=8),
+    # wide feature axes: 8 and 4 tokens per CTA in the fused transform+quantize kernel
+    "wide_k4096": gen.scaled(gen.config_llm_up(), L=256, K=4096, N=64, k_hi=8),
+    "wide_k8192": gen.scaled(gen.config_sweep(512, 8192), L=128, K=8192, N=64, levels=5, k_hi=4),
+    # two levels only: no cluster tree, approximation rows quantized by the same kernel
+    "two_levels": gen.scaled(gen.config_dit_proj(), B=2, L=256, K=1152, N=128, grid=16, levels=2, k_hi=64),
 }
 
 
