@@ -50,7 +50,8 @@ typedef enum {
   STAMP_ERR_UNSUPPORTED = 2, /* valid request outside the shape / transform rules above    */
   STAMP_ERR_WORKSPACE = 3,   /* ws is null, misaligned or smaller than required            */
   STAMP_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, tensor map)   */
-  STAMP_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (device status only)    */
+  STAMP_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (device status only)    */
+  STAMP_ERR_TOO_LARGE = 6    /* stamp_inverse_noalloc: scratch need exceeds the built-in array */
 } stamp_status;
 
 typedef enum { STAMP_F32 = 0, STAMP_BF16 = 1 } stamp_dtype;
@@ -135,6 +136,34 @@ int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, co
  */
 int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
                   int y_dtype, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * stamp_inverse() for callers that cannot hand over a workspace and must not allocate one.
+ * (No counterpart in the paper: this is a packaging variant of the inverse-transform call.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- an operator plug-in
+ * called from a serving loop whose host framework owns every byte of device memory, a callback
+ * on a latency-critical path where cudaMalloc would stall the whole device, or a thin language
+ * binding that has no allocator to ask.  Such a caller still owns Yt, bias and Y; what it lacks
+ * is the few MB of scratch the multi-pass inverse keeps between its passes.
+ *
+ * Here that scratch is an array compiled into the library, STAMP_NOALLOC_SCRATCH_BYTES per GPU
+ * that loads the library, resident until the process exits.  The call performs no cudaMalloc,
+ * cudaFree or any other allocating routine.
+ *   - Limit: the partial sums of the inverse -- about (B*L/32 + B*L/1024) * N * 4 bytes for a
+ *     Haar transform deeper than 5 levels, nothing for 5 levels or fewer -- must fit the array;
+ *     otherwise STAMP_ERR_TOO_LARGE is returned before anything is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to be cleared between
+ *     calls: each call writes every element before reading it, so leftovers of the previous
+ *     call are never seen.  Two calls that overlap on the GPU (different streams, no ordering
+ *     between them) would overwrite each other's partial sums: order them.
+ * Arguments and results are those of stamp_inverse().
+ */
+#define STAMP_NOALLOC_SCRATCH_BYTES (4u << 20)
+int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N,
+                          void* Y, int y_dtype, void* stream);
 
 /*
  * The whole Algorithm in one call: Y = L^-1( Q(L X) Q(W)^T ) + bias.  Intermediates (codes,

@@ -23,7 +23,7 @@ EXPORTS = (
     "stamp_linear", "stamp_inverse", "stamp_linear_fused", "stamp_workspace_bytes_host",
     "stamp_linear_fused_host", "stamp_profile_gemm_events", "stamp_debug_transform",
     "stamp_debug_unpack_codes", "stamp_debug_gemm_i32", "stamp_last_device_status",
-    "stamp_last_launch_count", "stamp_status_string",
+    "stamp_last_launch_count", "stamp_status_string", "stamp_inverse_noalloc",
 )
 
 
@@ -153,6 +153,18 @@ def stamp_inverse(cfg: StampConfig, Yt: torch.Tensor, bias: Optional[torch.Tenso
     wp, wb = _ws_args(ws)
     _check(lib().stamp_inverse(ctypes.byref(cfg), _ptr(Yt), _ptr(bias), B, L, N, _ptr(Y), _dtype_code(Y), wp, wb,
                                _stream()), "stamp_inverse")
+    return Y
+
+
+def stamp_inverse_noalloc(cfg: StampConfig, Yt: torch.Tensor, bias: Optional[torch.Tensor],
+                          out_dtype=torch.float32, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """stamp_inverse without a workspace argument, for callers that may not allocate device memory:
+    the scratch between the passes is an array built into the library (a few MB per GPU), so sizes
+    beyond it raise StampError (status 6).  Calls on one device share that array: keep them ordered."""
+    B, L, N = Yt.shape
+    Y = out if out is not None else torch.empty((B, L, N), dtype=out_dtype, device=Yt.device)
+    _check(lib().stamp_inverse_noalloc(ctypes.byref(cfg), _ptr(Yt), _ptr(bias), B, L, N, _ptr(Y), _dtype_code(Y),
+                                       _stream()), "stamp_inverse_noalloc")
     return Y
 
 

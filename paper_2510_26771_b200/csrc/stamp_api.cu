@@ -460,6 +460,32 @@ static int weights_as_int8(const Problem& pb, const void* w, int w_format, int8_
   return STAMP_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// Built-in scratch of stamp_inverse_noalloc(): one array per GPU that loads the library, held
+// until the process exits.  In host code the array's name is only a handle for the runtime, not
+// a device address, so the address is looked up once per device with that device current.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[STAMP_NOALLOC_SCRATCH_BYTES];
+
+static int noalloc_scratch_base(uint8_t** out) {
+  constexpr int MAX_DEVICES = 64;
+  static std::mutex mu;
+  static uint8_t* base_of[MAX_DEVICES] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return STAMP_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!base_of[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return STAMP_ERR_CUDA;
+    }
+    base_of[dev] = static_cast<uint8_t*>(p);
+  }
+  *out = base_of[dev];
+  return STAMP_OK;
+}
+
 }  // namespace stamp
 
 // ============================================================================================
@@ -558,6 +584,24 @@ int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, i
   uint8_t* base = static_cast<uint8_t*>(ws);
   return run_inverse_generic(pb, Yt, bias, Y, y_dtype, reinterpret_cast<float*>(base + wl.ping),
                              reinterpret_cast<float*>(base + wl.pong), static_cast<cudaStream_t>(stream));
+}
+
+int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
+                          int y_dtype, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, 128, N, true, &pb);
+  if (rc) return rc;
+  if (!Yt || !Y || !dtype_ok(y_dtype)) return STAMP_ERR_INVALID_ARG;
+  // partial sums between the coarse-to-fine passes: the only scratch the inverse needs
+  const PassPlan pl = make_plan(pb.levels);
+  const size_t ping_bytes = pl.npass > 1 ? align256(((size_t)pb.M >> pl.p[0]) * pb.N * 4) : 0;
+  const size_t pong_bytes = pl.npass > 2 ? align256(((size_t)pb.M >> (pl.p[0] + pl.p[1])) * pb.N * 4) : 0;
+  if (ping_bytes + pong_bytes > (size_t)STAMP_NOALLOC_SCRATCH_BYTES) return STAMP_ERR_TOO_LARGE;
+  uint8_t* base = nullptr;
+  if ((rc = noalloc_scratch_base(&base))) return rc;
+  return run_inverse_generic(pb, Yt, bias, Y, y_dtype, reinterpret_cast<float*>(base),
+                             reinterpret_cast<float*>(base + ping_bytes), static_cast<cudaStream_t>(stream));
 }
 
 int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, const void* w, int w_format,
@@ -706,6 +750,7 @@ const char* stamp_status_string(int status) {
     case STAMP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case STAMP_ERR_CUDA: return "CUDA call failed";
     case STAMP_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case STAMP_ERR_TOO_LARGE: return "problem needs more scratch than the built-in array of the allocation-free call holds";
     default: return "unknown status";
   }
 }
