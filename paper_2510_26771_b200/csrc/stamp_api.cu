@@ -7,6 +7,7 @@
 #include <unordered_map>
 
 #include "common.cuh"
+#include "k_dct.cuh"
 #include "k_gemm.cuh"
 #include "k_generic.cuh"
 #include "k_haar_tq.cuh"
@@ -53,6 +54,7 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
     levels = cfg->levels ? cfg->levels : full;
     if (levels > full) return STAMP_ERR_UNSUPPORTED;
   }
+  if (cfg->transform == STAMP_T_DCT2 && n > 4096) return STAMP_ERR_UNSUPPORTED;  // dense n x n matrix in scratch
   out->B = B;
   out->L = L;
   out->K = K;
@@ -98,7 +100,7 @@ static PassPlan make_plan(int levels) {
 // Workspace layout (one layout for all calls of a problem size).
 // ------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, a8, w8, yt, total;
+  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, total;
 };
 static Workspace layout(const Problem& pb) {
   Workspace w{};
@@ -117,6 +119,7 @@ static Workspace layout(const Problem& pb) {
   w.atop = off;     off += align256((M >> 5) * (size_t)pb.K * 4);
   w.top_ping = off; off += align256((M >> 10) * (size_t)pb.K * 4);
   w.top_pong = off; off += align256((M >> 15) * (size_t)pb.K * 4);
+  w.dctmat = off; off += align256(pb.transform == STAMP_T_DCT2 ? (size_t)pb.n * pb.n * 4 : 0);
   w.a8 = off;     off += align256(M * (size_t)pb.K);
   w.w8 = off;     off += align256((size_t)pb.N * pb.K);
   w.yt = off;     off += align256(M * (size_t)pb.N * 4);
@@ -270,10 +273,28 @@ static int run_haar_passes(const void* in, bool in_bf16, int nseq, int Lin, int 
   return STAMP_OK;
 }
 
-// T = L X (Haar or identity), fp32, logical order; optionally the per-row |T| maxima.
+static int make_dct_matrix(int n, float* mat, cudaStream_t st) {
+  k_dct_matrix<<<(unsigned)(((long)n * n + 255) / 256), 256, 0, st>>>(n, mat);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// T = L X (Haar, identity or blockwise DCT-II), fp32, logical order; optionally the per-row |T| maxima.
 static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, float* T, unsigned* rowmax,
-                                 float* ping, float* pong, cudaStream_t st) {
-  if (pb.transform == STAMP_T_DCT2) return STAMP_ERR_UNSUPPORTED;
+                                 float* ping, float* pong, float* mat, cudaStream_t st) {
+  if (pb.transform == STAMP_T_DCT2) {
+    if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+    if (int rc = make_dct_matrix(pb.n, mat, st)) return rc;
+    const dim3 grid((unsigned)(pb.nseq * ((pb.n + 63) / 64)), (unsigned)((pb.K + 63) / 64));
+    if (x_dtype == STAMP_BF16)
+      k_dct_apply<false, __nv_bfloat16, float><<<grid, 256, 0, st>>>(mat, pb.n, static_cast<const __nv_bfloat16*>(X),
+                                                                      pb.K, T, nullptr, rowmax);
+    else
+      k_dct_apply<false, float, float><<<grid, 256, 0, st>>>(mat, pb.n, static_cast<const float*>(X), pb.K, T, nullptr,
+                                                              rowmax);
+    STAMP_CHECK_LAUNCH();
+    return STAMP_OK;
+  }
   return run_haar_passes(X, x_dtype == STAMP_BF16, pb.nseq, pb.n, pb.K, pb.levels, T, pb.n, 0, 0, rowmax,
                          (size_t)pb.M, ping, pong, st);
 }
@@ -296,8 +317,18 @@ static int launch_inv_pass(int P, const float* Yt, const float* ain, int n, int 
 
 // Y = L^T Yt + bias (Haar or identity), coarse passes first.
 static int run_inverse_generic(const Problem& pb, const float* Yt, const float* bias, void* Y, int y_dtype,
-                               float* ping, float* pong, cudaStream_t st) {
-  if (pb.transform == STAMP_T_DCT2) return STAMP_ERR_UNSUPPORTED;
+                               float* ping, float* pong, float* mat, cudaStream_t st) {
+  if (pb.transform == STAMP_T_DCT2) {
+    if (int rc = make_dct_matrix(pb.n, mat, st)) return rc;
+    const dim3 grid((unsigned)(pb.nseq * ((pb.n + 63) / 64)), (unsigned)((pb.N + 63) / 64));
+    if (y_dtype == STAMP_BF16)
+      k_dct_apply<true, float, __nv_bfloat16><<<grid, 256, 0, st>>>(mat, pb.n, Yt, pb.N, static_cast<__nv_bfloat16*>(Y),
+                                                                     bias, nullptr);
+    else
+      k_dct_apply<true, float, float><<<grid, 256, 0, st>>>(mat, pb.n, Yt, pb.N, static_cast<float*>(Y), bias, nullptr);
+    STAMP_CHECK_LAUNCH();
+    return STAMP_OK;
+  }
   const PassPlan pl = make_plan(pb.levels);
   // forward pass i covered levels (sum p[0..i-1], sum p[0..i]]; run them in reverse
   int jlo_of[8];
@@ -546,7 +577,7 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   TqChoice tc;
   if (choose_tq(pb, x_dtype, &tc)) return run_quantize_fast(pb, tc, X, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
   rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
-                             reinterpret_cast<float*>(base + w.pong), st);
+                             reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st);
   if (rc) return rc;
   return run_quant_rows(pb, T, rowmax, pb.n, nullptr, q_hi, q_lo, x_scale, st);
 }
@@ -583,7 +614,8 @@ int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, i
   if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
   uint8_t* base = static_cast<uint8_t*>(ws);
   return run_inverse_generic(pb, Yt, bias, Y, y_dtype, reinterpret_cast<float*>(base + wl.ping),
-                             reinterpret_cast<float*>(base + wl.pong), static_cast<cudaStream_t>(stream));
+                             reinterpret_cast<float*>(base + wl.pong), reinterpret_cast<float*>(base + wl.dctmat),
+                             static_cast<cudaStream_t>(stream));
 }
 
 int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
@@ -597,11 +629,13 @@ int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float*
   const PassPlan pl = make_plan(pb.levels);
   const size_t ping_bytes = pl.npass > 1 ? align256(((size_t)pb.M >> pl.p[0]) * pb.N * 4) : 0;
   const size_t pong_bytes = pl.npass > 2 ? align256(((size_t)pb.M >> (pl.p[0] + pl.p[1])) * pb.N * 4) : 0;
-  if (ping_bytes + pong_bytes > (size_t)STAMP_NOALLOC_SCRATCH_BYTES) return STAMP_ERR_TOO_LARGE;
+  const size_t mat_bytes = pb.transform == STAMP_T_DCT2 ? align256((size_t)pb.n * pb.n * 4) : 0;
+  if (ping_bytes + pong_bytes + mat_bytes > (size_t)STAMP_NOALLOC_SCRATCH_BYTES) return STAMP_ERR_TOO_LARGE;
   uint8_t* base = nullptr;
   if ((rc = noalloc_scratch_base(&base))) return rc;
   return run_inverse_generic(pb, Yt, bias, Y, y_dtype, reinterpret_cast<float*>(base),
-                             reinterpret_cast<float*>(base + ping_bytes), static_cast<cudaStream_t>(stream));
+                             reinterpret_cast<float*>(base + ping_bytes),
+                             reinterpret_cast<float*>(base + ping_bytes + pong_bytes), static_cast<cudaStream_t>(stream));
 }
 
 int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, const void* w, int w_format,
@@ -627,13 +661,14 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   if (choose_tq(pb, x_dtype, &tc)) {
     if ((rc = run_quantize_fast(pb, tc, X, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
   } else {
-    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, st))) return rc;
+    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
+      return rc;
     if ((rc = run_quant_rows(pb, T, rowmax, pb.n, a8, nullptr, nullptr, x_scale, st))) return rc;
   }
   const int8_t* w8 = nullptr;
   if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
   if ((rc = launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_F32, st))) return rc;
-  return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, st);
+  return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
 }
 
 static size_t dtype_size(int d) { return d == STAMP_BF16 ? 2 : 4; }
@@ -687,7 +722,8 @@ int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, i
     return run_quantize_fast(pb, tc, X, nullptr, nullptr, nullptr, reinterpret_cast<float*>(base + wl.xscale), T, base,
                              wl, static_cast<cudaStream_t>(stream));
   return run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + wl.ping),
-                               reinterpret_cast<float*>(base + wl.pong), static_cast<cudaStream_t>(stream));
+                               reinterpret_cast<float*>(base + wl.pong), reinterpret_cast<float*>(base + wl.dctmat),
+                               static_cast<cudaStream_t>(stream));
 }
 
 int stamp_debug_unpack_codes(const stamp_config* cfg, const void* q_hi, const void* q_lo, int B, int L, int K,

@@ -1,0 +1,105 @@
+"""Parity at the full sizes of the named configurations, in the launch configuration the
+benchmark times (stamp_linear_fused on bf16 activations with prepared int8 weight codes).
+
+The oracle's integer GEMM is a triple loop, so the output is compared on a sample of output
+channels: output channels are independent given the activation codes, and the weight generator
+reproduces any subset of rows of the full matrix.  Transformed values are compared on a sample
+of input channels (the sequence transform acts on every channel separately); scales and codes
+are compared in full.  Tolerances are those of the stage-wise parity tests.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2510_26771_b200 import inputs as gen
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+T_TOL = 1e-5
+CODE_FRAC = 1e-5
+Y_TOL = 1e-3
+
+
+def _scale_rtol(cfg):
+    """A scale is absmax / qmax of a transformed row, so it inherits the tolerance on T.  Haar
+    coefficients see at most log2(n) fp32 roundings (1e-6 holds); a DCT coefficient is an fp32 sum
+    of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised."""
+    return 1e-5 if cfg.transform == gen.T_DCT2 else 1e-6
+
+FULL = {
+    "llm_mlp_up": gen.config_llm_up(),
+    "dit_attn_proj": gen.config_dit_proj(),
+    "llm_down_proj": gen.config_llm_down(),
+    "sweep_L512_D2048": gen.config_sweep(512, 2048),
+    "sweep_L8192_D4096": gen.config_sweep(8192, 4096),
+    "sweep_L32768_D8192": gen.config_sweep(32768, 8192),
+}
+
+
+def _oracle_transform_cols(oracle, cfg, Xc):
+    """T = L X on a channel subset Xc [B, L, C] with the oracle's explicit matrix."""
+    n = cfg.block_len
+    if cfg.transform == gen.T_HAAR and n > 4096:
+        return oracle.apply_csr(oracle.haar_matrix_csr(n, cfg.levels), n, Xc)
+    return oracle.apply_dense(oracle.transform_matrix(cfg.transform, n, cfg.levels), Xc)
+
+
+@pytest.mark.parametrize("name", list(FULL))
+def test_full_size_parity(oracle, name):
+    import torch
+    from paper_2510_26771_b200 import binding as st
+    cfg = FULL[name]
+    B, L, K, N, M = cfg.B, cfg.L, cfg.K, cfg.N, cfg.M
+    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi)
+    X = gen.make_activation(cfg)
+    rng = np.random.default_rng(1234)
+    ncols = min(N, 64)
+    cols = np.sort(rng.choice(N, size=ncols, replace=False))
+    Wc = gen.make_weight(cfg, cols)
+    bias = gen.make_bias(cfg)
+    ref = oracle.stamp_linear(X, Wc, bias[cols], transform=cfg.transform, block=cfg.block, levels=cfg.levels,
+                              k_hi=cfg.k_hi, want=("x_scale", "q", "Y"))
+
+    Xd = H.to_device(X, cfg.dtype)
+    ws = st.alloc_workspace(c, B, L, K, N)
+
+    # a1 on a sample of input channels
+    chans = np.sort(rng.choice(K, size=min(K, 96), replace=False))
+    T_ref = _oracle_transform_cols(oracle, cfg, np.ascontiguousarray(X[:, :, chans])).reshape(M, -1)
+    T = st.stamp_debug_transform(c, Xd, ws)
+    T_s = T.reshape(M, K)[:, torch.from_numpy(chans).cuda()].cpu().numpy().astype(np.float64)
+    del T
+    assert H.rel_fro(T_s, T_ref) <= T_TOL
+    col_max = np.abs(T_ref).max(axis=1, keepdims=True)
+    assert np.all(np.abs(T_s - T_ref) <= T_TOL * np.maximum(col_max, 1e-30))
+
+    # a2-a3 in full
+    q_hi, q_lo, xs = st.stamp_quantize(c, Xd, ws)
+    assert np.allclose(xs.cpu().numpy().reshape(-1), ref["x_scale"], rtol=_scale_rtol(cfg), atol=0)
+    codes = st.stamp_debug_unpack_codes(c, q_hi, q_lo, B, L, K).cpu().numpy().reshape(M, K)
+    bad, worst = H.code_mismatch(codes, ref["q"])
+    print(f"[{name}] code mismatches {bad} of {codes.size} (max |diff| {worst})")
+    assert worst <= 1 and bad <= int(math.ceil(CODE_FRAC * codes.size))
+    del codes, q_hi, q_lo
+
+    # the whole layer as the benchmark runs it; fp32 and bf16 output
+    Wd = H.to_device(gen.make_weight(cfg), cfg.dtype)
+    wq, w_scale = st.stamp_quantize_weights(c, Wd)
+    w8 = st.stamp_prepare_weights(c, wq)
+    del Wd
+    bd = torch.from_numpy(bias).cuda()
+    cols_d = torch.from_numpy(cols).cuda()
+    Y = st.stamp_linear_fused(c, Xd, w8, st.W_INT8, w_scale, bd, ws)
+    Y_s = Y.reshape(M, N)[:, cols_d].cpu().numpy()
+    del Y
+    err = H.rel_fro(Y_s, ref["Y"])
+    print(f"[{name}] output relative Frobenius error {err:.2e} on {ncols} sampled channels")
+    assert err <= Y_TOL
+    Yb = st.stamp_linear_fused(c, Xd, w8, st.W_INT8, w_scale, bd, ws, out_dtype=torch.bfloat16)
+    Yb_s = Yb.reshape(M, N)[:, cols_d].float().cpu().numpy()
+    # bf16 output: the fp32 result rounded once (2^-9 relative) on top of the fp32 path's own error
+    assert H.rel_fro(Yb_s, ref["Y"]) <= Y_TOL + 2.0 ** -8
+    assert np.all(np.abs(Yb_s - Y_s) <= np.abs(Y_s) * 2.0 ** -8 + 1e-30)
+    assert st.stamp_last_device_status() == 0

@@ -17,6 +17,13 @@ CODE_FRAC = 1e-5
 Y_TOL = 1e-3
 
 
+def _scale_rtol(cfg):
+    """A scale is absmax / qmax of a transformed row, so it inherits the tolerance on T.  Haar
+    coefficients see at most log2(n) fp32 roundings (1e-6 holds); a DCT coefficient is an fp32 sum
+    of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised."""
+    return 1e-5 if cfg.transform == gen.T_DCT2 else 1e-6
+
+
 @pytest.fixture(scope="module")
 def st():
     import torch
@@ -52,6 +59,9 @@ CASES = {
     # wide feature axes: 8 and 4 tokens per CTA in the fused transform+quantize kernel
     "wide_k4096": gen.scaled(gen.config_llm_up(), L=256, K=4096, N=64, k_hi=8),
     "wide_k8192": gen.scaled(gen.config_sweep(512, 8192), L=128, K=8192, N=64, levels=5, k_hi=4),
+    # blockwise DCT-II: several blocks per sequence, ragged output-channel tile; a short block
+    "dct_blocks": gen.scaled(gen.config_llm_down(), B=2, L=512, K=384, N=136),
+    "dct_short_block": gen.scaled(gen.config_llm_down(), B=1, L=256, K=128, N=64, block=32, k_hi=4),
     # two levels only: no cluster tree, approximation rows quantized by the same kernel
     "two_levels": gen.scaled(gen.config_dit_proj(), B=2, L=256, K=1152, N=128, grid=16, levels=2, k_hi=64),
 }
@@ -78,7 +88,7 @@ def test_stagewise_parity(st, oracle, name):
     # a2-a3: scales and codes
     q_hi, q_lo, xs = st.stamp_quantize(c, Xd, ws)
     codes = st.stamp_debug_unpack_codes(c, q_hi, q_lo, B, L, K).cpu().numpy().reshape(-1, K)
-    assert np.allclose(xs.cpu().numpy().reshape(-1), ref["x_scale"], rtol=1e-6, atol=0)
+    assert np.allclose(xs.cpu().numpy().reshape(-1), ref["x_scale"], rtol=_scale_rtol(cfg), atol=0)
     bad, worst = H.code_mismatch(codes, ref["q"])
     print(f"[{name}] activation code mismatches: {bad} of {codes.size} (max |diff| {worst})")
     assert worst <= 1 and bad <= _allowed(codes.size), (bad, worst, codes.size)
