@@ -182,6 +182,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true",
                     help="timed region only (no side measurements, no CPU baseline): for profiler captures")
+    ap.add_argument("--stage", default="fused", choices=("fused", "quantize", "inverse"),
+                    help="with --quick: the call each step makes (the whole layer, or one of its passes alone)")
     args = ap.parse_args()
     cfg = workloads()[args.workload]
 
@@ -228,6 +230,15 @@ def main():
     def step(i):
         st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], st.W_INT8, w_scale, bias, ws, out=Y)
 
+    if args.quick and args.stage == "quantize":
+        def step(i):  # noqa: F811
+            st.stamp_quantize(c, Xs[i % n_x], ws)
+    elif args.quick and args.stage == "inverse":
+        Yt_in = torch.randn((B, L, N), device="cuda")
+
+        def step(i):  # noqa: F811
+            st.stamp_inverse(c, Yt_in, bias, ws, out=Y)
+
     for i in range(warmup):
         step(i)
     launches_per_step = st.stamp_last_launch_count()
@@ -264,7 +275,7 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
     ms_per_step = total_ms / steps
-    gemm_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(g0, g1))
+    gemm_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(g0, g1)) if args.stage == "fused" or not args.quick else 0.0
     status = st.stamp_last_device_status()
 
     # keep the GPU under the same load a little longer if the timed region was too short to sample clocks
@@ -289,10 +300,11 @@ def main():
         return
 
     if args.quick:
-        gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
+        gemm_tops = ops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
         print(json.dumps({"metric": "stamp_linear_tops", "value": value, "unit": "TOPS", "n_gpus": world,
                           "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "quick": True,
-                          "config": {"workload": cfg.name}, "extra": {"gemm_ms": gemm_ms, "gemm_tops": gemm_tops},
+                          "config": {"workload": cfg.name, "stage": args.stage},
+                          "extra": {"gemm_ms": gemm_ms, "gemm_tops": gemm_tops},
                           "gpu_launches": launches_per_step * steps, "clocks": clocks}), flush=True)
         return
 

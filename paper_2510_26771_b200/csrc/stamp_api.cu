@@ -10,7 +10,7 @@
 #include "k_dct.cuh"
 #include "k_gemm.cuh"
 #include "k_generic.cuh"
-#include "k_haar_tq.cuh"
+#include "k_haar_cq.cuh"
 #include "stamp.h"
 
 namespace stamp {
@@ -115,10 +115,11 @@ static Workspace layout(const Problem& pb) {
   w.T = off;      off += align256(M * (size_t)pb.K * 4);
   w.ping = off;   off += align256(ping_rows * KN * 4);
   w.pong = off;   off += align256(pong_rows * KN * 4);
-  // level-5-or-coarser sums leaving the fused transform+quantize kernel, and its top passes
-  w.atop = off;     off += align256((M >> 5) * (size_t)pb.K * 4);
-  w.top_ping = off; off += align256((M >> 10) * (size_t)pb.K * 4);
-  w.top_pong = off; off += align256((M >> 15) * (size_t)pb.K * 4);
+  // un-normalised sums handed from one launch of the fused transform+quantize kernel to the next
+  // (at least 3 levels per launch but the last, so each buffer is 1/8 of the one before at most)
+  w.atop = off;     off += align256((M >> 3) * (size_t)pb.K * 4);
+  w.top_ping = off; off += align256((M >> 6) * (size_t)pb.K * 4);
+  w.top_pong = off; off += align256((M >> 9) * (size_t)pb.K * 4);
   w.dctmat = off; off += align256(pb.transform == STAMP_T_DCT2 ? (size_t)pb.n * pb.n * 4 : 0);
   w.a8 = off;     off += align256(M * (size_t)pb.K);
   w.w8 = off;     off += align256((size_t)pb.N * pb.K);
@@ -372,57 +373,102 @@ static int run_quant_rows(const Problem& pb, const float* T, const unsigned* row
 }
 
 // ------------------------------------------------------------------------------------------
-// Fused Haar transform + quantizer (bf16 input): one cluster kernel for the first D levels, the
-// general passes for the few coarse rows above.
+// Fused Haar transform + quantizer: cluster kernel, up to five levels per launch.
 // ------------------------------------------------------------------------------------------
-struct TqChoice {
-  int G, m, tree, D;
-  size_t smem;
+struct CqChoice {
+  int C;     // CTAs per cluster = strips along the feature axis
+  int NT;    // threads per CTA
+  int NCH;   // channel pairs per thread
+  int pmax;  // Haar levels per launch at most
 };
-static bool choose_tq(const Problem& pb, int x_dtype, TqChoice* c) {
-  if (pb.transform != STAMP_T_HAAR || x_dtype != STAMP_BF16 || pb.levels < 2) return false;
-  const int cand[3] = {16, 8, 4};
-  int G = 0;
-  for (int i = 0; i < 3; ++i) {
-    const int g = cand[i], m = ilog2(g);
-    if (m > pb.levels) continue;
-    const size_t slab = (size_t)g * pb.K * 2;
-    if (slab <= 65536 || (g == 4 && slab + (size_t)pb.K * 4 <= 200 * 1024)) {
-      G = g;
-      break;
+// Smallest number of strips for which a CTA of at most 512 threads covers its strip with one
+// (else two) channel pairs per thread.  False when the feature axis is too long for 8 CTAs.
+static bool choose_cq(int K, CqChoice* c) {
+  for (int nch = 1; nch <= 2; ++nch)
+    for (int C = 1; C <= 8; ++C) {
+      const int pairs = (K / 2 + C - 1) / C;
+      const int nt = (((pairs + nch - 1) / nch) + 31) / 32 * 32;
+      if (nt <= 512) {
+        c->C = C;
+        c->NT = nt;
+        c->NCH = nch;
+        c->pmax = nch == 1 ? 5 : 4;
+        return true;
+      }
     }
-  }
-  if (!G) return false;
-  c->G = G;
-  c->m = ilog2(G);
-  c->tree = pb.levels - c->m < 3 ? pb.levels - c->m : 3;
-  c->D = c->m + c->tree;
-  c->smem = G == 16 ? tq_smem_bytes<16>(pb.K) : G == 8 ? tq_smem_bytes<8>(pb.K) : tq_smem_bytes<4>(pb.K);
-  return true;
+  return false;
 }
 
-template <int G>
-static int launch_tq(const TqParams& tp, const TqChoice& c, long M, cudaStream_t st) {
-  auto kern = k_haar_tq<G>;
+static PassPlan make_plan_max(int levels, int pmax) {
+  PassPlan pl{};
+  int rem = levels;
+  if (rem == 0) {
+    pl.npass = 1;
+    pl.p[0] = 0;
+    return pl;
+  }
+  while (rem > 0) {
+    const int p = rem > pmax ? pmax : rem;
+    pl.p[pl.npass++] = p;
+    rem -= p;
+  }
+  return pl;
+}
+
+template <int P, int NCH, typename TIn, int OUT>
+static int launch_cq_t(CqParams cp, const CqChoice& c, cudaStream_t st) {
+  auto kern = k_haar_cq<P, NCH, TIn, OUT>;
+  constexpr bool STAGED = sizeof(TIn) == 2;
+  size_t smem = CQ_TAIL_BYTES;
+  cp.nstages = 1;
+  if (STAGED) {
+    const size_t slab = cq_slab_bytes<P, TIn>(cp.Kc);
+    size_t ns = (200 * 1024 - CQ_TAIL_BYTES) / slab;
+    ns = ns > 4 ? 4 : ns;
+    if (ns < 2) return STAMP_ERR_UNSUPPORTED;
+    cp.nstages = (int)ns;
+    smem += slab * ns;
+  }
   static size_t attr_smem = 0;
-  if (c.smem > attr_smem) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem) != cudaSuccess)
+  if (smem > attr_smem) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return STAMP_ERR_CUDA;
-    attr_smem = c.smem;
+    attr_smem = smem;
   }
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3((unsigned)(M / G));
-  lc.blockDim = dim3(TQ_THREADS);
-  lc.dynamicSmemBytes = c.smem;
+  lc.blockDim = dim3((unsigned)c.NT);
+  lc.dynamicSmemBytes = smem;
   lc.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = 1u << c.tree;
+  at[0].val.clusterDim.x = (unsigned)c.C;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   lc.attrs = at;
   lc.numAttrs = 1;
-  if (cudaLaunchKernelEx(&lc, kern, tp) != cudaSuccess) {
+  // persistent clusters: as many as can be resident at once (cached per launch shape)
+  static std::mutex mu;
+  static std::unordered_map<unsigned long long, int> resident;
+  const unsigned long long key = ((unsigned long long)smem << 24) | ((unsigned long long)c.NT << 8) | (unsigned)c.C;
+  int ncl = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    auto itr = resident.find(key);
+    if (itr != resident.end()) {
+      ncl = itr->second;
+    } else {
+      lc.gridDim = dim3((unsigned)(c.C * sm_count()));
+      if (cudaOccupancyMaxActiveClusters(&ncl, kern, &lc) != cudaSuccess || ncl <= 0) {
+        cudaGetLastError();
+        ncl = sm_count() / c.C;
+        if (ncl < 1) ncl = 1;
+      }
+      resident[key] = ncl;
+    }
+  }
+  if ((long)ncl > cp.ngroups) ncl = (int)cp.ngroups;
+  lc.gridDim = dim3((unsigned)(ncl * c.C));
+  if (cudaLaunchKernelEx(&lc, kern, cp) != cudaSuccess) {
     cudaGetLastError();
     return STAMP_ERR_CUDA;
   }
@@ -430,43 +476,69 @@ static int launch_tq(const TqParams& tp, const TqChoice& c, long M, cudaStream_t
   return STAMP_OK;
 }
 
-// Transform + quantize through the fused kernel.  Any of a8 / (q_hi, q_lo) / T_out may be null.
-static int run_quantize_fast(const Problem& pb, const TqChoice& c, const void* X, int8_t* a8, void* q_hi, void* q_lo,
-                             float* x_scale, float* T_out, uint8_t* base, const Workspace& wl, cudaStream_t st) {
-  TqParams tp{};
-  tp.X = static_cast<const __nv_bfloat16*>(X);
-  tp.K = pb.K;
-  tp.n = pb.n;
-  tp.levels = pb.levels;
-  tp.k_hi = pb.k_hi;
-  tp.qmax_hi = pb.qmax_hi;
-  tp.qmax_lo = pb.qmax_lo;
-  tp.tree_steps = c.tree;
-  tp.a8 = a8;
-  tp.q_hi = static_cast<int8_t*>(q_hi);
-  tp.q_lo = static_cast<uint8_t*>(q_lo);
-  tp.x_scale = x_scale;
-  tp.T_out = T_out;
-  const bool has_top = pb.levels > c.D;
-  float* atop = reinterpret_cast<float*>(base + wl.atop);
-  tp.atop = has_top ? atop : nullptr;
-  int rc = c.G == 16 ? launch_tq<16>(tp, c, pb.M, st) : c.G == 8 ? launch_tq<8>(tp, c, pb.M, st)
-                                                                 : launch_tq<4>(tp, c, pb.M, st);
-  if (rc || !has_top) return rc;
-  // the remaining levels act on the level-D sums: a short sequence of n >> D rows per block
-  const int n_top = pb.n >> c.D;
-  float* T_top = reinterpret_cast<float*>(base + wl.T);
-  unsigned* rowmax_top = reinterpret_cast<unsigned*>(base + wl.rowmax);
-  float* tping = reinterpret_cast<float*>(base + wl.top_ping);
-  float* tpong = reinterpret_cast<float*>(base + wl.top_pong);
-  rc = run_haar_passes(atop, false, pb.nseq, n_top, pb.K, pb.levels - c.D, T_top, n_top, 0, c.D, rowmax_top,
-                       (size_t)pb.nseq * n_top, tping, tpong, st);
-  if (rc) return rc;
-  if ((rc = run_quant_rows(pb, T_top, rowmax_top, n_top, a8, q_hi, q_lo, x_scale, st))) return rc;
-  if (T_out)  // debug export: the same coarse rows once more, written at their logical place
-    rc = run_haar_passes(atop, false, pb.nseq, n_top, pb.K, pb.levels - c.D, T_out, pb.n, c.D, 0, nullptr, 0, tping,
-                         tpong, st);
-  return rc;
+template <int NCH, typename TIn, int OUT>
+static int launch_cq_p(int P, const CqParams& cp, const CqChoice& c, cudaStream_t st) {
+  switch (P) {
+    case 0: return launch_cq_t<0, NCH, TIn, OUT>(cp, c, st);
+    case 1: return launch_cq_t<1, NCH, TIn, OUT>(cp, c, st);
+    case 2: return launch_cq_t<2, NCH, TIn, OUT>(cp, c, st);
+    case 3: return launch_cq_t<3, NCH, TIn, OUT>(cp, c, st);
+    case 4: return launch_cq_t<4, NCH, TIn, OUT>(cp, c, st);
+    default:
+      if constexpr (NCH == 1) return launch_cq_t<5, NCH, TIn, OUT>(cp, c, st);
+      return STAMP_ERR_UNSUPPORTED;
+  }
+}
+template <int OUT>
+static int launch_cq_o(int P, bool bf16_in, const CqParams& cp, const CqChoice& c, cudaStream_t st) {
+  if (bf16_in)
+    return c.NCH == 1 ? launch_cq_p<1, __nv_bfloat16, OUT>(P, cp, c, st) : launch_cq_p<2, __nv_bfloat16, OUT>(P, cp, c, st);
+  return c.NCH == 1 ? launch_cq_p<1, float, OUT>(P, cp, c, st) : launch_cq_p<2, float, OUT>(P, cp, c, st);
+}
+
+// Haar (or identity) transform + quantizer through the cluster kernel: one launch per group of
+// levels, each launch quantizing its own detail rows and handing fp32 sums to the next one.
+// Exactly one kind of output besides the scales: a8, or (q_hi, q_lo), or T_out.
+static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, int x_dtype, int8_t* a8, void* q_hi,
+                           void* q_lo, float* x_scale, float* T_out, uint8_t* base, const Workspace& wl,
+                           cudaStream_t st) {
+  const PassPlan pl = make_plan_max(pb.levels, c.pmax);
+  float* bufs[3] = {reinterpret_cast<float*>(base + wl.atop), reinterpret_cast<float*>(base + wl.top_ping),
+                    reinterpret_cast<float*>(base + wl.top_pong)};
+  CqParams cp{};
+  cp.K = pb.K;
+  cp.Kc = 2 * c.NCH * c.NT;
+  cp.n = pb.n;
+  cp.k_hi = pb.k_hi;
+  cp.qmax_hi = (float)pb.qmax_hi;
+  cp.qmax_lo = (float)pb.qmax_lo;
+  cp.a8 = a8;
+  cp.q_hi = static_cast<int8_t*>(q_hi);
+  cp.q_lo = static_cast<uint8_t*>(q_lo);
+  cp.x_scale = x_scale;
+  cp.T_out = T_out;
+  const void* in = X;
+  int Lin = pb.n, lvl0 = 0;
+  for (int i = 0; i < pl.npass; ++i) {
+    const int P = pl.p[i];
+    const bool last = (i == pl.npass - 1);
+    // launch i writes into buffer min(i, 1 + (i - 1) % 2): atop, then ping / pong alternately
+    float* aout = last ? nullptr : bufs[i == 0 ? 0 : 1 + ((i - 1) & 1)];
+    cp.in = in;
+    cp.aout = aout;
+    cp.Lin = Lin;
+    cp.lvl0 = lvl0;
+    cp.ngroups = (long)pb.nseq * (Lin >> P);
+    const bool bf16_in = (i == 0 && x_dtype == STAMP_BF16);
+    const int rc = a8 ? launch_cq_o<CQ_OUT_A8>(P, bf16_in, cp, c, st)
+                      : T_out ? launch_cq_o<CQ_OUT_T>(P, bf16_in, cp, c, st)
+                              : launch_cq_o<CQ_OUT_PUBLIC>(P, bf16_in, cp, c, st);
+    if (rc) return rc;
+    in = aout;
+    Lin >>= P;
+    lvl0 += P;
+  }
+  return STAMP_OK;
 }
 
 static int run_unpack_codes(const Problem& pb, const void* q_hi, const void* q_lo, int8_t* out, cudaStream_t st) {
@@ -574,8 +646,9 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   uint8_t* base = static_cast<uint8_t*>(ws);
   float* T = reinterpret_cast<float*>(base + w.T);
   unsigned* rowmax = reinterpret_cast<unsigned*>(base + w.rowmax);
-  TqChoice tc;
-  if (choose_tq(pb, x_dtype, &tc)) return run_quantize_fast(pb, tc, X, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
+  CqChoice cc;
+  if (pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc))
+    return run_quantize_cq(pb, cc, X, x_dtype, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
   rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
                              reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st);
   if (rc) return rc;
@@ -657,9 +730,9 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
   float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
   float* yt = reinterpret_cast<float*>(base + wl.yt);
-  TqChoice tc;
-  if (choose_tq(pb, x_dtype, &tc)) {
-    if ((rc = run_quantize_fast(pb, tc, X, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
+  CqChoice cc;
+  if (pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc)) {
+    if ((rc = run_quantize_cq(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
   } else {
     if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
       return rc;
@@ -717,10 +790,10 @@ int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, i
   const Workspace wl = layout(pb);
   if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
   uint8_t* base = static_cast<uint8_t*>(ws);
-  TqChoice tc;
-  if (choose_tq(pb, x_dtype, &tc))  // same kernels as the product path, with the fp32 export switched on
-    return run_quantize_fast(pb, tc, X, nullptr, nullptr, nullptr, reinterpret_cast<float*>(base + wl.xscale), T, base,
-                             wl, static_cast<cudaStream_t>(stream));
+  CqChoice cc;
+  if (pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc))  // the product path's kernel with the fp32 export on
+    return run_quantize_cq(pb, cc, X, x_dtype, nullptr, nullptr, nullptr, reinterpret_cast<float*>(base + wl.xscale), T,
+                           base, wl, static_cast<cudaStream_t>(stream));
   return run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + wl.ping),
                                reinterpret_cast<float*>(base + wl.pong), reinterpret_cast<float*>(base + wl.dctmat),
                                static_cast<cudaStream_t>(stream));
