@@ -1,26 +1,31 @@
 // Fused Haar transform + per-token mixed-precision quantizer (Algorithm lines "X <- L X" and
-// "x_i <- Q(x_i; b_i)"): one pass over the activation in HBM, up to five Haar levels per launch.
+// "x_i <- Q(x_i; b_i)"): one pass over the activation in HBM, up to four Haar levels per launch.
 //
 // The two axes pull in different directions: a transformed token's scale needs the maximum over
 // ALL K channels of its row, while a Haar coefficient of level l needs 2^l consecutive tokens of
-// ONE channel.  Here a thread owns two adjacent channels of a group of G = 2^P consecutive tokens
-// and keeps all G coefficients of both channels in registers; a CTA owns a strip of channels; a
-// thread-block cluster of C CTAs covers the whole feature axis.  The only thing the CTAs of a
-// cluster exchange is the G per-row maxima of their strips, read from each other's shared memory
-// (distributed shared memory, plain ld.shared::cluster) after one cluster barrier.  Every detail
-// row of the P levels is then quantized from registers and stored; the group's un-normalised sum
-// row (1/G of the data, fp32) is the input of the next launch, which runs the same kernel on
-// fp32 rows, until the last launch also quantizes the approximation rows.
+// ONE channel.  Here a thread owns four adjacent channels of a group of G = 2^P consecutive tokens
+// and keeps all G coefficients of its channels in registers; a CTA owns a strip of channels; a
+// thread-block cluster of C CTAs covers the whole feature axis (C = 1 up to 2048 channels).  The
+// only thing the CTAs of a cluster exchange is the G per-row maxima of their strips: each CTA
+// posts them into a mailbox in every peer's shared memory with asynchronous remote stores whose
+// arrival is counted on an mbarrier of the receiving CTA (st.async, distributed shared memory), so
+// there is no cluster-wide barrier and no fence on the sending side in the loop.  Every detail row of the P levels is then quantized from registers and stored; the
+// group's un-normalised sum row (1/G of the data, fp32) is the input of the next launch, which
+// runs the same kernel on fp32 rows, until the last launch also quantizes the approximation rows.
 //
 // Clusters are persistent: each walks over token groups with a stride of the number of clusters.
 // bf16 activations are staged through a shared-memory ring filled by bulk asynchronous copies
 // (one per token row of the strip) issued NS - 1 groups ahead, so HBM reads stay in flight while
 // a group is being reduced, exchanged and stored; fp32 rows (the small later launches) are read
-// with plain coalesced loads.
+// with plain coalesced 128-bit loads.
 //
-// Arithmetic: butterflies on un-normalised sums with packed fp32x2 operations, one multiplication
-// by 2^(-j/2) per coefficient (head + tail FMA), scale = absmax / qmax by IEEE division, t / scale
-// by reciprocal + one Newton step, round-to-nearest-even by the 1.5 * 2^23 trick.
+// Arithmetic.  Butterflies run on un-normalised sums with packed fp32x2 operations.  A level-j
+// coefficient is the un-normalised value times 2^(-j/2) = c * 2^(-(j >> 1)) with c = 1 (j even) or
+// 1/sqrt 2 (j odd).  Only c is applied to the data (head + tail FMA, so the product is rounded
+// once); the exact power of two is carried by the scale instead: with t' = fl(v c) and
+// s' = fl(absmax' / qmax), t / s and t' / s' are the same fp32 quotient and the stored scale is
+// s' * 2^(-(j >> 1)).  t' / s' is evaluated as reciprocal + one Newton step, and rounded to the
+// nearest integer (ties to even) by adding 1.5 * 2^23.
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
@@ -31,7 +36,7 @@ struct CqParams {
   const void* in;   // [nseq, Lin, K] bf16 / fp32 activations, or fp32 un-normalised sums over 2^lvl0 tokens
   float* aout;      // [nseq, Lin >> P, K] un-normalised sums over 2^(lvl0+P) tokens; nullptr in the last launch
   int K;            // channels
-  int Kc;           // channels per CTA strip (= 2 * NCH * blockDim.x)
+  int Kc;           // channels per CTA strip (= 4 * blockDim.x)
   int Lin;          // input rows per transform block in this launch
   int n;            // tokens per transform block
   int lvl0;         // Haar levels already applied to the input rows
@@ -39,82 +44,90 @@ struct CqParams {
   float qmax_hi, qmax_lo;
   long ngroups;     // nseq * (Lin >> P)
   int nstages;      // depth of the shared-memory ring (bf16 input only)
-  int8_t* a8;       // [M, K] one code per int8 (GEMM operand) or nullptr
-  int8_t* q_hi;     // public outputs or nullptr
+  int8_t* a8;       // [M, K] one code per int8 (GEMM operand)      -- CQ_OUT_A8
+  int8_t* q_hi;     // public packed outputs                         -- CQ_OUT_PUBLIC
   uint8_t* q_lo;
   float* x_scale;   // [M]
-  float* T_out;     // [M, K] transformed values (debug export) or nullptr
+  float* T_out;     // [M, K] transformed values (debug export)      -- CQ_OUT_T
 };
 
-constexpr float CQ_MAGIC = 12582912.0f;          // 1.5 * 2^23
+constexpr float CQ_MAGIC = 12582912.0f;            // 1.5 * 2^23
 constexpr long long CQ_WAIT_LIMIT = 2000000000LL;  // SM clocks before a wait on a copy gives up
+constexpr float CQ_RSQRT2_HI = 0.707106769084930419921875f;  // fp32(1/sqrt 2)
+constexpr float CQ_RSQRT2_LO = 1.2101617101e-8f;             // 1/sqrt 2 - fp32(1/sqrt 2)
 
 // What a launch writes besides the scales: the GEMM's int8 operand, the public packed codes, or
 // the fp32 transformed values (debug export).
 enum CqOut { CQ_OUT_A8 = 0, CQ_OUT_PUBLIC = 1, CQ_OUT_T = 2 };
 
-// Row table in shared memory, rebuilt for every group; constants are stored twice so that a
-// 128-bit load yields register pairs the packed fp32x2 instructions can use directly.
-struct CqRowA { float nhi0, nhi1, nlo0, nlo1; };      // 2^(-j/2) as head + tail
-struct CqRowB { float inv0, inv1, ns0, ns1; };        // 1 / scale and -scale
-struct CqRowC { int row; int pub; };                  // logical row; row in q_hi / q_lo, bit 31 set for 8-bit rows
-
 __device__ __forceinline__ float2 cq_f2(float a) { return make_float2(a, a); }
 
-// Shared memory: [ring: nstages x G x Kc x sizeof(TIn)] [full barriers: 8 x u64] [maxima: 2 x 32 u32]
-//                [row tables: 32 x (16 + 16 + 8) bytes]
+// Shared memory: [ring: nstages x G x Kc x sizeof(TIn)] [full barriers: 8 x u64] [mailbox barriers: 2 x u64]
+//   [maxima: 2 x 16 u32] [mailbox: 2 x 8 CTAs x 16 u32]
+//   [per row: {1/s', 1/s', -s', -s'} 16 B] [per row: {logical row, row in q_hi / q_lo | 8-bit flag,
+//   2^(-(j>>1)) bits, 0} 16 B]
 template <int P, typename TIn>
 __host__ __device__ constexpr size_t cq_slab_bytes(int Kc) { return (size_t)(1 << P) * Kc * sizeof(TIn); }
-constexpr size_t CQ_TAIL_BYTES = 8 * 8 + 2 * 32 * 4 + 32 * 40;
+constexpr size_t CQ_TAIL_BYTES = 8 * 8 + 64 + 2 * 16 * 4 + 2 * 8 * 16 * 4 + 16 * 16 + 16 * 16;
 
-template <int P, int NCH, typename TIn, int OUT>
+// LODD = lvl0 & 1: with it the parity of every row's level, hence whether it needs the 1/sqrt 2
+// factor, is known at compile time.
+template <int P, typename TIn, int OUT, int LODD>
 __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
   constexpr int G = 1 << P;
   constexpr bool STAGED = (sizeof(TIn) == 2);
-  static_assert(G * NCH <= 32, "a thread holds at most 32 channel pairs");
+  static_assert(P <= 4, "a thread holds 16 rows of four channels at most");
   extern __shared__ __align__(128) uint8_t cq_smem[];
   const size_t slab = STAGED ? cq_slab_bytes<P, TIn>(p.Kc) : 0;
   uint8_t* tail = cq_smem + (STAGED ? slab * p.nstages : 0);
   uint64_t* full = reinterpret_cast<uint64_t*>(tail);
-  unsigned* mymax = reinterpret_cast<unsigned*>(tail + 64);   // [2][32]
-  float4* tabA = reinterpret_cast<float4*>(tail + 64 + 256);          // [32] CqRowA
-  float4* tabB = reinterpret_cast<float4*>(tail + 64 + 256 + 512);    // [32] CqRowB
-  int2* tabC = reinterpret_cast<int2*>(tail + 64 + 256 + 1024);       // [32] CqRowC
+  uint64_t* mb = reinterpret_cast<uint64_t*>(tail + 64);           // [2] one per mailbox buffer
+  unsigned* mymax = reinterpret_cast<unsigned*>(tail + 128);       // [2][16]
+  unsigned* mailbox = reinterpret_cast<unsigned*>(tail + 256);     // [2][8][16]
+  float4* tabB = reinterpret_cast<float4*>(tail + 1280);           // [16]
+  int4* tabC = reinterpret_cast<int4*>(tail + 1536);               // [16]
   __shared__ uint32_t abort_word;
 
-  const int tid = threadIdx.x, NT = blockDim.x;
+  const int tid = threadIdx.x;
   const int lane = tid & 31;
   unsigned csize, rank;
   asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(csize));
   rank = ptx::cluster_ctarank();
   const long cid = blockIdx.x / csize, ncl = gridDim.x / csize;
+  const int K = p.K;
   const int cbase = static_cast<int>(rank) * p.Kc;
-  const int cvalid = max(0, min(p.Kc, p.K - cbase));   // channels of this strip (0: the strip is empty)
+  const int cvalid = max(0, min(p.Kc, K - cbase));   // channels of this strip (0: the strip is empty)
   const uint32_t row_bytes = static_cast<uint32_t>(cvalid) * sizeof(TIn);
-  const int gps = p.Lin >> P;                           // groups per transform block
+  const int gps = p.Lin >> P;                         // groups per transform block
   const bool last = (p.aout == nullptr);
   const int NS = p.nstages;
+  const bool valid = 4 * tid < cvalid;                // this thread's four channels exist
+  // threads past the end of a ragged strip redo its last quad: same maxima, nothing stored
+  const int qe = valid ? tid : max(cvalid / 4 - 1, 0);
+  const int c0 = cbase + 4 * tid;
 
+  if (tid < 32) mymax[tid] = 0u;
   if (tid == 0) {
     abort_word = 0;
-    if (STAGED) {
+    if (STAGED)
       for (int s = 0; s < NS; ++s) ptx::mbar_init(&full[s], 1);
-      ptx::fence_mbar_init();
-    }
+    ptx::mbar_init(&mb[0], 1);
+    ptx::mbar_init(&mb[1], 1);
+    ptx::fence_mbar_init();
   }
-  __syncthreads();
+  // every CTA of the cluster has initialised its barriers before anyone posts to them
+  ptx::cluster_sync();
 
   // warp 0 brings one group's rows of this strip into a ring stage: lane r copies token row r
   auto issue_load = [&](long grp, int stage) {
     if (!STAGED || cvalid == 0 || tid >= 32) return;
     const long sq = grp / gps;
     const long g = grp - sq * gps;
-    const uint8_t* src = static_cast<const uint8_t*>(p.in) +
-                         (((sq * p.Lin + g * G) * (long)p.K + cbase) * (long)sizeof(TIn));
+    const uint8_t* src = static_cast<const uint8_t*>(p.in) + (((sq * p.Lin + g * G) * (long)K + cbase) * (long)sizeof(TIn));
     uint8_t* dst = cq_smem + stage * slab;
     if (lane == 0) ptx::mbar_arrive_expect_tx(&full[stage], row_bytes * G);
     __syncwarp();
-    if (lane < G) ptx::bulk_load(dst + (size_t)lane * row_bytes, src + (size_t)lane * p.K * sizeof(TIn), row_bytes, &full[stage]);
+    if (lane < G) ptx::bulk_load(dst + (size_t)lane * row_bytes, src + (size_t)lane * K * sizeof(TIn), row_bytes, &full[stage]);
   };
 
   if (STAGED)
@@ -133,146 +146,164 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
       const long nxt = grp + (long)(NS - 1) * ncl;
       if (nxt < p.ngroups) issue_load(nxt, static_cast<int>((it + NS - 1) % NS));
     }
-    if (tid < 32) mymax[b * 32 + tid] = 0u;
+    // this group's mailbox buffer expects G maxima from each CTA of the cluster (its previous use,
+    // two groups ago, was completed and read before this thread passed that group's barrier)
+    if (tid == 0) ptx::mbar_arrive_expect_tx(&mb[b], csize * G * 4u);
     if (STAGED && cvalid > 0 && ok) {
-      const bool got = ptx::mbar_wait_bounded(&full[stage], static_cast<uint32_t>((it / NS) & 1), &abort_word, CQ_WAIT_LIMIT);
-      if (!got) abort_word = 1;
+      // every thread waits for the copies itself (that also makes the data visible to it); a
+      // thread that gives up tells the others through the abort word their waits poll
+      if (!ptx::mbar_wait_bounded(&full[stage], static_cast<uint32_t>((it / NS) & 1), &abort_word, CQ_WAIT_LIMIT)) {
+        ok = false;
+        abort_word = 1;
+        raise_device_status(STAMP_ERR_TIMEOUT);
+      }
     }
-    __syncthreads();
-    if (ok && abort_word != 0) {
-      ok = false;
-      if (tid == 0) raise_device_status(STAMP_ERR_TIMEOUT);
-    }
-
     const long sq = grp / gps;
     const int g = static_cast<int>(grp - sq * gps);
 
-    // ---- load G tokens x NCH channel pairs, butterflies in registers (un-normalised)
-    float2 v[NCH][G];
-    bool valid[NCH];
+    // ---- load G tokens x 4 channels, butterflies in registers (un-normalised)
+    float2 v[2][G];
+    if (ok && cvalid > 0) {
+      if (STAGED) {
+        const uint8_t* s8 = cq_smem + stage * slab + 8 * qe;
 #pragma unroll
-    for (int j = 0; j < NCH; ++j) {
-      const int pr = tid + j * NT;          // channel pair inside the strip
-      valid[j] = ok && (2 * pr < cvalid);
+        for (int r = 0; r < G; ++r) {
+          const uint2 w = *reinterpret_cast<const uint2*>(s8 + r * row_bytes);
+          v[0][r] = make_float2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
+          v[1][r] = make_float2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+        }
+      } else {
+        const float* src = static_cast<const float*>(p.in) + ((sq * p.Lin + (long)g * G) * (long)K + cbase + 4 * qe);
 #pragma unroll
-      for (int r = 0; r < G; ++r) v[j][r] = cq_f2(0.f);
-      if (valid[j]) {
-        if (STAGED) {
-          const uint32_t* s32 = reinterpret_cast<const uint32_t*>(cq_smem + stage * slab) + pr;
-#pragma unroll
-          for (int r = 0; r < G; ++r) {
-            const uint32_t w = s32[(size_t)r * (row_bytes / 4)];
-            v[j][r] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
-          }
-        } else {
-          const float* src = static_cast<const float*>(p.in) + ((sq * p.Lin + (long)g * G) * (long)p.K + cbase + 2 * pr);
-#pragma unroll
-          for (int r = 0; r < G; ++r) v[j][r] = *reinterpret_cast<const float2*>(src + (long)r * p.K);
+        for (int r = 0; r < G; ++r) {
+          const float4 w = *reinterpret_cast<const float4*>(src + (long)r * K);
+          v[0][r] = make_float2(w.x, w.y);
+          v[1][r] = make_float2(w.z, w.w);
         }
       }
+    } else {
+#pragma unroll
+      for (int r = 0; r < G; ++r) v[0][r] = v[1][r] = cq_f2(0.f);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
 #pragma unroll
       for (int len = G; len > 1; len >>= 1) {
         float2 t[G];
 #pragma unroll
         for (int i = 0; i < len / 2; ++i) {
-          t[i] = __fadd2_rn(v[j][2 * i], v[j][2 * i + 1]);
-          t[len / 2 + i] = __ffma2_rn(v[j][2 * i + 1], cq_f2(-1.0f), v[j][2 * i]);
+          t[i] = __fadd2_rn(v[h][2 * i], v[h][2 * i + 1]);
+          t[len / 2 + i] = __ffma2_rn(v[h][2 * i + 1], cq_f2(-1.0f), v[h][2 * i]);
         }
 #pragma unroll
-        for (int i = 0; i < len; ++i) v[j][i] = t[i];
+        for (int i = 0; i < len; ++i) v[h][i] = t[i];
       }
     }
-    // v[j] is now [a | d_P | d_(P-1) (2) | ... | d_1 (G/2)]
+    // v[h] is now [a | d_P | d_(P-1) (2) | ... | d_1 (G/2)]
 
     // ---- per-row maxima of this strip: lane r of every warp collects row r, one atomic per lane
     unsigned keep = 0u;
 #pragma unroll
     for (int r = 0; r < G; ++r) {
-      float m = 0.f;
-#pragma unroll
-      for (int j = 0; j < NCH; ++j) m = fmaxf(m, fmaxf(fabsf(v[j][r].x), fabsf(v[j][r].y)));
+      const float m = fmaxf(fmaxf(fabsf(v[0][r].x), fabsf(v[0][r].y)), fmaxf(fabsf(v[1][r].x), fabsf(v[1][r].y)));
       const unsigned mm = __reduce_max_sync(0xffffffffu, __float_as_uint(m));
       keep = (lane == r) ? mm : keep;
     }
-    if (lane < G) atomicMax(&mymax[b * 32 + lane], keep);
+    if (lane < G) atomicMax(&mymax[b * 16 + lane], keep);
     __syncthreads();
-    ptx::cluster_arrive();
-    if (!last) {
-#pragma unroll
-      for (int j = 0; j < NCH; ++j)
-        if (valid[j])
-          *reinterpret_cast<float2*>(p.aout + ((sq * gps + g) * (long)p.K + cbase + 2 * (tid + j * NT))) = v[j][0];
+    if (tid < G) {
+      // post this strip's maxima to every CTA of the cluster (this one included) and clear them
+      const unsigned mine = mymax[b * 16 + tid];
+      mymax[b * 16 + tid] = 0u;
+      const uint32_t slot = ptx::smem_u32(&mailbox[(b * 8 + rank) * 16 + tid]);
+      const uint32_t bar = ptx::smem_u32(&mb[b]);
+      for (unsigned q = 0; q < csize; ++q) ptx::st_async_u32(ptx::mapa(slot, q), mine, ptx::mapa(bar, q));
     }
-    ptx::cluster_wait();
+    if (!last && valid && ok)
+      *reinterpret_cast<float4*>(p.aout + ((sq * gps + g) * (long)K + c0)) =
+          make_float4(v[0][0].x, v[0][0].y, v[1][0].x, v[1][0].y);
 
     // ---- row tables: maxima over the cluster, scales, output rows
+    if (tid < G) {
+      if (!ptx::mbar_wait_bounded_cluster(&mb[b], static_cast<uint32_t>((it >> 1) & 1), &abort_word, CQ_WAIT_LIMIT)) {
+        ok = false;
+        abort_word = 1;
+        raise_device_status(STAMP_ERR_TIMEOUT);
+      }
+    }
     if (tid < G && (tid > 0 || last)) {
       const int r = tid;
       unsigned um = 0;
-      const uint32_t local = ptx::smem_u32(&mymax[b * 32 + r]);
-      for (unsigned q = 0; q < csize; ++q) {
-        unsigned x;
-        asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(x) : "r"(ptx::mapa(local, q)));
-        um = max(um, x);
-      }
+      for (unsigned q = 0; q < csize; ++q) um = max(um, mailbox[(b * 8 + q) * 16 + r]);
       int k = 0;                       // r in [2^k, 2^(k+1)): detail row of local level P - k
       while ((2 << k) <= r) ++k;
       const int l = (r == 0) ? P : P - k;
       const int j = p.lvl0 + l;
       const int i_in_blk = (r == 0) ? g : (p.n >> j) + (g << k) + (r - (1 << k));
-      const HaarNorm h = haar_norm(j);
       const float u = __uint_as_float(um);
-      const float amax = fmaf(u, h.hi, u * h.lo);
+      const float amax = (j & 1) ? fmaf(u, CQ_RSQRT2_HI, u * CQ_RSQRT2_LO) : u;   // in units of 2^(-(j >> 1))
       const bool hi = i_in_blk < p.k_hi;
       const float qmax = hi ? p.qmax_hi : p.qmax_lo;
       const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
       const float inv = __fdiv_rn(1.0f, scale);
+      const float pw = __int_as_float((127 - (j >> 1)) << 23);                     // 2^(-(j >> 1))
       const long row = sq * p.n + i_in_blk;
       const long pub = hi ? sq * p.k_hi + i_in_blk : sq * (p.n - p.k_hi) + (i_in_blk - p.k_hi);
-      tabA[r] = make_float4(h.hi, h.hi, h.lo, h.lo);
       tabB[r] = make_float4(inv, inv, -scale, -scale);
-      tabC[r] = make_int2(static_cast<int>(row), static_cast<int>(pub) | (hi ? static_cast<int>(0x80000000u) : 0));
-      if (rank == 0 && ok) p.x_scale[row] = scale;
+      tabC[r] = make_int4(static_cast<int>(row), static_cast<int>(pub) | (hi ? static_cast<int>(0x80000000u) : 0),
+                          __float_as_int(pw), 0);
+      if (rank == 0 && ok) p.x_scale[row] = (amax > 0.f) ? scale * pw : 1.0f;
     }
     __syncthreads();
 
     // ---- normalise, quantize and store from registers
-#pragma unroll
-    for (int j = 0; j < NCH; ++j) {
-      if (!valid[j]) continue;
-      const int c = cbase + 2 * (tid + j * NT);
-      const int8_t* a8c = p.a8 + c;
-      const int8_t* qhc = p.q_hi + c;
-      const uint8_t* qlc = p.q_lo + (c >> 1);
-      const float* Tc = p.T_out + c;
+    if (valid && ok) {
 #pragma unroll
       for (int r = 0; r < G; ++r) {
         if (r == 0 && !last) continue;
-        const float4 A = tabA[r];
-        const int2 Cc = tabC[r];
-        const float2 t = __ffma2_rn(v[j][r], make_float2(A.x, A.y), __fmul2_rn(v[j][r], make_float2(A.z, A.w)));
+        // local level of row r: P for the sum row, P - floor(log2 r) for a detail row
+        int lg = 0;
+#pragma unroll
+        for (int s = 1; s < 5; ++s) lg += (r >> s) ? 1 : 0;
+        const int l = (r == 0) ? P : P - lg;
+        const bool odd = ((LODD + l) & 1) != 0;
+        const int4 Cc = tabC[r];
+        float2 t[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          t[h] = odd ? __ffma2_rn(v[h][r], cq_f2(CQ_RSQRT2_HI), __fmul2_rn(v[h][r], cq_f2(CQ_RSQRT2_LO))) : v[h][r];
         if (OUT == CQ_OUT_T) {
-          *const_cast<float2*>(reinterpret_cast<const float2*>(Tc + (long)Cc.x * p.K)) = t;
+          const float pw = __int_as_float(Cc.z);
+          *reinterpret_cast<float4*>(p.T_out + ((long)Cc.x * K + c0)) =
+              make_float4(t[0].x * pw, t[0].y * pw, t[1].x * pw, t[1].y * pw);
           continue;
         }
         const float4 Bv = tabB[r];
-        const float2 inv2 = make_float2(Bv.x, Bv.y);
-        const float2 q0 = __fmul2_rn(t, inv2);
-        const float2 rem = __ffma2_rn(q0, make_float2(Bv.z, Bv.w), t);
-        const float2 q = __fadd2_rn(__ffma2_rn(rem, inv2, q0), cq_f2(CQ_MAGIC));
-        const uint32_t bx = __float_as_uint(q.x), by = __float_as_uint(q.y);
+        const float2 inv2 = make_float2(Bv.x, Bv.y), ns2 = make_float2(Bv.z, Bv.w);
+        uint32_t bits[4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float2 q0 = __fmul2_rn(t[h], inv2);
+          const float2 rem = __ffma2_rn(q0, ns2, t[h]);
+          const float2 q = __fadd2_rn(__ffma2_rn(rem, inv2, q0), cq_f2(CQ_MAGIC));
+          bits[2 * h] = __float_as_uint(q.x);
+          bits[2 * h + 1] = __float_as_uint(q.y);
+        }
+        // the low byte of each word is the two's complement code
+        const uint32_t four = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
         if (OUT == CQ_OUT_A8) {
-          *const_cast<uint16_t*>(reinterpret_cast<const uint16_t*>(a8c + (long)Cc.x * p.K)) =
-              static_cast<uint16_t>(__byte_perm(bx, by, 0x0040));
+          *reinterpret_cast<uint32_t*>(p.a8 + ((long)Cc.x * K + c0)) = four;
         } else if (Cc.y < 0) {
-          *const_cast<uint16_t*>(reinterpret_cast<const uint16_t*>(qhc + (long)(Cc.y & 0x7FFFFFFF) * p.K)) =
-              static_cast<uint16_t>(__byte_perm(bx, by, 0x0040));
+          *reinterpret_cast<uint32_t*>(p.q_hi + ((long)(Cc.y & 0x7FFFFFFF) * K + c0)) = four;
         } else {
-          *const_cast<uint8_t*>(qlc + (long)Cc.y * (p.K >> 1)) = static_cast<uint8_t>((bx & 0xFu) | ((by << 4) & 0xF0u));
+          const uint32_t nib = (four & 0x0F0F0F0Fu);
+          const uint32_t two = (nib | (nib >> 4)) & 0x00FF00FFu;   // bytes 0 and 2 hold two codes each
+          *reinterpret_cast<uint16_t*>(p.q_lo + ((long)Cc.y * (K >> 1) + (c0 >> 1))) =
+              static_cast<uint16_t>(__byte_perm(two, 0u, 0x4420));
         }
       }
     }
-    // the row tables and the ring stage are reused in the next iteration: its first barrier orders that
+    // the row tables and the ring stage are reused in the next iteration: its barriers order that
   }
   if (STAGED && !ok) {
     // copies issued ahead were never consumed: give them time to land before the shared memory is released
@@ -280,7 +311,7 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
     while (clock64() - t0 < 4000000LL) {
     }
   }
-  // nobody leaves while a peer may still read its maxima
+  // leave together: no CTA's shared memory goes away while a peer's posts could still be in flight
   ptx::cluster_sync();
 }
 

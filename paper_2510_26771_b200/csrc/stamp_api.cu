@@ -377,25 +377,22 @@ static int run_quant_rows(const Problem& pb, const float* T, const unsigned* row
 // ------------------------------------------------------------------------------------------
 struct CqChoice {
   int C;     // CTAs per cluster = strips along the feature axis
-  int NT;    // threads per CTA
-  int NCH;   // channel pairs per thread
+  int NT;    // threads per CTA (four channels each)
   int pmax;  // Haar levels per launch at most
 };
-// Smallest number of strips for which a CTA of at most 512 threads covers its strip with one
-// (else two) channel pairs per thread.  False when the feature axis is too long for 8 CTAs.
+// Fewest strips for which a CTA of at most 512 threads covers its strip.  False when the feature
+// axis is too long for a portable cluster of 8 CTAs (more than 16384 channels).
 static bool choose_cq(int K, CqChoice* c) {
-  for (int nch = 1; nch <= 2; ++nch)
-    for (int C = 1; C <= 8; ++C) {
-      const int pairs = (K / 2 + C - 1) / C;
-      const int nt = (((pairs + nch - 1) / nch) + 31) / 32 * 32;
-      if (nt <= 512) {
-        c->C = C;
-        c->NT = nt;
-        c->NCH = nch;
-        c->pmax = nch == 1 ? 5 : 4;
-        return true;
-      }
+  for (int C = 1; C <= 8; ++C) {
+    const int quads = (K / 4 + C - 1) / C;
+    const int nt = (quads + 31) / 32 * 32;
+    if (nt <= 512) {
+      c->C = C;
+      c->NT = nt;
+      c->pmax = 4;
+      return true;
     }
+  }
   return false;
 }
 
@@ -415,9 +412,9 @@ static PassPlan make_plan_max(int levels, int pmax) {
   return pl;
 }
 
-template <int P, int NCH, typename TIn, int OUT>
+template <int P, typename TIn, int OUT, int LODD>
 static int launch_cq_t(CqParams cp, const CqChoice& c, cudaStream_t st) {
-  auto kern = k_haar_cq<P, NCH, TIn, OUT>;
+  auto kern = k_haar_cq<P, TIn, OUT, LODD>;
   constexpr bool STAGED = sizeof(TIn) == 2;
   size_t smem = CQ_TAIL_BYTES;
   cp.nstages = 1;
@@ -476,24 +473,22 @@ static int launch_cq_t(CqParams cp, const CqChoice& c, cudaStream_t st) {
   return STAMP_OK;
 }
 
-template <int NCH, typename TIn, int OUT>
+template <typename TIn, int OUT, int LODD>
 static int launch_cq_p(int P, const CqParams& cp, const CqChoice& c, cudaStream_t st) {
   switch (P) {
-    case 0: return launch_cq_t<0, NCH, TIn, OUT>(cp, c, st);
-    case 1: return launch_cq_t<1, NCH, TIn, OUT>(cp, c, st);
-    case 2: return launch_cq_t<2, NCH, TIn, OUT>(cp, c, st);
-    case 3: return launch_cq_t<3, NCH, TIn, OUT>(cp, c, st);
-    case 4: return launch_cq_t<4, NCH, TIn, OUT>(cp, c, st);
-    default:
-      if constexpr (NCH == 1) return launch_cq_t<5, NCH, TIn, OUT>(cp, c, st);
-      return STAMP_ERR_UNSUPPORTED;
+    case 0: return launch_cq_t<0, TIn, OUT, LODD>(cp, c, st);
+    case 1: return launch_cq_t<1, TIn, OUT, LODD>(cp, c, st);
+    case 2: return launch_cq_t<2, TIn, OUT, LODD>(cp, c, st);
+    case 3: return launch_cq_t<3, TIn, OUT, LODD>(cp, c, st);
+    default: return launch_cq_t<4, TIn, OUT, LODD>(cp, c, st);
   }
 }
 template <int OUT>
 static int launch_cq_o(int P, bool bf16_in, const CqParams& cp, const CqChoice& c, cudaStream_t st) {
+  const bool lodd = (cp.lvl0 & 1) != 0;
   if (bf16_in)
-    return c.NCH == 1 ? launch_cq_p<1, __nv_bfloat16, OUT>(P, cp, c, st) : launch_cq_p<2, __nv_bfloat16, OUT>(P, cp, c, st);
-  return c.NCH == 1 ? launch_cq_p<1, float, OUT>(P, cp, c, st) : launch_cq_p<2, float, OUT>(P, cp, c, st);
+    return lodd ? launch_cq_p<__nv_bfloat16, OUT, 1>(P, cp, c, st) : launch_cq_p<__nv_bfloat16, OUT, 0>(P, cp, c, st);
+  return lodd ? launch_cq_p<float, OUT, 1>(P, cp, c, st) : launch_cq_p<float, OUT, 0>(P, cp, c, st);
 }
 
 // Haar (or identity) transform + quantizer through the cluster kernel: one launch per group of
@@ -507,7 +502,7 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
                     reinterpret_cast<float*>(base + wl.top_pong)};
   CqParams cp{};
   cp.K = pb.K;
-  cp.Kc = 2 * c.NCH * c.NT;
+  cp.Kc = 4 * c.NT;
   cp.n = pb.n;
   cp.k_hi = pb.k_hi;
   cp.qmax_hi = (float)pb.qmax_hi;
