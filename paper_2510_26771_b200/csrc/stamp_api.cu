@@ -420,7 +420,9 @@ static int launch_cq_t(CqParams cp, const CqChoice& c, cudaStream_t st) {
   cp.nstages = 1;
   if (STAGED) {
     const size_t slab = cq_slab_bytes<P, TIn>(cp.Kc);
-    size_t ns = (200 * 1024 - CQ_TAIL_BYTES) / slab;
+    // leave room for as many CTAs per SM as the register file allows (512 threads of 128 registers)
+    const size_t budget = (size_t)200 * 1024 * c.NT / 512;
+    size_t ns = (budget - CQ_TAIL_BYTES) / slab;
     ns = ns > 4 ? 4 : ns;
     if (ns < 2) return STAMP_ERR_UNSUPPORTED;
     cp.nstages = (int)ns;
