@@ -25,16 +25,23 @@
 
 namespace stamp {
 
-enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1 };
+enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1, EPI_HAAR_F32 = 2, EPI_HAAR_BF16 = 3 };
 
 struct GemmParams {
   int n_out;               // output channels (MMA M extent)
   int m_tok;               // tokens (MMA N extent)
   int k;                   // reduction length, multiple of 128
   const float* x_scale;    // [m_tok]
-  const float* w_scale;    // [n_out]
+  const float* w_scale;    // [n_out], or nullptr for 1
   void* out;               // [m_tok, n_out] float (EPI_DEQUANT_F32) or int32 (EPI_RAW_I32)
   int group;               // channel tiles per raster band
+  // EPI_HAAR_*: the token operand is in the tiled row order of the transform+quantize kernel, x_scale
+  // holds scale * 2^(-j/2) per tile row, and the epilogue applies the inverse Haar transform of the
+  // tile's 256 tokens (Algorithm line "Y <- L^-1 Y"), w_scale and the bias before storing Y.
+  int depth;               // Haar levels closed inside a tile, 5..8
+  const float* a8v;        // [m_tok / 256, n_out] level-8 approximation of every tile when the transform
+                           // has more than 8 levels (orthonormal scaling), else nullptr
+  const float* bias;       // [n_out] or nullptr
 };
 
 constexpr int GEMM_BM = 128;           // output channels per tile
@@ -213,8 +220,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       float* sxs = sx_stage + a * BN;
       float sw = 0.f;
       float my_sx[BN / 128];
-      if (EPI == EPI_DEQUANT_F32) {
-        if (ch_ok) sw = __ldg(p.w_scale + ch);
+      if (EPI != EPI_RAW_I32) {
+        if (ch_ok) sw = p.w_scale ? __ldg(p.w_scale + ch) : 1.0f;
         // fetch this tile's token scales while the accumulator is still being filled
 #pragma unroll
         for (int i = 0; i < BN / 128; ++i) {
@@ -228,7 +235,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
         break;
       }
       ptx::tc_fence_after();
-      if (EPI == EPI_DEQUANT_F32) {
+      if (EPI != EPI_RAW_I32) {
         // every epilogue thread has finished the previous tile that used accumulator `a` (all 128
         // arrived on tempty[a] before tfull[a] could complete again), so its staging buffer is free
 #pragma unroll
@@ -236,6 +243,80 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
         asm volatile("bar.sync 1, 128;" ::: "memory");
       }
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(a * BN);
+      if constexpr (EPI == EPI_HAAR_F32 || EPI == EPI_HAAR_BF16) {
+        static_assert(EPI < EPI_HAAR_F32 || BN == 256, "the fused inverse works on 256-token tiles");
+        // ---- the tile's eight coarse values (column 32 q), synthesised down to the level-5 sums
+        float hd[8];
+        {
+          uint32_t h[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) ptx::tmem_ld_32x32b_x1(taddr + 32 * q, h[q]);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 8; ++q) hd[q] = static_cast<float>(static_cast<int>(h[q])) * sxs[32 * q];
+        }
+        float bch = 0.f;
+        if (ch_ok) {
+          if (p.a8v) hd[0] = __ldg(p.a8v + (long)tok_t * p.n_out + ch) * 0.0625f;   // 2^(-8/2)
+          if (p.bias) bch = __ldg(p.bias + ch);
+        }
+        float a5[8];
+        {
+          float c2[4];
+          if (p.depth == 8) {
+            const float u0 = hd[0] + hd[1], u1 = hd[0] - hd[1];
+            c2[0] = u0 + hd[2]; c2[1] = u0 - hd[2]; c2[2] = u1 + hd[3]; c2[3] = u1 - hd[3];
+          } else if (p.depth == 7) {
+            c2[0] = hd[0] + hd[2]; c2[1] = hd[0] - hd[2]; c2[2] = hd[1] + hd[3]; c2[3] = hd[1] - hd[3];
+          } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) c2[i] = hd[i];
+          }
+          if (p.depth >= 6) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              a5[2 * i] = c2[i] + hd[4 + i];
+              a5[2 * i + 1] = c2[i] - hd[4 + i];
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a5[i] = hd[i];
+          }
+        }
+        // ---- eight chunks of 32 tokens: slot 0 <- level-5 sum, 31 details, five synthesis levels
+        uint32_t r[2][32];
+        ptx::tmem_ld_32x32b_x32(taddr, r[0]);
+#pragma unroll
+        for (int chunk = 0; chunk < 8; ++chunk) {
+          ptx::tmem_ld_wait();
+          if (chunk + 1 < 8) ptx::tmem_ld_32x32b_x32(taddr + (chunk + 1) * 32, r[(chunk + 1) & 1]);
+          const uint32_t(&rc)[32] = r[chunk & 1];
+          float y[32];
+          y[0] = a5[chunk];
+#pragma unroll
+          for (int len = 1; len < 32; len <<= 1) {
+#pragma unroll
+            for (int i = len - 1; i >= 0; --i) {
+              const float d = static_cast<float>(static_cast<int>(rc[len + i])) * sxs[chunk * 32 + len + i];
+              const float t = y[i];
+              y[2 * i] = t + d;
+              y[2 * i + 1] = t - d;
+            }
+          }
+          if (ch_ok) {
+            const long o = (long)(tok0 + chunk * 32) * p.n_out + ch;
+            if constexpr (EPI == EPI_HAAR_F32) {
+              float* out = static_cast<float*>(p.out) + o;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) out[(long)j * p.n_out] = fmaf(y[j], sw, bch);
+            } else {
+              __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out) + o;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) out[(long)j * p.n_out] = __float2bfloat16_rn(fmaf(y[j], sw, bch));
+            }
+          }
+        }
+      } else {
       uint32_t r[2][32];
       ptx::tmem_ld_32x32b_x32(taddr, r[0]);
 #pragma unroll
@@ -262,6 +343,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
           for (int j = 0; j < 32; ++j)
             if (tbase + j < p.m_tok && ch_ok) out[(long)j * p.n_out] = static_cast<int>(rc[j]);
         }
+      }
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&tempty[a]);

@@ -49,6 +49,10 @@ struct CqParams {
   uint8_t* q_lo;
   float* x_scale;   // [M]
   float* T_out;     // [M, K] transformed values (debug export)      -- CQ_OUT_T
+  // CQ_OUT_TILED: a8 rows in the order the GEMM's fused inverse epilogue consumes them
+  int8_t* a8_top;   // [M / 256, K] codes of the rows of levels > 8 (logical order inside a block), or nullptr
+  float* sx_top;    // [M / 256]    their scales
+  float* sx_epi;    // [M]          scale * 2^(-j/2) of every tile row, indexed like a8
 };
 
 constexpr float CQ_MAGIC = 12582912.0f;            // 1.5 * 2^23
@@ -58,7 +62,23 @@ constexpr float CQ_RSQRT2_LO = 1.2101617101e-8f;             // 1/sqrt 2 - fp32(
 
 // What a launch writes besides the scales: the GEMM's int8 operand, the public packed codes, or
 // the fp32 transformed values (debug export).
-enum CqOut { CQ_OUT_A8 = 0, CQ_OUT_PUBLIC = 1, CQ_OUT_T = 2 };
+enum CqOut { CQ_OUT_A8 = 0, CQ_OUT_PUBLIC = 1, CQ_OUT_T = 2, CQ_OUT_TILED = 3 };
+
+// Row order of the tiled operand (CQ_OUT_TILED).  The GEMM's token tile t covers the 256 original
+// tokens [256 t, 256 t + 256) and must own every coefficient their reconstruction needs from
+// levels 1..D, D = min(levels, 8) >= 5 (rows of levels > 8 go to a small separate table).  Inside a tile, column 32 c + r (r = 1..31) holds the r-th value,
+// in [d_5 | d_4 (2) | d_3 (4) | d_2 (8) | d_1 (16)] order, of the 32-token chunk c; column 32 q holds
+// the q-th of the tile's eight coarse values in band order [a_D | d_D | ... | d_6].  An epilogue
+// thread thus finds, per chunk, the 31 details in the order its in-register synthesis wants them,
+// with the chunk's level-5 sum (rebuilt from the eight coarse values) in slot 0.
+// Returns the column inside the tile; `i` is the coefficient's index inside its 256-token tile.
+__device__ __forceinline__ int cq_tile_col_detail(int j, int i_loc) {
+  if (j <= 5) {
+    const int sh = 5 - j;
+    return 32 * (i_loc >> sh) + (1 << sh) + (i_loc & ((1 << sh) - 1));
+  }
+  return 32 * ((256 >> j) + i_loc);
+}
 
 __device__ __forceinline__ float2 cq_f2(float a) { return make_float2(a, a); }
 
@@ -250,9 +270,29 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
       const long row = sq * p.n + i_in_blk;
       const long pub = hi ? sq * p.k_hi + i_in_blk : sq * (p.n - p.k_hi) + (i_in_blk - p.k_hi);
       tabB[r] = make_float4(inv, inv, -scale, -scale);
-      tabC[r] = make_int4(static_cast<int>(row), static_cast<int>(pub) | (hi ? static_cast<int>(0x80000000u) : 0),
-                          __float_as_int(pw), 0);
-      if (rank == 0 && ok) p.x_scale[row] = (amax > 0.f) ? scale * pw : 1.0f;
+      const float true_scale = (amax > 0.f) ? scale * pw : 1.0f;
+      if (OUT == CQ_OUT_TILED) {
+        // where the row lives in the tiled operand (or in the small table of rows above the tiles)
+        const bool top = j > 8;
+        long prow;
+        if (top) {
+          prow = sq * (p.n >> 8) + i_in_blk;     // the first n / 256 logical rows of a block are exactly those
+          if (rank == 0 && ok) p.sx_top[prow] = true_scale;
+        } else {
+          const int idx = (r == 0) ? g : (g << k) + (r - (1 << k));   // index inside the block at level j
+          const long tile = (sq * p.n + ((long)idx << j)) >> 8;
+          const int i_loc = idx & ((256 >> j) - 1);
+          const int col = (r == 0) ? 32 * i_loc : cq_tile_col_detail(j, i_loc);
+          prow = tile * 256 + col;
+          const float nrm = (j & 1) ? pw * CQ_RSQRT2_HI : pw;        // 2^(-j/2)
+          if (rank == 0 && ok) p.sx_epi[prow] = true_scale * nrm;
+        }
+        tabC[r] = make_int4(static_cast<int>(prow), 0, __float_as_int(pw), top ? 1 : 0);
+      } else {
+        tabC[r] = make_int4(static_cast<int>(row), static_cast<int>(pub) | (hi ? static_cast<int>(0x80000000u) : 0),
+                            __float_as_int(pw), 0);
+        if (rank == 0 && ok) p.x_scale[row] = true_scale;
+      }
     }
     __syncthreads();
 
@@ -291,7 +331,9 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
         }
         // the low byte of each word is the two's complement code
         const uint32_t four = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
-        if (OUT == CQ_OUT_A8) {
+        if (OUT == CQ_OUT_TILED) {
+          *reinterpret_cast<uint32_t*>((Cc.w ? p.a8_top : p.a8) + ((long)Cc.x * K + c0)) = four;
+        } else if (OUT == CQ_OUT_A8) {
           *reinterpret_cast<uint32_t*>(p.a8 + ((long)Cc.x * K + c0)) = four;
         } else if (Cc.y < 0) {
           *reinterpret_cast<uint32_t*>(p.q_hi + ((long)(Cc.y & 0x7FFFFFFF) * K + c0)) = four;

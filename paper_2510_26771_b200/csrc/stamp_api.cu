@@ -100,7 +100,7 @@ static PassPlan make_plan(int levels) {
 // Workspace layout (one layout for all calls of a problem size).
 // ------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, total;
+  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, total;
 };
 static Workspace layout(const Problem& pb) {
   Workspace w{};
@@ -124,6 +124,11 @@ static Workspace layout(const Problem& pb) {
   w.a8 = off;     off += align256(M * (size_t)pb.K);
   w.w8 = off;     off += align256((size_t)pb.N * pb.K);
   w.yt = off;     off += align256(M * (size_t)pb.N * 4);
+  // rows above the GEMM's 256-token tiles (Haar levels > 8): codes, scales, their GEMM output, its inverse
+  w.a8top = off;  off += align256((M >> 8) * (size_t)pb.K);
+  w.sxtop = off;  off += align256((M >> 8) * 4 + 4);
+  w.yttop = off;  off += align256((M >> 8) * (size_t)pb.N * 4);
+  w.a8v = off;    off += align256((M >> 8) * (size_t)pb.N * 4);
   w.total = off;
   return w;
 }
@@ -204,7 +209,8 @@ static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const Gem
 
 // acc/out[tok, ch] from int8 operands a8 [M, K], w8 [N, K].
 static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K, const float* x_scale,
-                       const float* w_scale, void* out, int epi, cudaStream_t st) {
+                       const float* w_scale, void* out, int epi, cudaStream_t st, const float* bias = nullptr,
+                       const float* a8v = nullptr, int depth = 0) {
   GemmParams gp{};
   gp.n_out = N;
   gp.m_tok = (int)M;
@@ -213,12 +219,20 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
   gp.w_scale = w_scale;
   gp.out = out;
   gp.group = 16;
+  gp.bias = bias;
+  gp.a8v = a8v;
+  gp.depth = depth;
   CUtensorMap tw, tx;
   int rc = make_tmap_i8(w8, N, K, GEMM_BM, &tw);
   if (rc) return rc;
   const bool wide = M >= 256;
   rc = make_tmap_i8(a8, M, K, wide ? 256 : 128, &tx);
   if (rc) return rc;
+  if (epi == EPI_HAAR_F32 || epi == EPI_HAAR_BF16) {
+    if (!wide || M % 256 != 0 || depth < 5 || depth > 8) return STAMP_ERR_UNSUPPORTED;
+    if (epi == EPI_HAAR_F32) return launch_gemm_t<256, 4, EPI_HAAR_F32>(tw, tx, gp, st);
+    return launch_gemm_t<256, 4, EPI_HAAR_BF16>(tw, tx, gp, st);
+  }
   if (wide) {
     if (epi == EPI_DEQUANT_F32) return launch_gemm_t<256, 4, EPI_DEQUANT_F32>(tw, tx, gp, st);
     return launch_gemm_t<256, 4, EPI_RAW_I32>(tw, tx, gp, st);
@@ -496,9 +510,14 @@ static int launch_cq_o(int P, bool bf16_in, const CqParams& cp, const CqChoice& 
 // Haar (or identity) transform + quantizer through the cluster kernel: one launch per group of
 // levels, each launch quantizing its own detail rows and handing fp32 sums to the next one.
 // Exactly one kind of output besides the scales: a8, or (q_hi, q_lo), or T_out.
+struct CqTiled {
+  int8_t* a8_top;
+  float* sx_top;
+  float* sx_epi;
+};
 static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, int x_dtype, int8_t* a8, void* q_hi,
                            void* q_lo, float* x_scale, float* T_out, uint8_t* base, const Workspace& wl,
-                           cudaStream_t st) {
+                           cudaStream_t st, const CqTiled* tiled = nullptr) {
   const PassPlan pl = make_plan_max(pb.levels, c.pmax);
   float* bufs[3] = {reinterpret_cast<float*>(base + wl.atop), reinterpret_cast<float*>(base + wl.top_ping),
                     reinterpret_cast<float*>(base + wl.top_pong)};
@@ -514,6 +533,11 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
   cp.q_lo = static_cast<uint8_t*>(q_lo);
   cp.x_scale = x_scale;
   cp.T_out = T_out;
+  if (tiled) {
+    cp.a8_top = tiled->a8_top;
+    cp.sx_top = tiled->sx_top;
+    cp.sx_epi = tiled->sx_epi;
+  }
   const void* in = X;
   int Lin = pb.n, lvl0 = 0;
   for (int i = 0; i < pl.npass; ++i) {
@@ -527,7 +551,8 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
     cp.lvl0 = lvl0;
     cp.ngroups = (long)pb.nseq * (Lin >> P);
     const bool bf16_in = (i == 0 && x_dtype == STAMP_BF16);
-    const int rc = a8 ? launch_cq_o<CQ_OUT_A8>(P, bf16_in, cp, c, st)
+    const int rc = tiled ? launch_cq_o<CQ_OUT_TILED>(P, bf16_in, cp, c, st)
+                   : a8  ? launch_cq_o<CQ_OUT_A8>(P, bf16_in, cp, c, st)
                       : T_out ? launch_cq_o<CQ_OUT_T>(P, bf16_in, cp, c, st)
                               : launch_cq_o<CQ_OUT_PUBLIC>(P, bf16_in, cp, c, st);
     if (rc) return rc;
@@ -728,7 +753,36 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
   float* yt = reinterpret_cast<float*>(base + wl.yt);
   CqChoice cc;
-  if (pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc)) {
+  const bool have_cq = pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc);
+  if (have_cq && pb.transform == STAMP_T_HAAR && pb.levels >= 5 && pb.n % 256 == 0) {
+    // Fused route: the transform+quantize kernel writes the token operand in tile order, the GEMM's
+    // epilogue de-quantizes and inverts the (up to) 8 levels that close inside its 256-token tile.
+    // Levels above 8 live in M / 256 extra rows: a small GEMM and the general inverse turn them into
+    // the level-8 approximation of every tile first.
+    CqTiled tl{reinterpret_cast<int8_t*>(base + wl.a8top), reinterpret_cast<float*>(base + wl.sxtop), x_scale};
+    if ((rc = run_quantize_cq(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st, &tl))) return rc;
+    const int8_t* w8f = nullptr;
+    if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8f, st))) return rc;
+    const float* a8v = nullptr;
+    if (pb.levels > 8) {
+      float* yttop = reinterpret_cast<float*>(base + wl.yttop);
+      float* a8v_w = reinterpret_cast<float*>(base + wl.a8v);
+      // (no weight scales here: they are applied once, after the synthesis, by the main GEMM's epilogue)
+      if ((rc = launch_gemm(tl.a8_top, w8f, pb.M >> 8, N, K, tl.sx_top, nullptr, yttop, EPI_DEQUANT_F32, st))) return rc;
+      Problem pt = pb;
+      pt.n = pb.n >> 8;
+      pt.L = pb.L >> 8;
+      pt.M = pb.M >> 8;
+      pt.levels = pb.levels - 8;
+      if ((rc = run_inverse_generic(pt, yttop, nullptr, a8v_w, STAMP_F32, ping, pong,
+                                    reinterpret_cast<float*>(base + wl.dctmat), st)))
+        return rc;
+      a8v = a8v_w;
+    }
+    return launch_gemm(a8, w8f, pb.M, N, K, x_scale, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR_BF16 : EPI_HAAR_F32, st,
+                       bias, a8v, pb.levels < 8 ? pb.levels : 8);
+  }
+  if (have_cq) {
     if ((rc = run_quantize_cq(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
   } else {
     if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
