@@ -117,6 +117,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  ptx::grid_dependency_wait();   // operands and scales come from the kernels launched before
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer

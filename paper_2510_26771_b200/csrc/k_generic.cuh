@@ -4,6 +4,7 @@
 // specialised kernels do not cover, and the unfused API calls.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace stamp {
 
@@ -95,6 +96,7 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
                                                        int n, int jlo, long ngroups, int N,
                                                        const float* __restrict__ bias, void* __restrict__ out_) {
   constexpr int G = 1 << P;
+  ptx::grid_dependency_wait();
   const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
   if (c >= N) return;
   const int gps = n >> (jlo + P);

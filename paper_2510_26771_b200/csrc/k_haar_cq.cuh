@@ -137,6 +137,7 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
   }
   // every CTA of the cluster has initialised its barriers before anyone posts to them
   ptx::cluster_sync();
+  ptx::grid_dependency_wait();   // the input rows may come from the previous launch
 
   // warp 0 brings one group's rows of this strip into a ring stage: lane r copies token row r
   auto issue_load = [&](long grp, int stage) {

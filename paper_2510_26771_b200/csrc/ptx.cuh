@@ -193,6 +193,12 @@ __host__ __device__ constexpr uint32_t make_i8_idesc(int m, int n) {
          | (static_cast<uint32_t>(m >> 4) << 24);
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Blocks until the grids this one depends on have completed and their writes are visible.  A no-op
+// for a launch without the programmatic-serialization attribute.  Everything before it (barrier
+// set-up, TMEM allocation) may overlap the tail of the previous kernel.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- clusters
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;

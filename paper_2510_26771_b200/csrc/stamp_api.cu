@@ -171,6 +171,23 @@ static int make_tmap_i8(const void* base, long rows, int K, int box_rows, CUtens
   return r == CUDA_SUCCESS ? STAMP_OK : STAMP_ERR_CUDA;
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while the previous
+// kernel of the stream drains; it calls grid_dependency_wait() before touching that kernel's output.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kern, KArgs(args)...);
+}
+
 static int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -201,7 +218,7 @@ static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const Gem
   const int grid = tiles < sm_count() ? tiles : sm_count();
   const bool timed = t_gemm_ev_start && t_gemm_ev_stop;
   if (timed) cudaEventRecord(t_gemm_ev_start, st);
-  kern<<<grid, GEMM_THREADS, SM::DYN_BYTES, st>>>(tw, tx, gp);
+  launch_pdl(kern, dim3((unsigned)grid), dim3(GEMM_THREADS), SM::DYN_BYTES, st, tw, tx, gp);
   if (timed) cudaEventRecord(t_gemm_ev_stop, st);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
@@ -319,12 +336,12 @@ static int launch_inv_pass(int P, const float* Yt, const float* ain, int n, int 
                            const float* bias, void* out, cudaStream_t st) {
   dim3 grid((N / 2 + 127) / 128, (unsigned)(ngroups < 32768 ? ngroups : 32768));
   switch (P) {
-    case 0: k_haar_inv_pass<0, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 1: k_haar_inv_pass<1, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 2: k_haar_inv_pass<2, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 3: k_haar_inv_pass<3, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 4: k_haar_inv_pass<4, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    default: k_haar_inv_pass<5, TOut><<<grid, 128, 0, st>>>(Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 0: launch_pdl(k_haar_inv_pass<0, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 1: launch_pdl(k_haar_inv_pass<1, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 2: launch_pdl(k_haar_inv_pass<2, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 3: launch_pdl(k_haar_inv_pass<3, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 4: launch_pdl(k_haar_inv_pass<4, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    default: launch_pdl(k_haar_inv_pass<5, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
   }
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
@@ -452,13 +469,15 @@ static int launch_cq_t(CqParams cp, const CqChoice& c, cudaStream_t st) {
   lc.blockDim = dim3((unsigned)c.NT);
   lc.dynamicSmemBytes = smem;
   lc.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)c.C;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
   // persistent clusters: as many as can be resident at once (cached per launch shape)
   static std::mutex mu;
   static std::unordered_map<unsigned long long, int> resident;
