@@ -25,7 +25,7 @@
 
 namespace stamp {
 
-enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1, EPI_HAAR_F32 = 2, EPI_HAAR_BF16 = 3 };
+enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1, EPI_HAAR_F32 = 2, EPI_HAAR_BF16 = 3, EPI_DEQUANT_BF16X2 = 4 };
 
 struct GemmParams {
   int n_out;               // output channels (MMA M extent)
@@ -33,7 +33,8 @@ struct GemmParams {
   int k;                   // reduction length, multiple of 128
   const float* x_scale;    // [m_tok]
   const float* w_scale;    // [n_out], or nullptr for 1
-  void* out;               // [m_tok, n_out] float (EPI_DEQUANT_F32) or int32 (EPI_RAW_I32)
+  void* out;               // [m_tok, n_out] float (EPI_DEQUANT_F32) or int32 (EPI_RAW_I32); EPI_DEQUANT_BF16X2:
+                           // two bf16 planes [2][m_tok, n_out], value = hi + lo (operand of the DCT inverse)
   int group;               // channel tiles per raster band
   // EPI_HAAR_*: the token operand is in the tiled row order of the transform+quantize kernel, x_scale
   // holds scale * 2^(-j/2) per tile row, and the epilogue applies the inverse Haar transform of the
@@ -338,6 +339,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
               if (tbase + j < p.m_tok && ch_ok)
                 out[(long)j * p.n_out] = static_cast<float>(static_cast<int>(rc[j])) * sxs[chunk * 32 + j] * sw;
           }
+        } else if (EPI == EPI_DEQUANT_BF16X2) {
+          __nv_bfloat16* hi = static_cast<__nv_bfloat16*>(p.out) + (long)tbase * p.n_out + ch;
+          __nv_bfloat16* lo = hi + (long)p.m_tok * p.n_out;
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (tbase + j < p.m_tok && ch_ok) {
+              const float v = static_cast<float>(static_cast<int>(rc[j])) * sxs[chunk * 32 + j] * sw;
+              const __nv_bfloat16 h = __float2bfloat16_rn(v);
+              hi[(long)j * p.n_out] = h;
+              lo[(long)j * p.n_out] = __float2bfloat16_rn(v - __bfloat162float(h));
+            }
         } else {
           int* out = static_cast<int*>(p.out) + (long)tbase * p.n_out + ch;
 #pragma unroll

@@ -225,6 +225,25 @@ __global__ void __launch_bounds__(256) k_unpack_codes(const int8_t* __restrict__
   }
 }
 
+// One int8 per code, logical token order -> the public code format (inverse of k_unpack_codes).
+__global__ void __launch_bounds__(256) k_pack_codes(const int8_t* __restrict__ codes, int K, int n, int k_hi,
+                                                    int8_t* __restrict__ q_hi, uint8_t* __restrict__ q_lo) {
+  const long r = blockIdx.x;
+  const long s = r / n;
+  const int i = static_cast<int>(r - s * n);
+  const char4* src = reinterpret_cast<const char4*>(codes + r * (long)K);
+  if (i < k_hi) {
+    char4* dst = reinterpret_cast<char4*>(q_hi + (s * k_hi + i) * (long)K);
+    for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) dst[k4] = src[k4];
+  } else {
+    uint16_t* dst = reinterpret_cast<uint16_t*>(q_lo + (s * (n - k_hi) + (i - k_hi)) * (long)(K / 2));
+    for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) {
+      const char4 c = src[k4];
+      dst[k4] = static_cast<uint16_t>((c.x & 0xF) | ((c.y & 0xF) << 4) | ((c.z & 0xF) << 8) | ((c.w & 0xF) << 12));
+    }
+  }
+}
+
 // Packed 4-bit rows -> int8 rows (weights). One CTA per row.
 __global__ void __launch_bounds__(256) k_unpack_rows4(const uint8_t* __restrict__ packed, int K, int8_t* __restrict__ out) {
   const long r = blockIdx.x;

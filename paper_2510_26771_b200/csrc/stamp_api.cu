@@ -8,6 +8,7 @@
 
 #include "common.cuh"
 #include "k_dct.cuh"
+#include "k_dct_tc.cuh"
 #include "k_gemm.cuh"
 #include "k_generic.cuh"
 #include "k_haar_cq.cuh"
@@ -100,7 +101,7 @@ static PassPlan make_plan(int levels) {
 // Workspace layout (one layout for all calls of a problem size).
 // ------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, total;
+  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, dctsplit, total;
 };
 static Workspace layout(const Problem& pb) {
   Workspace w{};
@@ -129,6 +130,8 @@ static Workspace layout(const Problem& pb) {
   w.sxtop = off;  off += align256((M >> 8) * 4 + 4);
   w.yttop = off;  off += align256((M >> 8) * (size_t)pb.N * 4);
   w.a8v = off;    off += align256((M >> 8) * (size_t)pb.N * 4);
+  // bf16 terms of the DCT matrix and of its transpose (tensor-core DCT)
+  w.dctsplit = off; off += align256(pb.transform == STAMP_T_DCT2 ? (size_t)2 * 3 * DCT_N * DCT_N * 2 : 0);
   w.total = off;
   return w;
 }
@@ -171,6 +174,21 @@ static int make_tmap_i8(const void* base, long rows, int K, int box_rows, CUtens
   return r == CUDA_SUCCESS ? STAMP_OK : STAMP_ERR_CUDA;
 }
 
+// bf16 matrix [rows, cols] row-major; box = 64 columns (128 bytes) x 256 rows, 128-byte swizzle.
+static int make_tmap_bf16(const void* base, long rows, long cols, CUtensorMap* out) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return STAMP_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) != 0) return STAMP_ERR_INVALID_ARG;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64u, 256u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? STAMP_OK : STAMP_ERR_CUDA;
+}
+
 // Launch with programmatic stream serialization: the kernel may be scheduled while the previous
 // kernel of the stream drains; it calls grid_dependency_wait() before touching that kernel's output.
 template <typename... KArgs, typename... Args>
@@ -202,6 +220,27 @@ static int sm_count() {
 // ------------------------------------------------------------------------------------------
 // Launchers
 // ------------------------------------------------------------------------------------------
+template <int MODE, int NATOM, int NPLANE>
+static int launch_dct_tc(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const DctTcParams& dp,
+                         cudaStream_t st) {
+  using SM = DctSmem<NATOM, NPLANE>;
+  auto kern = k_dct_tc<MODE, NATOM, NPLANE>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::DYN_BYTES) != cudaSuccess)
+      return STAMP_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles = dp.nblk * (dp.cols / (NATOM * 64));
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  if (launch_pdl(kern, dim3((unsigned)grid), dim3(DCT_THREADS), SM::DYN_BYTES, st, ta, tb0, tb1, dp) != cudaSuccess) {
+    cudaGetLastError();
+    return STAMP_ERR_CUDA;
+  }
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
 template <int BN, int STAGES, int EPI>
 static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const GemmParams& gp, cudaStream_t st) {
   using SM = GemmSmem<BN, STAGES>;
@@ -250,6 +289,9 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
     if (epi == EPI_HAAR_F32) return launch_gemm_t<256, 4, EPI_HAAR_F32>(tw, tx, gp, st);
     return launch_gemm_t<256, 4, EPI_HAAR_BF16>(tw, tx, gp, st);
   }
+  if (epi == EPI_DEQUANT_BF16X2)
+    return wide ? launch_gemm_t<256, 4, EPI_DEQUANT_BF16X2>(tw, tx, gp, st)
+                : launch_gemm_t<128, 6, EPI_DEQUANT_BF16X2>(tw, tx, gp, st);
   if (wide) {
     if (epi == EPI_DEQUANT_F32) return launch_gemm_t<256, 4, EPI_DEQUANT_F32>(tw, tx, gp, st);
     return launch_gemm_t<256, 4, EPI_RAW_I32>(tw, tx, gp, st);
@@ -582,6 +624,58 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
   return STAMP_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// Blockwise 256-point DCT-II on the tensor cores (bf16 activations).
+// ------------------------------------------------------------------------------------------
+static bool dct_tc_ok(const Problem& pb, int x_dtype) {
+  return pb.transform == STAMP_T_DCT2 && pb.n == DCT_N && x_dtype == STAMP_BF16;
+}
+
+// Transform + quantizer: row maxima in a first launch, codes (a8, logical order) and scales in a second.
+static int run_quantize_dct_tc(const Problem& pb, const void* X, int8_t* a8, float* x_scale, uint8_t* base,
+                               const Workspace& wl, cudaStream_t st) {
+  __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(base + wl.dctsplit);
+  unsigned* rowmax = reinterpret_cast<unsigned*>(base + wl.rowmax);
+  k_dct_split_matrix<<<DCT_N * DCT_N / 256, 256, 0, st>>>(0, split);
+  STAMP_CHECK_LAUNCH();
+  if (cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+  CUtensorMap ta, tb;
+  int rc = make_tmap_bf16(split, 3 * DCT_N, DCT_N, &ta);
+  if (rc) return rc;
+  if ((rc = make_tmap_bf16(X, pb.M, pb.K, &tb))) return rc;
+  DctTcParams dp{};
+  dp.nblk = pb.nseq;
+  dp.cols = pb.K;
+  dp.k_hi = pb.k_hi;
+  dp.qmax_hi = (float)pb.qmax_hi;
+  dp.qmax_lo = (float)pb.qmax_lo;
+  dp.rowmax = rowmax;
+  dp.a8 = a8;
+  dp.x_scale = x_scale;
+  if ((rc = launch_dct_tc<DCT_TC_MAX, 2, 1>(ta, tb, tb, dp, st))) return rc;
+  return launch_dct_tc<DCT_TC_QUANT, 2, 1>(ta, tb, tb, dp, st);
+}
+
+// Y = C^T (hi + lo) + bias from the two bf16 planes the GEMM's epilogue wrote.  N % 64 == 0.
+static int run_inverse_dct_tc(const Problem& pb, const __nv_bfloat16* planes, const float* bias, void* Y, int y_dtype,
+                              uint8_t* base, const Workspace& wl, cudaStream_t st) {
+  __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(base + wl.dctsplit) + 3 * DCT_N * DCT_N;
+  k_dct_split_matrix<<<DCT_N * DCT_N / 256, 256, 0, st>>>(1, split);
+  STAMP_CHECK_LAUNCH();
+  CUtensorMap ta, tb0, tb1;
+  int rc = make_tmap_bf16(split, 3 * DCT_N, DCT_N, &ta);
+  if (rc) return rc;
+  if ((rc = make_tmap_bf16(planes, pb.M, pb.N, &tb0))) return rc;
+  if ((rc = make_tmap_bf16(planes + (size_t)pb.M * pb.N, pb.M, pb.N, &tb1))) return rc;
+  DctTcParams dp{};
+  dp.nblk = pb.nseq;
+  dp.cols = pb.N;
+  dp.y = Y;
+  dp.y_bf16 = (y_dtype == STAMP_BF16);
+  dp.bias = bias;
+  return launch_dct_tc<DCT_TC_INVERSE, 1, 2>(ta, tb0, tb1, dp, st);
+}
+
 static int run_unpack_codes(const Problem& pb, const void* q_hi, const void* q_lo, int8_t* out, cudaStream_t st) {
   k_unpack_codes<<<(unsigned)pb.M, 256, 0, st>>>(static_cast<const int8_t*>(q_hi), static_cast<const uint8_t*>(q_lo),
                                                   pb.K, pb.n, pb.k_hi, out);
@@ -690,6 +784,14 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   CqChoice cc;
   if (pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc))
     return run_quantize_cq(pb, cc, X, x_dtype, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
+  if (dct_tc_ok(pb, x_dtype)) {
+    int8_t* a8 = reinterpret_cast<int8_t*>(base + w.a8);
+    if ((rc = run_quantize_dct_tc(pb, X, a8, x_scale, base, w, st))) return rc;
+    k_pack_codes<<<(unsigned)pb.M, 256, 0, st>>>(a8, pb.K, pb.n, pb.k_hi, static_cast<int8_t*>(q_hi),
+                                                  static_cast<uint8_t*>(q_lo));
+    STAMP_CHECK_LAUNCH();
+    return STAMP_OK;
+  }
   rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
                              reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st);
   if (rc) return rc;
@@ -800,6 +902,17 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     }
     return launch_gemm(a8, w8f, pb.M, N, K, x_scale, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR_BF16 : EPI_HAAR_F32, st,
                        bias, a8v, pb.levels < 8 ? pb.levels : 8);
+  }
+  if (dct_tc_ok(pb, x_dtype)) {
+    if ((rc = run_quantize_dct_tc(pb, X, a8, x_scale, base, wl, st))) return rc;
+    const int8_t* w8d = nullptr;
+    if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8d, st))) return rc;
+    if (N % 64 == 0) {   // the GEMM writes its output as two bf16 planes, the operand of the tensor-core inverse
+      if ((rc = launch_gemm(a8, w8d, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_BF16X2, st))) return rc;
+      return run_inverse_dct_tc(pb, reinterpret_cast<const __nv_bfloat16*>(yt), bias, Y, y_dtype, base, wl, st);
+    }
+    if ((rc = launch_gemm(a8, w8d, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_F32, st))) return rc;
+    return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
   }
   if (have_cq) {
     if ((rc = run_quantize_cq(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;

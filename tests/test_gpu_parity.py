@@ -61,6 +61,8 @@ CASES = {
     "wide_k8192": gen.scaled(gen.config_sweep(512, 8192), L=128, K=8192, N=64, levels=5, k_hi=4),
     # blockwise DCT-II: several blocks per sequence, ragged output-channel tile; a short block
     "dct_blocks": gen.scaled(gen.config_llm_down(), B=2, L=512, K=384, N=136),
+    # output width a multiple of 64: the layer's inverse DCT also runs on the tensor cores
+    "dct_tensor_inverse": gen.scaled(gen.config_llm_down(), B=1, L=768, K=256, N=192),
     "dct_short_block": gen.scaled(gen.config_llm_down(), B=1, L=256, K=128, N=64, block=32, k_hi=4),
     # two levels only: no cluster tree, approximation rows quantized by the same kernel
     "two_levels": gen.scaled(gen.config_dit_proj(), B=2, L=256, K=1152, N=128, grid=16, levels=2, k_hi=64),
