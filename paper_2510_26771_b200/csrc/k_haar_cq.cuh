@@ -50,7 +50,7 @@ struct CqParams {
   float* x_scale;   // [M]
   float* T_out;     // [M, K] transformed values (debug export)      -- CQ_OUT_T
   // CQ_OUT_TILED: a8 rows in the order the GEMM's fused inverse epilogue consumes them
-  int8_t* a8_top;   // [M / 256, K] codes of the rows of levels > 8 (logical order inside a block), or nullptr
+  long a8_top_row;  // codes of the rows of levels > 8 (logical order inside a block) go to rows a8_top_row + i of a8
   float* sx_top;    // [M / 256]    their scales
   float* sx_epi;    // [M]          scale * 2^(-j/2) of every tile row, indexed like a8
 };
@@ -81,6 +81,17 @@ __device__ __forceinline__ int cq_tile_col_detail(int j, int i_loc) {
 }
 
 __device__ __forceinline__ float2 cq_f2(float a) { return make_float2(a, a); }
+
+// The butterflies run in place: a pair (x[2i], x[2i+1]) of stride-s neighbours becomes (sum, difference)
+// where it stands, and the next level pairs the sums (stride 2s).  The coefficient that the output
+// order [a | d_P | d_(P-1) (2) | ... | d_1 (G/2)] calls row r therefore sits in register:
+__host__ __device__ constexpr int cq_reg_of_row(int P, int r) {
+  if (r == 0) return 0;
+  int k = 0;
+  while ((2 << k) <= r) ++k;          // r in [2^k, 2^(k+1)): detail of local level l = P - k
+  const int l = P - k, i = r - (1 << k);
+  return (2 * i + 1) << (l - 1);
+}
 
 // Shared memory: [ring: nstages x G x Kc x sizeof(TIn)] [full barriers: 8 x u64] [mailbox barriers: 2 x u64]
 //   [maxima: 2 x 16 u32] [mailbox: 2 x 8 CTAs x 16 u32]
@@ -190,8 +201,9 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
 #pragma unroll
         for (int r = 0; r < G; ++r) {
           const uint2 w = *reinterpret_cast<const uint2*>(s8 + r * row_bytes);
-          v[0][r] = make_float2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
-          v[1][r] = make_float2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+          // bf16 -> fp32 by byte permutation (keeps the shifts off the FMA pipe)
+          v[0][r] = make_float2(__uint_as_float(__byte_perm(w.x, 0u, 0x1044)), __uint_as_float(__byte_perm(w.x, 0u, 0x3244)));
+          v[1][r] = make_float2(__uint_as_float(__byte_perm(w.y, 0u, 0x1044)), __uint_as_float(__byte_perm(w.y, 0u, 0x3244)));
         }
       } else {
         const float* src = static_cast<const float*>(p.in) + ((sq * p.Lin + (long)g * G) * (long)K + cbase + 4 * qe);
@@ -209,28 +221,44 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
 #pragma unroll
-      for (int len = G; len > 1; len >>= 1) {
-        float2 t[G];
+      for (int st = 1; st < G; st <<= 1) {
 #pragma unroll
-        for (int i = 0; i < len / 2; ++i) {
-          t[i] = __fadd2_rn(v[h][2 * i], v[h][2 * i + 1]);
-          t[len / 2 + i] = __ffma2_rn(v[h][2 * i + 1], cq_f2(-1.0f), v[h][2 * i]);
+        for (int i = 0; i < G; i += 2 * st) {
+          const float2 a = v[h][i], b2 = v[h][i + st];
+          v[h][i] = __fadd2_rn(a, b2);
+          v[h][i + st] = __ffma2_rn(b2, cq_f2(-1.0f), a);
         }
-#pragma unroll
-        for (int i = 0; i < len; ++i) v[h][i] = t[i];
       }
     }
-    // v[h] is now [a | d_P | d_(P-1) (2) | ... | d_1 (G/2)]
+    // row r of [a | d_P | d_(P-1) (2) | ... | d_1 (G/2)] is now v[h][cq_reg_of_row(P, r)]
 
-    // ---- per-row maxima of this strip: lane r of every warp collects row r, one atomic per lane
-    unsigned keep = 0u;
+    // ---- per-row maxima of this strip.  G values per lane are reduced over the warp by a transposing
+    // butterfly: at each stage half of the rows go to the partner lane (xor of one lane bit), so the
+    // work halves every stage; lane L ends up with the warp-wide maximum of row (L >> 1) & (G - 1).
+    {
+      float m[G];
 #pragma unroll
-    for (int r = 0; r < G; ++r) {
-      const float m = fmaxf(fmaxf(fabsf(v[0][r].x), fabsf(v[0][r].y)), fmaxf(fabsf(v[1][r].x), fabsf(v[1][r].y)));
-      const unsigned mm = __reduce_max_sync(0xffffffffu, __float_as_uint(m));
-      keep = (lane == r) ? mm : keep;
+      for (int r = 0; r < G; ++r) {
+        const int ri = cq_reg_of_row(P, r);
+        m[r] = fmaxf(fmaxf(fabsf(v[0][ri].x), fabsf(v[0][ri].y)), fmaxf(fabsf(v[1][ri].x), fabsf(v[1][ri].y)));
+      }
+#pragma unroll
+      for (int n = G; n >= 2; n >>= 1) {
+        const bool upper = (lane & n) != 0;
+#pragma unroll
+        for (int r = 0; r < n / 2; ++r) {
+          const float send = upper ? m[r] : m[r + n / 2];
+          const float keepv = upper ? m[r + n / 2] : m[r];
+          m[r] = fmaxf(keepv, __shfl_xor_sync(0xffffffffu, send, n));
+        }
+      }
+      // the lane bits no stage used: bit 0 and the bits above log2 G
+      m[0] = fmaxf(m[0], __shfl_xor_sync(0xffffffffu, m[0], 1));
+#pragma unroll
+      for (int bit = 2 * G; bit < 32; bit <<= 1)
+        if (bit >= 2) m[0] = fmaxf(m[0], __shfl_xor_sync(0xffffffffu, m[0], bit));
+      if (lane < 2 * G && (lane & 1) == 0) atomicMax(&mymax[b * 16 + (lane >> 1)], __float_as_uint(m[0]));
     }
-    if (lane < G) atomicMax(&mymax[b * 16 + lane], keep);
     __syncthreads();
     if (tid < G) {
       // post this strip's maxima to every CTA of the cluster (this one included) and clear them
@@ -277,8 +305,9 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
         const bool top = j > 8;
         long prow;
         if (top) {
-          prow = sq * (p.n >> 8) + i_in_blk;     // the first n / 256 logical rows of a block are exactly those
-          if (rank == 0 && ok) p.sx_top[prow] = true_scale;
+          const long trow = sq * (p.n >> 8) + i_in_blk;   // the first n / 256 logical rows of a block are exactly those
+          if (rank == 0 && ok) p.sx_top[trow] = true_scale;
+          prow = p.a8_top_row + trow;
         } else {
           const int idx = (r == 0) ? g : (g << k) + (r - (1 << k));   // index inside the block at level j
           const long tile = (sq * p.n + ((long)idx << j)) >> 8;
@@ -299,6 +328,7 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
 
     // ---- normalise, quantize and store from registers
     if (valid && ok) {
+      int8_t* const a8c = p.a8 + c0;
 #pragma unroll
       for (int r = 0; r < G; ++r) {
         if (r == 0 && !last) continue;
@@ -308,11 +338,12 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
         for (int s = 1; s < 5; ++s) lg += (r >> s) ? 1 : 0;
         const int l = (r == 0) ? P : P - lg;
         const bool odd = ((LODD + l) & 1) != 0;
+        const int ri = cq_reg_of_row(P, r);
         const int4 Cc = tabC[r];
         float2 t[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h)
-          t[h] = odd ? __ffma2_rn(v[h][r], cq_f2(CQ_RSQRT2_HI), __fmul2_rn(v[h][r], cq_f2(CQ_RSQRT2_LO))) : v[h][r];
+          t[h] = odd ? __ffma2_rn(v[h][ri], cq_f2(CQ_RSQRT2_HI), __fmul2_rn(v[h][ri], cq_f2(CQ_RSQRT2_LO))) : v[h][ri];
         if (OUT == CQ_OUT_T) {
           const float pw = __int_as_float(Cc.z);
           *reinterpret_cast<float4*>(p.T_out + ((long)Cc.x * K + c0)) =
@@ -333,9 +364,9 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
         // the low byte of each word is the two's complement code
         const uint32_t four = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
         if (OUT == CQ_OUT_TILED) {
-          *reinterpret_cast<uint32_t*>((Cc.w ? p.a8_top : p.a8) + ((long)Cc.x * K + c0)) = four;
+          *reinterpret_cast<uint32_t*>(a8c + (long)Cc.x * K) = four;
         } else if (OUT == CQ_OUT_A8) {
-          *reinterpret_cast<uint32_t*>(p.a8 + ((long)Cc.x * K + c0)) = four;
+          *reinterpret_cast<uint32_t*>(a8c + (long)Cc.x * K) = four;
         } else if (Cc.y < 0) {
           *reinterpret_cast<uint32_t*>(p.q_hi + ((long)(Cc.y & 0x7FFFFFFF) * K + c0)) = four;
         } else {

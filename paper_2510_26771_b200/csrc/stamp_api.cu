@@ -122,11 +122,13 @@ static Workspace layout(const Problem& pb) {
   w.top_ping = off; off += align256((M >> 6) * (size_t)pb.K * 4);
   w.top_pong = off; off += align256((M >> 9) * (size_t)pb.K * 4);
   w.dctmat = off; off += align256(pb.transform == STAMP_T_DCT2 ? (size_t)pb.n * pb.n * 4 : 0);
-  w.a8 = off;     off += align256(M * (size_t)pb.K);
+  // the top table follows the M rows of a8 directly: the tiled route addresses it as rows M, M + 1, ...
+  w.a8 = off;     off += M * (size_t)pb.K;
+  w.a8top = off;  off += align256((M >> 8) * (size_t)pb.K) + 256;
+  off = align256(off);
   w.w8 = off;     off += align256((size_t)pb.N * pb.K);
   w.yt = off;     off += align256(M * (size_t)pb.N * 4);
   // rows above the GEMM's 256-token tiles (Haar levels > 8): codes, scales, their GEMM output, its inverse
-  w.a8top = off;  off += align256((M >> 8) * (size_t)pb.K);
   w.sxtop = off;  off += align256((M >> 8) * 4 + 4);
   w.yttop = off;  off += align256((M >> 8) * (size_t)pb.N * 4);
   w.a8v = off;    off += align256((M >> 8) * (size_t)pb.N * 4);
@@ -572,7 +574,7 @@ static int launch_cq_o(int P, bool bf16_in, const CqParams& cp, const CqChoice& 
 // levels, each launch quantizing its own detail rows and handing fp32 sums to the next one.
 // Exactly one kind of output besides the scales: a8, or (q_hi, q_lo), or T_out.
 struct CqTiled {
-  int8_t* a8_top;
+  int8_t* a8_top;   // must be a8 + M * K
   float* sx_top;
   float* sx_epi;
 };
@@ -595,7 +597,7 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
   cp.x_scale = x_scale;
   cp.T_out = T_out;
   if (tiled) {
-    cp.a8_top = tiled->a8_top;
+    cp.a8_top_row = pb.M;
     cp.sx_top = tiled->sx_top;
     cp.sx_epi = tiled->sx_epi;
   }
