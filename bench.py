@@ -110,6 +110,23 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks_ms(local_ms: float, device="cpu") -> float:
+    """Timed-region duration of the whole job: the slowest rank's (all-reduce MAX; identity for one rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(local_ms)
+    t = torch.tensor([float(local_ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(ops_per_replica_step: float, world: int, ms_per_step: float) -> float:
+    """Replicas only: every rank runs the same step on its own GPU, so the job did world x the work
+    in the time of the slowest rank."""
+    return world * ops_per_replica_step / (ms_per_step * 1e-3) / 1e12
+
+
 def cpu_oracle_sample(cfg, seconds_target=15.0):
     """Time the CPU oracle, as it stands, on a bounded sample of the workload: all tokens and
     features, a subset of output channels chosen so that the run takes roughly seconds_target."""
@@ -270,10 +287,7 @@ def main():
     if world > 1:
         dist.barrier()
     total_ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks_ms(total_ms, device="cuda")
     ms_per_step = total_ms / steps
     gemm_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(g0, g1)) if args.stage == "fused" or not args.quick else 0.0
     status = st.stamp_last_device_status()
@@ -292,7 +306,7 @@ def main():
         clocks = sampler.stop()
 
     ops = 2.0 * M * N * K
-    value = world * ops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tops(ops, world, ms_per_step)
 
     if rank != 0:
         if world > 1:
