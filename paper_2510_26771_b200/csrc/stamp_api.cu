@@ -12,6 +12,7 @@
 #include "k_gemm.cuh"
 #include "k_generic.cuh"
 #include "k_haar_cq.cuh"
+#include "k_top_gemv.cuh"
 #include "stamp.h"
 
 namespace stamp {
@@ -678,6 +679,42 @@ static int run_inverse_dct_tc(const Problem& pb, const __nv_bfloat16* planes, co
   return launch_dct_tc<DCT_TC_INVERSE, 1, 2>(ta, tb0, tb1, dp, st);
 }
 
+// Top rows of a short sequence: codes x weights, de-quantization and the inverse of the levels above 8
+// in one launch (k_top_gemv).  Returns STAMP_ERR_UNSUPPORTED when the shape is outside its range.
+template <int R>
+static int launch_top_gemv(const int8_t* codes, const float* sx, const int8_t* w8, int K, int N, int top_levels,
+                           float* a8v, cudaStream_t st) {
+  auto kern = k_top_gemv<R>;
+  const size_t smem = (size_t)R * K;
+  static size_t attr_smem = 0;
+  if (smem > attr_smem) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return STAMP_ERR_CUDA;
+    attr_smem = smem;
+  }
+  const int per_cta = (TOPG_THREADS / 32) * TOPG_CH_PER_WARP;
+  if (launch_pdl(kern, dim3((unsigned)((N + per_cta - 1) / per_cta)), dim3(TOPG_THREADS), smem, st, codes, sx, w8, K, N,
+                 top_levels, a8v) != cudaSuccess) {
+    cudaGetLastError();
+    return STAMP_ERR_CUDA;
+  }
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+static int run_top_gemv(const Problem& pb, const int8_t* codes, const float* sx, const int8_t* w8, float* a8v,
+                        cudaStream_t st) {
+  const long R = pb.M >> 8;
+  if (R > 16 || (size_t)R * pb.K > 160 * 1024 || pb.K % 16 != 0) return STAMP_ERR_UNSUPPORTED;
+  const int tl = pb.levels - 8;
+  switch (R) {
+    case 2: return launch_top_gemv<2>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    case 4: return launch_top_gemv<4>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    case 8: return launch_top_gemv<8>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    case 16: return launch_top_gemv<16>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    default: return STAMP_ERR_UNSUPPORTED;
+  }
+}
+
 static int run_unpack_codes(const Problem& pb, const void* q_hi, const void* q_lo, int8_t* out, cudaStream_t st) {
   k_unpack_codes<<<(unsigned)pb.M, 256, 0, st>>>(static_cast<const int8_t*>(q_hi), static_cast<const uint8_t*>(q_lo),
                                                   pb.K, pb.n, pb.k_hi, out);
@@ -890,6 +927,12 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     if (pb.levels > 8) {
       float* yttop = reinterpret_cast<float*>(base + wl.yttop);
       float* a8v_w = reinterpret_cast<float*>(base + wl.a8v);
+      rc = run_top_gemv(pb, tl.a8_top, tl.sx_top, w8f, a8v_w, st);
+      if (rc == STAMP_OK) {
+        a8v = a8v_w;
+      } else if (rc != STAMP_ERR_UNSUPPORTED) {
+        return rc;
+      } else {
       // (no weight scales here: they are applied once, after the synthesis, by the main GEMM's epilogue)
       if ((rc = launch_gemm(tl.a8_top, w8f, pb.M >> 8, N, K, tl.sx_top, nullptr, yttop, EPI_DEQUANT_F32, st))) return rc;
       Problem pt = pb;
@@ -901,6 +944,7 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
                                     reinterpret_cast<float*>(base + wl.dctmat), st)))
         return rc;
       a8v = a8v_w;
+      }
     }
     return launch_gemm(a8, w8f, pb.M, N, K, x_scale, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR_BF16 : EPI_HAAR_F32, st,
                        bias, a8v, pb.levels < 8 ? pb.levels : 8);
