@@ -72,12 +72,12 @@ __device__ __forceinline__ void mma_bf16_ss(uint32_t tmem_d, uint64_t adesc, uin
 }
 
 // Shared-memory descriptor of an MN-major operand tile stored as rows (= K index) of 128 bytes
-// (64 bf16 along MN) with the 128-byte swizzle, 8-row groups 1024 bytes apart.  One tile is one
-// 64-element atom along MN, so the MN-direction stride field is not exercised.
+// (64 bf16 along MN) with the 128-byte swizzle, 8-row groups 1024 bytes apart; a wider operand is
+// several such [256 x 64] atoms, DCT_ATOM_BYTES apart (the descriptor's MN-direction stride).
 __device__ __forceinline__ uint64_t make_mnmajor_sw128_desc(uint32_t smem_addr_bytes) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((smem_addr_bytes >> 4) & 0x3FFFu);
-  d |= static_cast<uint64_t>(DCT_ATOM_BYTES >> 4) << 16;  // stride between 64-wide atoms along MN (unused)
+  d |= static_cast<uint64_t>(DCT_ATOM_BYTES >> 4) << 16;  // stride between 64-wide atoms along MN
   d |= static_cast<uint64_t>(1024 >> 4) << 32;            // stride between 8-row groups along K
   d |= static_cast<uint64_t>(1) << 46;
   d |= static_cast<uint64_t>(2) << 61;                    // SWIZZLE_128B
@@ -198,7 +198,8 @@ __global__ void __launch_bounds__(DCT_THREADS, 1)
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (ptx::elect_one()) {
-      constexpr uint32_t idesc = make_bf16_idesc_bmn(128, 64);
+      // one MMA spans all NATOM 64-channel atoms of the tile (the descriptor's MN stride = one atom)
+      constexpr uint32_t idesc = make_bf16_idesc_bmn(128, 64 * NATOM);
       int st = 0;
       uint32_t aphase = 0;
       int it = 0;
@@ -223,12 +224,8 @@ __global__ void __launch_bounds__(DCT_THREADS, 1)
 #pragma unroll
               for (int h = 0; h < 2; ++h) {
                 const uint64_t adesc = ptx::make_kmajor_sw128_desc(abase + h * (128 * 128) + k * 32);
-#pragma unroll
-                for (int a = 0; a < NATOM; ++a) {
-                  const uint64_t bdesc = make_mnmajor_sw128_desc(bbase + (plane * NATOM + a) * DCT_ATOM_BYTES +
-                                                                 (tb * 64 + k * 16) * 128);
-                  mma_bf16_ss(dbase + h * (NATOM * 64) + a * 64, adesc, bdesc, idesc, (term | tb | k) != 0 ? 1u : 0u);
-                }
+                const uint64_t bdesc = make_mnmajor_sw128_desc(bbase + plane * NATOM * DCT_ATOM_BYTES + (tb * 64 + k * 16) * 128);
+                mma_bf16_ss(dbase + h * (NATOM * 64), adesc, bdesc, idesc, (term | tb | k) != 0 ? 1u : 0u);
               }
             ptx::tc_commit(&aempty[st]);
             if (++st == DCT_A_STAGES) { st = 0; aphase ^= 1u; }
