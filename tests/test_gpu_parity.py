@@ -64,6 +64,10 @@ CASES = {
     # output width a multiple of 64: the layer's inverse DCT also runs on the tensor cores
     "dct_tensor_inverse": gen.scaled(gen.config_llm_down(), B=1, L=768, K=256, N=192),
     "dct_short_block": gen.scaled(gen.config_llm_down(), B=1, L=256, K=128, N=64, block=32, k_hi=4),
+    # fused inverse epilogue with 5 and 7 levels closed inside a 256-token tile (8 and 6 are covered above)
+    "tile_depth5": gen.scaled(gen.config_dit_proj(), B=2, L=512, K=256, N=200, grid=0, block=256, levels=5, k_hi=8,
+                              recipe="ar1"),
+    "tile_depth7": gen.scaled(gen.config_llm_up(), B=1, L=1024, K=384, N=128, levels=7, k_hi=8),
     # two levels only: no cluster tree, approximation rows quantized by the same kernel
     "two_levels": gen.scaled(gen.config_dit_proj(), B=2, L=256, K=1152, N=128, grid=16, levels=2, k_hi=64),
 }
@@ -154,6 +158,27 @@ def test_transform_then_inverse_is_identity(st):
     e_t = float((T.double() ** 2).sum())
     e_x = float((X.astype(np.float64) ** 2).sum())
     assert abs(e_t - e_x) <= 1e-6 * e_x
+
+
+def test_host_buffer_call_matches_device_call(st):
+    """stamp_linear_fused_host = the same layer with the two copies enqueued around it."""
+    import torch
+    cfg = gen.scaled(gen.config_llm_up(), B=1, L=512, K=256, N=264)
+    c = _cfg_struct(st, cfg)
+    X, W, bias = gen.make_activation(cfg), gen.make_weight(cfg), gen.make_bias(cfg)
+    Xd, Wd, bd = H.to_device(X, cfg.dtype), H.to_device(W, cfg.dtype), torch.from_numpy(bias).cuda()
+    wq, wsc = st.stamp_quantize_weights(c, Wd)
+    w8 = st.stamp_prepare_weights(c, wq)
+    ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+    want = st.stamp_linear_fused(c, Xd, w8, st.W_INT8, wsc, bd, ws, out_dtype=torch.bfloat16)
+    X_host = Xd.cpu().pin_memory()
+    Y_host = torch.empty((cfg.B, cfg.L, cfg.N), dtype=torch.bfloat16).pin_memory()
+    ws_h = torch.empty(st.stamp_workspace_bytes_host(c, cfg.B, cfg.L, cfg.K, cfg.N, st.BF16, st.BF16), dtype=torch.uint8,
+                       device="cuda")
+    st.stamp_linear_fused_host(c, X_host, w8, st.W_INT8, wsc, bd, Y_host, ws_h)
+    torch.cuda.synchronize()
+    assert torch.equal(Y_host, want.cpu())
+    assert st.stamp_last_device_status() == 0
 
 
 def test_edge_cases(st, oracle):
