@@ -328,7 +328,11 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
 
     // ---- normalise, quantize and store from registers
     if (valid && ok) {
+      // per-thread bases; a row's address is base + row * pitch
       int8_t* const a8c = p.a8 + c0;
+      int8_t* const qhc = p.q_hi + c0;
+      uint8_t* const qlc = p.q_lo + (c0 >> 1);
+      uint8_t* const Tc = reinterpret_cast<uint8_t*>(p.T_out + c0);
 #pragma unroll
       for (int r = 0; r < G; ++r) {
         if (r == 0 && !last) continue;
@@ -346,7 +350,7 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
           t[h] = odd ? __ffma2_rn(v[h][ri], cq_f2(CQ_RSQRT2_HI), __fmul2_rn(v[h][ri], cq_f2(CQ_RSQRT2_LO))) : v[h][ri];
         if (OUT == CQ_OUT_T) {
           const float pw = __int_as_float(Cc.z);
-          *reinterpret_cast<float4*>(p.T_out + ((long)Cc.x * K + c0)) =
+          *reinterpret_cast<float4*>(ptx::ptr_mad_wide(Tc, Cc.x, 4 * K)) =
               make_float4(t[0].x * pw, t[0].y * pw, t[1].x * pw, t[1].y * pw);
           continue;
         }
@@ -364,15 +368,15 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
         // the low byte of each word is the two's complement code
         const uint32_t four = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
         if (OUT == CQ_OUT_TILED) {
-          *reinterpret_cast<uint32_t*>(a8c + (long)Cc.x * K) = four;
+          *reinterpret_cast<uint32_t*>(ptx::ptr_mad_wide(a8c, Cc.x, K)) = four;
         } else if (OUT == CQ_OUT_A8) {
-          *reinterpret_cast<uint32_t*>(a8c + (long)Cc.x * K) = four;
+          *reinterpret_cast<uint32_t*>(ptx::ptr_mad_wide(a8c, Cc.x, K)) = four;
         } else if (Cc.y < 0) {
-          *reinterpret_cast<uint32_t*>(p.q_hi + ((long)(Cc.y & 0x7FFFFFFF) * K + c0)) = four;
+          *reinterpret_cast<uint32_t*>(ptx::ptr_mad_wide(qhc, Cc.y & 0x7FFFFFFF, K)) = four;
         } else {
           const uint32_t nib = (four & 0x0F0F0F0Fu);
           const uint32_t two = (nib | (nib >> 4)) & 0x00FF00FFu;   // bytes 0 and 2 hold two codes each
-          *reinterpret_cast<uint16_t*>(p.q_lo + ((long)Cc.y * (K >> 1) + (c0 >> 1))) =
+          *reinterpret_cast<uint16_t*>(ptx::ptr_mad_wide(qlc, Cc.y, K >> 1)) =
               static_cast<uint16_t>(__byte_perm(two, 0u, 0x4420));
         }
       }

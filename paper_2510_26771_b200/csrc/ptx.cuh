@@ -13,6 +13,15 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// base + a * b bytes with a 32 x 32 -> 64-bit multiply-add (one instruction; the C++ expression
+// base + (long)a * b is compiled as a full 64-bit multiplication)
+template <typename T>
+__device__ __forceinline__ T* ptr_mad_wide(T* base, int a, int b) {
+  uint64_t r;
+  asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"(reinterpret_cast<uint64_t>(base)));
+  return reinterpret_cast<T*>(r);
+}
+
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(
