@@ -109,6 +109,9 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
     const long s = grp / gps;
     const int g = static_cast<int>(grp - s * gps);
     const float* Yseq = Yt + (s * n) * (long)N + c;
+    // In-place synthesis with compile-time register indices: the running value of the token range
+    // [i, i + 2^l) sits in v[i]; adding / subtracting the level-l detail splits it into the two halves
+    // v[i] and v[i + 2^(l-1)], so after level 1 the registers are in natural token order.
     float v0[G], v1[G];
     if (ain) {
       const float2 a = load2(ain + ((s * gps + g) * (long)N + c));
@@ -122,19 +125,19 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
     }
 #pragma unroll
     for (int l = P; l >= 1; --l) {
-      const int cur = 1 << (P - l);
+      const int span = 1 << l;               // tokens covered by one level-l coefficient
       const int j = jlo + l;
       const HaarNorm nrm = haar_norm(j);
-      const int row0 = (n >> j) + g * cur;
+      const int row0 = (n >> j) + g * (G >> l);
 #pragma unroll
-      for (int i = cur - 1; i >= 0; --i) {
-        const float2 d = load2(Yseq + (long)(row0 + i) * N);
+      for (int i = 0; i < G; i += span) {
+        const float2 d = load2(Yseq + (long)(row0 + i / span) * N);
         const float d0 = mul_norm(d.x, nrm), d1 = mul_norm(d.y, nrm);
         const float p0 = v0[i], p1 = v1[i];
-        v0[2 * i] = p0 + d0;
-        v0[2 * i + 1] = p0 - d0;
-        v1[2 * i] = p1 + d1;
-        v1[2 * i + 1] = p1 - d1;
+        v0[i] = p0 + d0;
+        v0[i + span / 2] = p0 - d0;
+        v1[i] = p1 + d1;
+        v1[i + span / 2] = p1 - d1;
       }
     }
     if (jlo == 0) {
