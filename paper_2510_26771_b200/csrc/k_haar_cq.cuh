@@ -129,7 +129,8 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
   const int cbase = static_cast<int>(rank) * p.Kc;
   const int cvalid = max(0, min(p.Kc, K - cbase));   // channels of this strip (0: the strip is empty)
   const uint32_t row_bytes = static_cast<uint32_t>(cvalid) * sizeof(TIn);
-  const int gps = p.Lin >> P;                         // groups per transform block
+  const int gps = p.Lin >> P;                         // groups per transform block: a power of two
+  const int gps_shift = 31 - __clz(gps);              // (64-bit divisions in the loop would cost more than a row)
   const bool last = (p.aout == nullptr);
   const int NS = p.nstages;
   const bool valid = 4 * tid < cvalid;                // this thread's four channels exist
@@ -153,8 +154,8 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
   // warp 0 brings one group's rows of this strip into a ring stage: lane r copies token row r
   auto issue_load = [&](long grp, int stage) {
     if (!STAGED || cvalid == 0 || tid >= 32) return;
-    const long sq = grp / gps;
-    const long g = grp - sq * gps;
+    const long sq = grp >> gps_shift;
+    const long g = grp & (gps - 1);
     const uint8_t* src = static_cast<const uint8_t*>(p.in) + (((sq * p.Lin + g * G) * (long)K + cbase) * (long)sizeof(TIn));
     uint8_t* dst = cq_smem + stage * slab;
     if (lane == 0) ptx::mbar_arrive_expect_tx(&full[stage], row_bytes * G);
@@ -169,14 +170,15 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
     }
 
   bool ok = true;
-  long it = 0;
+  int it = 0;
+  int stage = 0;           // ring stage of this group and the parity of its barrier phase, kept
+  uint32_t ring_phase = 0; // incrementally: a division per iteration costs more than a row's arithmetic
   for (long grp = cid; grp < p.ngroups; grp += ncl, ++it) {
-    const int stage = static_cast<int>(it % NS);
     const int b = static_cast<int>(it & 1);
     if (STAGED && ok) {
       // the stage read in the previous iteration is free: every thread passed a barrier since
       const long nxt = grp + (long)(NS - 1) * ncl;
-      if (nxt < p.ngroups) issue_load(nxt, static_cast<int>((it + NS - 1) % NS));
+      if (nxt < p.ngroups) issue_load(nxt, stage == 0 ? NS - 1 : stage - 1);
     }
     // this group's mailbox buffer expects G maxima from each CTA of the cluster (its previous use,
     // two groups ago, was completed and read before this thread passed that group's barrier)
@@ -184,14 +186,14 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
     if (STAGED && cvalid > 0 && ok) {
       // every thread waits for the copies itself (that also makes the data visible to it); a
       // thread that gives up tells the others through the abort word their waits poll
-      if (!ptx::mbar_wait_bounded(&full[stage], static_cast<uint32_t>((it / NS) & 1), &abort_word, CQ_WAIT_LIMIT)) {
+      if (!ptx::mbar_wait_bounded(&full[stage], ring_phase, &abort_word, CQ_WAIT_LIMIT)) {
         ok = false;
         abort_word = 1;
         raise_device_status(STAMP_ERR_TIMEOUT);
       }
     }
-    const long sq = grp / gps;
-    const int g = static_cast<int>(grp - sq * gps);
+    const long sq = grp >> gps_shift;
+    const int g = static_cast<int>(grp & (gps - 1));
 
     // ---- load G tokens x 4 channels, butterflies in registers (un-normalised)
     float2 v[2][G];
@@ -269,7 +271,7 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
       for (unsigned q = 0; q < csize; ++q) ptx::st_async_u32(ptx::mapa(slot, q), mine, ptx::mapa(bar, q));
     }
     if (!last && valid && ok)
-      *reinterpret_cast<float4*>(p.aout + ((sq * gps + g) * (long)K + c0)) =
+      *reinterpret_cast<float4*>(p.aout + (grp * (long)K + c0)) =
           make_float4(v[0][0].x, v[0][0].y, v[1][0].x, v[1][0].y);
 
     // ---- row tables: maxima over the cluster, scales, output rows
@@ -382,6 +384,10 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
       }
     }
     // the row tables and the ring stage are reused in the next iteration: its barriers order that
+    if (++stage == NS) {
+      stage = 0;
+      ring_phase ^= 1u;
+    }
   }
   if (STAGED && !ok) {
     // copies issued ahead were never consumed: give them time to land before the shared memory is released
