@@ -231,18 +231,22 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
           my_sx[i] = (tok < p.m_tok) ? __ldg(p.x_scale + tok) : 0.f;
         }
       }
-      // the TMEM loads below are warp-collective: the whole warp continues or the whole warp stops
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&tfull[a], acc_phase, abort_word, GEMM_WAIT_LIMIT))) {
-        ok = false;
-        break;
-      }
+      // The four epilogue warps continue or stop TOGETHER: a warp whose wait ran out raises the abort
+      // word, and everybody reads it behind the named barrier below -- no warp is left waiting at that
+      // barrier for one that already gave up.  (The TMEM loads are warp-collective as well.)
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&tfull[a], acc_phase, abort_word, GEMM_WAIT_LIMIT)))
+        *abort_word = 1;
       ptx::tc_fence_after();
       if (EPI != EPI_RAW_I32) {
         // every epilogue thread has finished the previous tile that used accumulator `a` (all 128
         // arrived on tempty[a] before tfull[a] could complete again), so its staging buffer is free
 #pragma unroll
         for (int i = 0; i < BN / 128; ++i) sxs[i * 128 + ep_tid] = my_sx[i];
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (*abort_word != 0u) {
+        ok = false;
+        break;
       }
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(a * BN);
       if constexpr (EPI == EPI_HAAR_F32 || EPI == EPI_HAAR_BF16) {
