@@ -38,7 +38,7 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_T_IDENTITY = 0, ORACLE_T_HAAR = 1, ORACLE_T_DCT2 = 2 };
+enum { ORACLE_T_IDENTITY = 0, ORACLE_T_HAAR = 1, ORACLE_T_DCT2 = 2, ORACLE_T_HAAR2D = 3 };
 
 int oracle_num_threads(void) {
 #ifdef _OPENMP
@@ -138,6 +138,61 @@ int oracle_transform_matrix(int transform, int n, int levels, double* Lmat) {
     return 0;
   }
   return 2;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * 2-D Haar DWT over a patch grid (Sec. "Efficient Energy Concentration": for image tokens the
+ * wavelet transform is taken over the two spatial axes, "one quarter" of the tokens staying
+ * low-pass per level; Set-up of the LVM experiments: 3 levels on a 64 x 64 grid leave 64 low-pass
+ * tokens).  The n tokens of a block are a grid of h = n / w rows by w columns in raster order.
+ * One level maps every 2 x 2 cell (a b / c d) to
+ *     LL = (a + b + c + d) / 2   LH = (a - b + c - d) / 2   (difference along a row)
+ *     HL = (a + b - c - d) / 2   HH = (a - b - c + d) / 2   (difference across rows / both)
+ * and recurses on the LL grid.  Output order after l levels:
+ *     [LL_l | LH_l | HL_l | HH_l | LH_(l-1) | HL_(l-1) | HH_(l-1) | ... | LH_1 | HL_1 | HH_1],
+ * each band in raster order of its (h >> level) x (w >> level) grid.  Band order and signs are a
+ * convention of this implementation (the paper fixes neither).
+ * ------------------------------------------------------------------------------------------ */
+static void haar2d_forward(double* v, int h, int w, int levels, double* tmp) {
+  int n = h * w;
+  /* grid[] holds the current LL grid in raster order at the front of v */
+  int ch = h, cw = w;
+  for (int l = 1; l <= levels; ++l) {
+    int nh = ch / 2, nw = cw / 2, q = nh * nw;
+    for (int y = 0; y < nh; ++y)
+      for (int x = 0; x < nw; ++x) {
+        double a = v[(2 * y) * cw + 2 * x], b = v[(2 * y) * cw + 2 * x + 1];
+        double c = v[(2 * y + 1) * cw + 2 * x], d = v[(2 * y + 1) * cw + 2 * x + 1];
+        int i = y * nw + x;
+        tmp[i] = (a + b + c + d) * 0.5;
+        tmp[q + i] = (a - b + c - d) * 0.5;
+        tmp[2 * q + i] = (a + b - c - d) * 0.5;
+        tmp[3 * q + i] = (a - b - c + d) * 0.5;
+      }
+    memcpy(v, tmp, sizeof(double) * (size_t)(4 * q));
+    ch = nh;
+    cw = nw;
+  }
+  (void)n;
+}
+
+/* Dense matrix of the 2-D Haar transform of a block of n tokens laid out as (n / grid_w) x grid_w. */
+int oracle_transform_matrix2d(int n, int grid_w, int levels, double* Lmat) {
+  if (n <= 0 || grid_w <= 0 || n % grid_w) return 1;
+  int h = n / grid_w;
+  if (levels <= 0 || (h >> levels) << levels != h || (grid_w >> levels) << levels != grid_w) return 2;
+  double* v = (double*)malloc(sizeof(double) * (size_t)n);
+  double* tmp = (double*)malloc(sizeof(double) * (size_t)n);
+  if (!v || !tmp) { free(v); free(tmp); return 3; }
+  for (int t = 0; t < n; ++t) {
+    memset(v, 0, sizeof(double) * (size_t)n);
+    v[t] = 1.0;
+    haar2d_forward(v, h, grid_w, levels, tmp);
+    for (int i = 0; i < n; ++i) Lmat[(size_t)i * n + t] = v[i];
+  }
+  free(v);
+  free(tmp);
+  return 0;
 }
 
 /* The same Haar matrix in CSR form for block lengths whose dense matrix would not fit in
@@ -429,7 +484,7 @@ int oracle_matmul_f64(const float* X, const float* W, long M, int N, int K, doub
 int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B, int L, int K, int N,
                         int transform, int block, int levels, int k_hi, int bits_hi, int bits_lo,
                         int bits_w, double* T, float* x_scale, int8_t* q, float* w_scale, int8_t* wq,
-                        int32_t* acc, double* Yt, double* Y) {
+                        int32_t* acc, double* Yt, double* Y, int grid_w) {
   int n = block ? block : L;
   if (n <= 0 || L % n) return 1;
   long M = (long)B * L;
@@ -463,7 +518,8 @@ int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B
   } else {
     Lmat = (double*)malloc(sizeof(double) * (size_t)n * n);
     if (!Lmat) { rc = 3; goto done; }
-    rc = oracle_transform_matrix(transform, n, levels, Lmat);
+    rc = (transform == ORACLE_T_HAAR2D) ? oracle_transform_matrix2d(n, grid_w, levels, Lmat)
+                                        : oracle_transform_matrix(transform, n, levels, Lmat);
   }
   if (rc) goto done;
 

@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "stamp_oracle.c")
 _LIB = os.path.join(_HERE, "libstamp_oracle.so")
 _lib = None
 
-T_IDENTITY, T_HAAR, T_DCT2 = 0, 1, 2
+T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -50,9 +50,12 @@ def _check(rc: int, what: str) -> None:
         raise RuntimeError(f"oracle {what} failed with code {rc}")
 
 
-def transform_matrix(transform: int, n: int, levels: int = 0) -> np.ndarray:
-    """Dense n x n fp64 matrix of the sequence transform."""
+def transform_matrix(transform: int, n: int, levels: int = 0, grid_w: int = 0) -> np.ndarray:
+    """Dense n x n fp64 matrix of the sequence transform (grid_w: patch-grid width of the 2-D Haar)."""
     out = np.empty((n, n), dtype=np.float64)
+    if transform == T_HAAR2D:
+        _check(lib().oracle_transform_matrix2d(int(n), int(grid_w), int(levels), _p(out)), "transform_matrix2d")
+        return out
     _check(lib().oracle_transform_matrix(int(transform), int(n), int(levels), _p(out)), "transform_matrix")
     return out
 
@@ -156,7 +159,7 @@ def matmul_f64(X: np.ndarray, W: np.ndarray) -> np.ndarray:
 
 def stamp_linear(X: np.ndarray, W: np.ndarray, bias: Optional[np.ndarray] = None, *, transform: int,
                  block: int = 0, levels: int = 0, k_hi: int = 64, bits_hi: int = 8, bits_lo: int = 4,
-                 bits_w: int = 4, want=("T", "x_scale", "q", "w_scale", "wq", "acc", "Yt", "Y")) -> Dict[str, np.ndarray]:
+                 bits_w: int = 4, grid_w: int = 0, want=("T", "x_scale", "q", "w_scale", "wq", "acc", "Yt", "Y")) -> Dict[str, np.ndarray]:
     """Run the whole layer; returns the stages named in `want`.
 
     X [B, L, K] float32 (values already rounded to the storage dtype), W [N, K] float32."""
@@ -175,6 +178,6 @@ def stamp_linear(X: np.ndarray, W: np.ndarray, bias: Optional[np.ndarray] = None
     rc = lib().oracle_stamp_linear(_p(X), _p(W), _p(bias), B, L, K, N, int(transform), int(block), int(levels),
                                    int(k_hi), int(bits_hi), int(bits_lo), int(bits_w), _p(g("T")),
                                    _p(g("x_scale")), _p(g("q")), _p(g("w_scale")), _p(g("wq")), _p(g("acc")),
-                                   _p(g("Yt")), _p(g("Y")))
+                                   _p(g("Yt")), _p(g("Y")), int(grid_w))
     _check(rc, "stamp_linear")
     return out

@@ -392,3 +392,70 @@ def test_energy_concentrates_and_stamp_beats_uniform_4bit(oracle):
     assert e[:cfg.k_hi].mean() > 10 * e[cfg.k_hi:].mean()
     uniform = oracle.stamp_linear(X, W, None, transform=T_ID, k_hi=0, want=("Y",))
     assert _sqnr(ref, stamp["Y"]) > _sqnr(ref, uniform["Y"])
+
+
+# ---------------------------------------------------------------------------------------------
+# 2-D Haar over the patch grid (Sec. "Efficient Energy Concentration"; LVM set-up: 3 levels on a
+# 64 x 64 grid leave 64 low-pass tokens)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("h,w,levels", [(8, 8, 3), (16, 8, 2), (4, 16, 1), (64, 64, 3)])
+def test_haar2d_orthonormal_and_lowpass_closed_form(oracle, h, w, levels):
+    n = h * w
+    Lm = oracle.transform_matrix(oracle.T_HAAR2D, n, levels, grid_w=w)
+    assert np.abs(Lm @ Lm.T - np.eye(n)).max() <= 1e-12
+    # LL_l[y, x] = 2^-l * (sum over the 2^l x 2^l patch): the first n / 4^l rows, raster order
+    s = 1 << levels
+    for y in range(h // s):
+        for x in range(w // s):
+            want = np.zeros((h, w))
+            want[y * s:(y + 1) * s, x * s:(x + 1) * s] = 2.0 ** -levels
+            assert np.array_equal(Lm[y * (w // s) + x], want.reshape(-1))
+    # a constant image has no detail: only the low-pass rows respond, with c * 2^l
+    t = Lm @ np.full(n, 3.0)
+    q = n >> (2 * levels)
+    assert np.allclose(t[:q], 3.0 * 2.0 ** levels, rtol=0, atol=1e-12) and np.abs(t[q:]).max() <= 1e-12
+
+
+def test_haar2d_one_level_is_the_kronecker_product_of_1d_steps(oracle):
+    """Independent construction: one 2-D level = (1-D Haar step across rows) (x) (1-D step along a row)."""
+    h, w = 4, 8
+    Hy = oracle.transform_matrix(oracle.T_HAAR, h, 1)     # rows: [averages | differences], pinned above
+    Hx = oracle.transform_matrix(oracle.T_HAAR, w, 1)
+    ay, dy, ax, dx = Hy[:h // 2], Hy[h // 2:], Hx[:w // 2], Hx[w // 2:]
+    want = np.concatenate([np.kron(ay, ax),    # LL
+                           np.kron(ay, dx),    # LH: difference along a row
+                           np.kron(dy, ax),    # HL: difference across rows
+                           np.kron(dy, dx)])   # HH
+    got = oracle.transform_matrix(oracle.T_HAAR2D, h * w, 1, grid_w=w)
+    assert np.abs(got - want).max() <= 1e-15
+
+
+def test_haar2d_levels_nest_and_pipeline_is_plain_matmul(oracle):
+    """Level l+1 only re-mixes the low-pass quarter; with the quantizers off the layer is X W^T."""
+    h = w = 8
+    n = h * w
+    L1 = oracle.transform_matrix(oracle.T_HAAR2D, n, 1, grid_w=w)
+    L2 = oracle.transform_matrix(oracle.T_HAAR2D, n, 2, grid_w=w)
+    assert np.array_equal(L1[n // 4:], L2[n // 4:])                    # level-1 detail bands untouched
+    inner = oracle.transform_matrix(oracle.T_HAAR2D, n // 4, 1, grid_w=w // 2)
+    assert np.abs(L2[:n // 4] - inner @ L1[:n // 4]).max() <= 1e-15   # the LL grid transformed once more
+    rng = np.random.default_rng(7)
+    X = rng.standard_normal((2, n, 24))
+    W = rng.standard_normal((10, 24))
+    T = oracle.apply_dense(L2, X)
+    back = oracle.apply_dense(L2, T @ W.T, transpose=True)
+    assert np.abs(back - X @ W.T).max() <= 1e-12
+    assert abs((T ** 2).sum() - (X ** 2).sum()) <= 1e-10 * (X ** 2).sum()
+
+
+def test_haar2d_layer_runs_and_marks_the_lowpass_tokens_high_precision(oracle):
+    cfg = gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=128, N=64, grid=16, levels=2, k_hi=16)
+    X, W = gen.make_activation(cfg), gen.make_weight(cfg)
+    out = oracle.stamp_linear(X, W, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi,
+                              grid_w=cfg.grid, want=("T", "q", "Y"))
+    # the 16 low-pass tokens (a 4 x 4 grid of 4 x 4 patch sums) are the 8-bit rows and carry most energy
+    assert np.abs(out["q"][:16]).max() > 7 and np.abs(out["q"][16:]).max() <= 7
+    e = (out["T"] ** 2).sum(axis=1)
+    assert e[:16].sum() > 0.9 * e.sum()
+    ref = oracle.matmul_f64(X.reshape(-1, cfg.K), W)
+    assert np.linalg.norm(out["Y"] - ref) / np.linalg.norm(ref) < 0.2
