@@ -28,6 +28,12 @@
  *       Haar, l levels: [a_l (n/2^l rows) | d_l | d_(l-1) | ... | d_1 (n/2 rows)], with
  *         a[i] = (x[2i] + x[2i+1]) / sqrt2,  d[i] = (x[2i] - x[2i+1]) / sqrt2  per level;
  *       DCT-II (orthonormal): row u = frequency u, row 0 = DC.
+ *       2-D Haar (STAMP_T_HAAR2D; Sec. "Efficient Energy Concentration", LVM set-up: 3 levels on the
+ *         64 x 64 patch grid leave 64 low-pass tokens): the block's n tokens are a raster-ordered
+ *         grid of n / grid_w rows x grid_w columns; per level every 2 x 2 cell (a b / c d) gives
+ *         LL = (a+b+c+d)/2, LH = (a-b+c-d)/2, HL = (a+b-c-d)/2, HH = (a-b-c+d)/2 and LL recurses;
+ *         order [LL_l | LH_l | HL_l | HH_l | LH_(l-1) | ... | HH_1], bands in raster order;
+ *         levels = 1..3, 2^levels divides both grid sides.
  *     The 8-bit tokens are the rows {i : i mod n < k_hi} ("the first 64 tokens are kept at
  *     8 bits", Sec. "Optimal bit allocation").
  *   - Quantizer (Sec. 2.1, first equation, symmetric form): scale = absmax / qmax,
@@ -56,7 +62,7 @@ typedef enum {
 
 typedef enum { STAMP_F32 = 0, STAMP_BF16 = 1 } stamp_dtype;
 
-typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2 } stamp_transform;
+typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2, STAMP_T_HAAR2D = 3 } stamp_transform;
 
 typedef enum { STAMP_G_PER_TOKEN = 0, STAMP_G_PER_CHANNEL = 1 } stamp_granularity;
 
@@ -79,7 +85,7 @@ typedef struct {
   int32_t bits_w;    /* 4 (weights, per output channel)                                        */
   int32_t act_gran;  /* STAMP_G_PER_TOKEN   (scales shared across features, Sec. 2.1)          */
   int32_t w_gran;    /* STAMP_G_PER_CHANNEL (one scale per output channel, Sec. "Set-up")      */
-  int32_t reserved;  /* must be 0                                                              */
+  int32_t grid_w;    /* STAMP_T_HAAR2D: width of the patch grid a block's tokens form; else 0  */
 } stamp_config;
 
 /* Bytes of scratch any call below may need for this problem size (the maximum over the calls). */

@@ -14,7 +14,7 @@ from .build import LIB_PATH
 
 STAMP_OK = 0
 F32, BF16 = 0, 1
-T_IDENTITY, T_HAAR, T_DCT2 = 0, 1, 2
+T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D = 0, 1, 2, 3
 G_PER_TOKEN, G_PER_CHANNEL = 0, 1
 W_PACKED4, W_INT8 = 0, 1
 
@@ -29,12 +29,14 @@ EXPORTS = (
 
 class StampConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("transform", "block", "levels", "k_hi", "bits_hi", "bits_lo",
-                                              "bits_w", "act_gran", "w_gran", "reserved")]
+                                              "bits_w", "act_gran", "w_gran", "grid_w")]
 
 
 def make_config(transform: int, block: int = 0, levels: int = 0, k_hi: int = 64, bits_hi: int = 8,
-                bits_lo: int = 4, bits_w: int = 4) -> StampConfig:
-    return StampConfig(transform, block, levels, k_hi, bits_hi, bits_lo, bits_w, G_PER_TOKEN, G_PER_CHANNEL, 0)
+                bits_lo: int = 4, bits_w: int = 4, grid_w: int = 0) -> StampConfig:
+    """grid_w: width of the patch grid for T_HAAR2D (0 for the other transforms)."""
+    return StampConfig(transform, block, levels, k_hi, bits_hi, bits_lo, bits_w, G_PER_TOKEN, G_PER_CHANNEL,
+                       grid_w if transform == T_HAAR2D else 0)
 
 
 class StampError(RuntimeError):

@@ -10,6 +10,7 @@
 #include "k_dct.cuh"
 #include "k_dct_tc.cuh"
 #include "k_gemm.cuh"
+#include "k_haar2d.cuh"
 #include "k_generic.cuh"
 #include "k_haar_cq.cuh"
 #include "k_top_gemv.cuh"
@@ -40,8 +41,9 @@ static inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool need_n, Problem* out) {
   if (!cfg || !out) return STAMP_ERR_INVALID_ARG;
   if (B <= 0 || L <= 0 || K <= 0 || (need_n && N <= 0)) return STAMP_ERR_INVALID_ARG;
-  if (cfg->transform < STAMP_T_IDENTITY || cfg->transform > STAMP_T_DCT2) return STAMP_ERR_INVALID_ARG;
-  if (cfg->block < 0 || cfg->levels < 0 || cfg->k_hi < 0 || cfg->reserved != 0) return STAMP_ERR_INVALID_ARG;
+  if (cfg->transform < STAMP_T_IDENTITY || cfg->transform > STAMP_T_HAAR2D) return STAMP_ERR_INVALID_ARG;
+  if (cfg->block < 0 || cfg->levels < 0 || cfg->k_hi < 0 || cfg->grid_w < 0) return STAMP_ERR_INVALID_ARG;
+  if (cfg->transform != STAMP_T_HAAR2D && cfg->grid_w != 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->bits_hi != 8 || cfg->bits_lo != 4 || cfg->bits_w != 4) return STAMP_ERR_UNSUPPORTED;
   if (cfg->act_gran != STAMP_G_PER_TOKEN || cfg->w_gran != STAMP_G_PER_CHANNEL) return STAMP_ERR_UNSUPPORTED;
   const int n = cfg->block ? cfg->block : L;
@@ -57,6 +59,13 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
     if (levels > full) return STAMP_ERR_UNSUPPORTED;
   }
   if (cfg->transform == STAMP_T_DCT2 && n > 4096) return STAMP_ERR_UNSUPPORTED;  // dense n x n matrix in scratch
+  if (cfg->transform == STAMP_T_HAAR2D) {
+    const int w = cfg->grid_w;
+    if (w <= 0 || n % w != 0) return STAMP_ERR_INVALID_ARG;
+    levels = cfg->levels;
+    if (levels < 1 || levels > 3 || (w & ((1 << levels) - 1)) != 0 || ((n / w) & ((1 << levels) - 1)) != 0)
+      return STAMP_ERR_UNSUPPORTED;
+  }
   out->B = B;
   out->L = L;
   out->K = K;
@@ -65,6 +74,7 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
   out->n = n;
   out->levels = levels;
   out->k_hi = cfg->k_hi;
+  out->grid_w = cfg->grid_w;
   out->nseq = B * (L / n);
   out->M = (long)B * L;
   out->qmax_hi = (1 << (cfg->bits_hi - 1)) - 1;
@@ -357,8 +367,36 @@ static int make_dct_matrix(int n, float* mat, cudaStream_t st) {
 }
 
 // T = L X (Haar, identity or blockwise DCT-II), fp32, logical order; optionally the per-row |T| maxima.
+template <int LV, typename TIn>
+static int launch_haar2d_fwd(const Problem& pb, const TIn* X, float* T, unsigned* rowmax, cudaStream_t st) {
+  const long npatch = pb.M >> (2 * LV);
+  dim3 grid((pb.K / 2 + 127) / 128, (unsigned)(npatch < 32768 ? npatch : 32768));
+  k_haar2d_fwd<LV, TIn><<<grid, 128, 0, st>>>(X, pb.n, pb.grid_w, npatch, pb.K, T, rowmax);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+template <int LV, typename TOut>
+static int launch_haar2d_inv(const Problem& pb, const float* Yt, const float* bias, TOut* Y, cudaStream_t st) {
+  const long npatch = pb.M >> (2 * LV);
+  dim3 grid((pb.N / 2 + 127) / 128, (unsigned)(npatch < 32768 ? npatch : 32768));
+  k_haar2d_inv<LV, TOut><<<grid, 128, 0, st>>>(Yt, pb.n, pb.grid_w, npatch, pb.N, bias, Y);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
 static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, float* T, unsigned* rowmax,
                                  float* ping, float* pong, float* mat, cudaStream_t st) {
+  if (pb.transform == STAMP_T_HAAR2D) {
+    if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+    const bool bf = x_dtype == STAMP_BF16;
+    const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(X);
+    const float* xf = static_cast<const float*>(X);
+    switch (pb.levels) {
+      case 1: return bf ? launch_haar2d_fwd<1>(pb, xb, T, rowmax, st) : launch_haar2d_fwd<1>(pb, xf, T, rowmax, st);
+      case 2: return bf ? launch_haar2d_fwd<2>(pb, xb, T, rowmax, st) : launch_haar2d_fwd<2>(pb, xf, T, rowmax, st);
+      default: return bf ? launch_haar2d_fwd<3>(pb, xb, T, rowmax, st) : launch_haar2d_fwd<3>(pb, xf, T, rowmax, st);
+    }
+  }
   if (pb.transform == STAMP_T_DCT2) {
     if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
     if (int rc = make_dct_matrix(pb.n, mat, st)) return rc;
@@ -395,6 +433,16 @@ static int launch_inv_pass(int P, const float* Yt, const float* ain, int n, int 
 // Y = L^T Yt + bias (Haar or identity), coarse passes first.
 static int run_inverse_generic(const Problem& pb, const float* Yt, const float* bias, void* Y, int y_dtype,
                                float* ping, float* pong, float* mat, cudaStream_t st) {
+  if (pb.transform == STAMP_T_HAAR2D) {
+    const bool bf = y_dtype == STAMP_BF16;
+    __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(Y);
+    float* yf = static_cast<float*>(Y);
+    switch (pb.levels) {
+      case 1: return bf ? launch_haar2d_inv<1>(pb, Yt, bias, yb, st) : launch_haar2d_inv<1>(pb, Yt, bias, yf, st);
+      case 2: return bf ? launch_haar2d_inv<2>(pb, Yt, bias, yb, st) : launch_haar2d_inv<2>(pb, Yt, bias, yf, st);
+      default: return bf ? launch_haar2d_inv<3>(pb, Yt, bias, yb, st) : launch_haar2d_inv<3>(pb, Yt, bias, yf, st);
+    }
+  }
   if (pb.transform == STAMP_T_DCT2) {
     if (int rc = make_dct_matrix(pb.n, mat, st)) return rc;
     const dim3 grid((unsigned)(pb.nseq * ((pb.n + 63) / 64)), (unsigned)((pb.N + 63) / 64));
@@ -821,7 +869,7 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   float* T = reinterpret_cast<float*>(base + w.T);
   unsigned* rowmax = reinterpret_cast<unsigned*>(base + w.rowmax);
   CqChoice cc;
-  if (pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc))
+  if ((pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc))
     return run_quantize_cq(pb, cc, X, x_dtype, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
   if (dct_tc_ok(pb, x_dtype)) {
     int8_t* a8 = reinterpret_cast<int8_t*>(base + w.a8);
@@ -913,7 +961,7 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
   float* yt = reinterpret_cast<float*>(base + wl.yt);
   CqChoice cc;
-  const bool have_cq = pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc);
+  const bool have_cq = (pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc);
   if (have_cq && pb.transform == STAMP_T_HAAR && pb.levels >= 5 && pb.n % 256 == 0) {
     // Fused route: the transform+quantize kernel writes the token operand in tile order, the GEMM's
     // epilogue de-quantizes and inverts the (up to) 8 levels that close inside its 256-token tile.
@@ -1020,7 +1068,7 @@ int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, i
   if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
   uint8_t* base = static_cast<uint8_t*>(ws);
   CqChoice cc;
-  if (pb.transform != STAMP_T_DCT2 && choose_cq(pb.K, &cc))  // the product path's kernel with the fp32 export on
+  if ((pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc))  // the product path's kernel with the fp32 export on
     return run_quantize_cq(pb, cc, X, x_dtype, nullptr, nullptr, nullptr, reinterpret_cast<float*>(base + wl.xscale), T,
                            base, wl, static_cast<cudaStream_t>(stream));
   return run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + wl.ping),

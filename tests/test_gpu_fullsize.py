@@ -32,6 +32,7 @@ FULL = {
     "llm_mlp_up": gen.config_llm_up(),
     "dit_attn_proj": gen.config_dit_proj(),
     "llm_down_proj": gen.config_llm_down(),
+    "dit_attn_proj_2d": gen.config_dit_proj_2d(),
     "sweep_L512_D2048": gen.config_sweep(512, 2048),
     "sweep_L8192_D4096": gen.config_sweep(8192, 4096),
     "sweep_L32768_D8192": gen.config_sweep(32768, 8192),
@@ -43,7 +44,7 @@ def _oracle_transform_cols(oracle, cfg, Xc):
     n = cfg.block_len
     if cfg.transform == gen.T_HAAR and n > 4096:
         return oracle.apply_csr(oracle.haar_matrix_csr(n, cfg.levels), n, Xc)
-    return oracle.apply_dense(oracle.transform_matrix(cfg.transform, n, cfg.levels), Xc)
+    return oracle.apply_dense(oracle.transform_matrix(cfg.transform, n, cfg.levels, grid_w=cfg.grid), Xc)
 
 
 @pytest.mark.parametrize("name", list(FULL))
@@ -52,7 +53,7 @@ def test_full_size_parity(oracle, name):
     from paper_2510_26771_b200 import binding as st
     cfg = FULL[name]
     B, L, K, N, M = cfg.B, cfg.L, cfg.K, cfg.N, cfg.M
-    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi)
+    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid)
     X = gen.make_activation(cfg)
     rng = np.random.default_rng(1234)
     ncols = min(N, 64)
@@ -60,7 +61,7 @@ def test_full_size_parity(oracle, name):
     Wc = gen.make_weight(cfg, cols)
     bias = gen.make_bias(cfg)
     ref = oracle.stamp_linear(X, Wc, bias[cols], transform=cfg.transform, block=cfg.block, levels=cfg.levels,
-                              k_hi=cfg.k_hi, want=("x_scale", "q", "Y"))
+                              k_hi=cfg.k_hi, grid_w=cfg.grid, want=("x_scale", "q", "Y"))
 
     Xd = H.to_device(X, cfg.dtype)
     ws = st.alloc_workspace(c, B, L, K, N)

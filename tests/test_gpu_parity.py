@@ -34,12 +34,12 @@ def st():
 
 
 def _cfg_struct(st, cfg):
-    return st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi)
+    return st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid)
 
 
 def _oracle_all(oracle, cfg, X, W, bias=None, want=("T", "x_scale", "q", "w_scale", "wq", "acc", "Yt", "Y")):
     return oracle.stamp_linear(X, W, bias, transform=cfg.transform, block=cfg.block, levels=cfg.levels,
-                               k_hi=cfg.k_hi, want=want)
+                               k_hi=cfg.k_hi, grid_w=cfg.grid, want=want)
 
 
 def _allowed(count):
@@ -68,6 +68,9 @@ CASES = {
     "tile_depth5": gen.scaled(gen.config_dit_proj(), B=2, L=512, K=256, N=200, grid=0, block=256, levels=5, k_hi=8,
                               recipe="ar1"),
     "tile_depth7": gen.scaled(gen.config_llm_up(), B=1, L=1024, K=384, N=128, levels=7, k_hi=8),
+    # 2-D Haar over the patch grid: square and oblong grids, one to three levels
+    "haar2d_3": gen.scaled(gen.config_dit_proj_2d(), B=2, L=1024, K=256, N=136, grid=32, levels=3, k_hi=16),
+    "haar2d_1": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=128, N=64, grid=16, levels=1, k_hi=64),
     # two levels only: no cluster tree, approximation rows quantized by the same kernel
     "two_levels": gen.scaled(gen.config_dit_proj(), B=2, L=256, K=1152, N=128, grid=16, levels=2, k_hi=64),
 }
