@@ -38,7 +38,7 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_T_IDENTITY = 0, ORACLE_T_HAAR = 1, ORACLE_T_DCT2 = 2, ORACLE_T_HAAR2D = 3 };
+enum { ORACLE_T_IDENTITY = 0, ORACLE_T_HAAR = 1, ORACLE_T_DCT2 = 2, ORACLE_T_HAAR2D = 3, ORACLE_T_WHT = 4 };
 
 int oracle_num_threads(void) {
 #ifdef _OPENMP
@@ -127,6 +127,36 @@ int oracle_transform_matrix(int transform, int n, int levels, double* Lmat) {
       free(tmp);
     }
     return err;
+  }
+  if (transform == ORACLE_T_WHT) {
+    /* Walsh-Hadamard transform (Sec. "Efficient Energy Concentration": the DCT with only the signs
+     * of the basis kept).  Rows are the Walsh functions in SEQUENCY order -- row u changes sign u
+     * times along the tokens -- so that, as for the DCT, the slowly varying rows come first.  Built
+     * from the definition: the natural-order Hadamard matrix H[i][j] = (-1)^popcount(i & j), every
+     * row put at the index given by its number of sign changes, scaled by 1 / sqrt n. */
+    if (ilog2_exact(n) < 0) return 2;
+    double r = 1.0 / sqrt((double)n);
+    unsigned char* used = (unsigned char*)calloc((size_t)n, 1);
+    if (!used) return 3;
+    int bad = 0;
+    for (int i = 0; i < n; ++i) {
+      int changes = 0, prev = 0;
+      for (int j = 0; j < n; ++j) {
+        int bits = i & j, par = 0;
+        while (bits) { par ^= 1; bits &= bits - 1; }
+        if (j > 0 && par != prev) ++changes;
+        prev = par;
+      }
+      if (used[changes]) bad = 1;
+      used[changes] = 1;
+      for (int j = 0; j < n; ++j) {
+        int bits = i & j, par = 0;
+        while (bits) { par ^= 1; bits &= bits - 1; }
+        Lmat[(size_t)changes * n + j] = par ? -r : r;
+      }
+    }
+    free(used);
+    return bad ? 4 : 0;
   }
   if (transform == ORACLE_T_DCT2) {
     const double pi = 3.14159265358979323846264338327950288;

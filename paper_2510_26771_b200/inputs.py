@@ -21,7 +21,7 @@ import numpy as np
 from scipy.signal import lfilter
 
 # transform identifiers (values match the public C header's stamp_transform)
-T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D = 0, 1, 2, 3
+T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT = 0, 1, 2, 3, 4
 # storage dtypes (values match stamp_dtype)
 F32, BF16 = 0, 1
 
@@ -189,6 +189,11 @@ def config_dit_proj() -> LayerConfig:
                        outlier_gain=30.0, w_std=0.03, grid=64, length_scale=8.0)
 
 
+def config_llm_down_wht() -> LayerConfig:
+    """The down-projection workload with the Walsh-Hadamard transform in place of the DCT (same blocks)."""
+    return dataclasses.replace(config_llm_down(), name="llm_down_proj_wht", transform=T_WHT)
+
+
 def config_dit_proj_2d() -> LayerConfig:
     """The DiT projection with the paper's own LVM transform: 3-level 2-D Haar over the 64 x 64 patch grid,
     whose 64 low-pass tokens are the 8-bit ones."""
@@ -213,7 +218,7 @@ def config_sweep(L: int, D: int, levels: int = 0) -> LayerConfig:
 
 
 def named_configs() -> dict:
-    return {c.name: c for c in (config_tiny(), config_llm_up(), config_dit_proj(), config_llm_down(), config_dit_proj_2d())}
+    return {c.name: c for c in (config_tiny(), config_llm_up(), config_dit_proj(), config_llm_down(), config_dit_proj_2d(), config_llm_down_wht())}
 
 
 def scaled(cfg: LayerConfig, **kw) -> LayerConfig:

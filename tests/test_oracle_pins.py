@@ -459,3 +459,43 @@ def test_haar2d_layer_runs_and_marks_the_lowpass_tokens_high_precision(oracle):
     assert e[:16].sum() > 0.9 * e.sum()
     ref = oracle.matmul_f64(X.reshape(-1, cfg.K), W)
     assert np.linalg.norm(out["Y"] - ref) / np.linalg.norm(ref) < 0.2
+
+
+# ---------------------------------------------------------------------------------------------
+# Walsh-Hadamard transform (Sec. "Efficient Energy Concentration": the DCT with only the signs kept)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n", [2, 8, 64, 256])
+def test_wht_is_the_sequency_ordered_hadamard_matrix(oracle, n):
+    import scipy.linalg
+    Wm = oracle.transform_matrix(oracle.T_WHT, n)
+    assert np.abs(Wm @ Wm.T - np.eye(n)).max() <= 1e-12
+    assert np.array_equal(Wm, Wm.T)                                   # symmetric, hence its own inverse
+    assert np.allclose(np.abs(Wm), 1.0 / math.sqrt(n), rtol=0, atol=1e-15)
+    changes = (np.diff(np.sign(Wm), axis=1) != 0).sum(axis=1)
+    assert np.array_equal(changes, np.arange(n))                      # row u changes sign u times
+    # the same rows as the library's natural-order Hadamard matrix, reordered
+    Hn = scipy.linalg.hadamard(n) / math.sqrt(n)
+    assert {tuple(np.sign(r)) for r in Hn} == {tuple(np.sign(r)) for r in Wm}
+    assert np.allclose(Wm[0], 1.0 / math.sqrt(n))                     # row 0 = DC, as for the DCT
+
+
+def test_wht_rows_follow_the_sign_of_the_cosine_basis_at_low_sequency(oracle):
+    """"Retaining only the sign": the first rows of the WHT are the signs of the first DCT rows."""
+    n = 64
+    Wm = oracle.transform_matrix(oracle.T_WHT, n)
+    Cm = oracle.transform_matrix(oracle.T_DCT2, n)
+    for u in (0, 1, 2, 4, 8, 16, 32):     # dyadic frequencies: square waves with the cosine's zero crossings
+        assert np.array_equal(np.sign(Wm[u]), np.sign(Cm[u]))
+
+
+def test_wht_layer_runs_blockwise(oracle):
+    cfg = gen.scaled(gen.config_llm_down_wht(), B=1, L=512, K=128, N=64)
+    X, W = gen.make_activation(cfg), gen.make_weight(cfg)
+    out = oracle.stamp_linear(X, W, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi,
+                              want=("T", "q", "Y"))
+    Wm = oracle.transform_matrix(oracle.T_WHT, cfg.block)
+    T_np = np.einsum("ut,btk->buk", Wm, X.astype(np.float64).reshape(-1, cfg.block, cfg.K)).reshape(-1, cfg.K)
+    assert np.abs(out["T"] - T_np).max() <= 1e-12 * np.abs(T_np).max()
+    assert abs((out["T"] ** 2).sum() - (X.astype(np.float64) ** 2).sum()) <= 1e-10 * (X.astype(np.float64) ** 2).sum()
+    ref = oracle.matmul_f64(X.reshape(-1, cfg.K), W)
+    assert np.linalg.norm(out["Y"] - ref) / np.linalg.norm(ref) < 0.2
