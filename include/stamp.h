@@ -28,6 +28,8 @@
  *       Haar, l levels: [a_l (n/2^l rows) | d_l | d_(l-1) | ... | d_1 (n/2 rows)], with
  *         a[i] = (x[2i] + x[2i+1]) / sqrt2,  d[i] = (x[2i] - x[2i+1]) / sqrt2  per level;
  *       DCT-II (orthonormal): row u = frequency u, row 0 = DC.
+ *       Walsh-Hadamard (STAMP_T_WHT; the DCT reduced to its signs, same Section): orthonormal,
+ *         sequency order -- row u changes sign u times along the block's tokens, row 0 = DC.
  *       2-D Haar (STAMP_T_HAAR2D; Sec. "Efficient Energy Concentration", LVM set-up: 3 levels on the
  *         64 x 64 patch grid leave 64 low-pass tokens): the block's n tokens are a raster-ordered
  *         grid of n / grid_w rows x grid_w columns; per level every 2 x 2 cell (a b / c d) gives
@@ -62,7 +64,7 @@ typedef enum {
 
 typedef enum { STAMP_F32 = 0, STAMP_BF16 = 1 } stamp_dtype;
 
-typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2, STAMP_T_HAAR2D = 3 } stamp_transform;
+typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2, STAMP_T_HAAR2D = 3, STAMP_T_WHT = 4 } stamp_transform;
 
 typedef enum { STAMP_G_PER_TOKEN = 0, STAMP_G_PER_CHANNEL = 1 } stamp_granularity;
 

@@ -14,7 +14,7 @@ from .build import LIB_PATH
 
 STAMP_OK = 0
 F32, BF16 = 0, 1
-T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D = 0, 1, 2, 3
+T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT = 0, 1, 2, 3, 4
 G_PER_TOKEN, G_PER_CHANNEL = 0, 1
 W_PACKED4, W_INT8 = 0, 1
 

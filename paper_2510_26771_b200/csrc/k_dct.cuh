@@ -20,6 +20,26 @@ __global__ void __launch_bounds__(256) k_dct_matrix(int n, float* __restrict__ C
   C[idx] = static_cast<float>(cu * sqrt(2.0 / n) * cospi(static_cast<double>(a) / (2.0 * n)));
 }
 
+// Sign (+1 / -1) of entry (u, t) of the sequency-ordered Walsh-Hadamard matrix of size 2^bits: row u is
+// the natural-order Hadamard row  bit_reverse(gray(u)),  whose entry t is (-1)^popcount(row & t); that
+// row changes sign exactly u times (Sec. "Efficient Energy Concentration": the DCT reduced to its signs).
+__host__ __device__ __forceinline__ int wht_sign(int u, int t, int bits) {
+  const unsigned g = static_cast<unsigned>(u) ^ (static_cast<unsigned>(u) >> 1);
+  unsigned row = 0;
+  for (int b = 0; b < bits; ++b) row |= ((g >> b) & 1u) << (bits - 1 - b);
+  unsigned x = row & static_cast<unsigned>(t);
+  x ^= x >> 16; x ^= x >> 8; x ^= x >> 4; x ^= x >> 2; x ^= x >> 1;
+  return (x & 1u) ? -1 : 1;
+}
+
+// The n x n Walsh-Hadamard matrix (sequency order, orthonormal) in fp32.
+__global__ void __launch_bounds__(256) k_wht_matrix(int n, int bits, float* __restrict__ C) {
+  const long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long)n * n) return;
+  const int u = static_cast<int>(idx / n), t = static_cast<int>(idx - (long)u * n);
+  C[idx] = static_cast<float>(wht_sign(u, t, bits) / sqrt(static_cast<double>(n)));
+}
+
 __device__ __forceinline__ float ld_as_float(const float* p) { return *p; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p) {
   return __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(p)) << 16);

@@ -43,6 +43,8 @@ struct DctTcParams {
   void* y;               // [nblk * 256, cols] output of the inverse, float or bf16
   int y_bf16;
   const float* bias;     // [cols] or nullptr (inverse)
+  int nterms;            // products accumulated per tile: 3 for the DCT; the Walsh-Hadamard matrix (+-1/16) is one
+                         // exact bf16 term, so 1 forward and 2 (hi and lo plane) for its inverse
 };
 
 constexpr int DCT_N = 256;                 // block length
@@ -98,10 +100,11 @@ struct DctSmem {
 
 // term -> (which split of the matrix, which plane of B)
 template <int MODE>
-__device__ __forceinline__ void dct_term(int term, int& split, int& plane) {
+__device__ __forceinline__ void dct_term(int term, int nterms, int& split, int& plane) {
   if (MODE == DCT_TC_INVERSE) {
-    split = (term == 1) ? 1 : 0;
-    plane = (term == 2) ? 1 : 0;
+    // three terms: C1 hi, C2 hi, C1 lo;  two terms (single-term matrix): C1 hi, C1 lo
+    split = (nterms == 3 && term == 1) ? 1 : 0;
+    plane = (term == nterms - 1) ? 1 : 0;
   } else {
     split = term;
     plane = 0;
@@ -176,9 +179,9 @@ __global__ void __launch_bounds__(DCT_THREADS, 1)
           for (int a = 0; a < NATOM; ++a)
             ptx::tma_load_2d(bdst + (pl * NATOM + a) * DCT_ATOM_BYTES, pl == 0 ? &tmap_b0 : &tmap_b1, &bfull[bb],
                              (strip * NATOM + a) * 64, blk * DCT_N);
-        for (int term = 0; term < 3 && ok; ++term) {
+        for (int term = 0; term < p.nterms && ok; ++term) {
           int split, plane;
-          dct_term<MODE>(term, split, plane);
+          dct_term<MODE>(term, p.nterms, split, plane);
           for (int tb = 0; tb < 4; ++tb) {
             if (!ptx::mbar_wait_bounded(&aempty[st], aphase ^ 1u, abort_word, DCT_WAIT_LIMIT)) { ok = false; break; }
             ptx::mbar_arrive_expect_tx(&afull[st], DCT_A_BYTES);
@@ -212,9 +215,9 @@ __global__ void __launch_bounds__(DCT_THREADS, 1)
         ptx::tc_fence_after();
         const uint32_t bbase = ptx::smem_u32(smem + bb * SM::B_BYTES);
         const uint32_t dbase = tmem_base + static_cast<uint32_t>(bb * SM::ACC_COLS);
-        for (int term = 0; term < 3 && ok; ++term) {
+        for (int term = 0; term < p.nterms && ok; ++term) {
           int split, plane;
-          dct_term<MODE>(term, split, plane);
+          dct_term<MODE>(term, p.nterms, split, plane);
           for (int tb = 0; tb < 4; ++tb) {
             if (!ptx::mbar_wait_bounded(&afull[st], aphase, abort_word, DCT_WAIT_LIMIT)) { ok = false; break; }
             ptx::tc_fence_after();
@@ -344,14 +347,20 @@ __global__ void __launch_bounds__(DCT_THREADS, 1)
 // The three bf16 terms of the orthonormal 256-point DCT-II matrix, as A operands:
 //   out[(s * 256 + r) * 256 + k] = term s of  C[r][k]  (forward: rows = frequencies)
 //                                  or of      C[k][r]  (transpose = inverse: rows = tokens)
-__global__ void __launch_bounds__(256) k_dct_split_matrix(int transpose, __nv_bfloat16* __restrict__ out) {
+// wht != 0: the sequency-ordered Walsh-Hadamard matrix instead (entries +-1/16: term 1 is exact, the others 0).
+__global__ void __launch_bounds__(256) k_dct_split_matrix(int transpose, int wht, __nv_bfloat16* __restrict__ out) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= DCT_N * DCT_N) return;
   const int r = idx / DCT_N, k = idx - r * DCT_N;
   const int u = transpose ? k : r, t = transpose ? r : k;
-  const long a = ((long)(2 * t + 1) * u) % (4L * DCT_N);
-  const double cu = (u == 0) ? 0.70710678118654752440 : 1.0;
-  double c = cu * sqrt(2.0 / DCT_N) * cospi(static_cast<double>(a) / (2.0 * DCT_N));
+  double c;
+  if (wht) {
+    c = wht_sign(u, t, 8) * 0.0625;
+  } else {
+    const long a = ((long)(2 * t + 1) * u) % (4L * DCT_N);
+    const double cu = (u == 0) ? 0.70710678118654752440 : 1.0;
+    c = cu * sqrt(2.0 / DCT_N) * cospi(static_cast<double>(a) / (2.0 * DCT_N));
+  }
 #pragma unroll
   for (int s = 0; s < 3; ++s) {
     const __nv_bfloat16 h = __double2bfloat16(c);

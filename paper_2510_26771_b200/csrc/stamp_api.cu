@@ -41,7 +41,7 @@ static inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool need_n, Problem* out) {
   if (!cfg || !out) return STAMP_ERR_INVALID_ARG;
   if (B <= 0 || L <= 0 || K <= 0 || (need_n && N <= 0)) return STAMP_ERR_INVALID_ARG;
-  if (cfg->transform < STAMP_T_IDENTITY || cfg->transform > STAMP_T_HAAR2D) return STAMP_ERR_INVALID_ARG;
+  if (cfg->transform < STAMP_T_IDENTITY || cfg->transform > STAMP_T_WHT) return STAMP_ERR_INVALID_ARG;
   if (cfg->block < 0 || cfg->levels < 0 || cfg->k_hi < 0 || cfg->grid_w < 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->transform != STAMP_T_HAAR2D && cfg->grid_w != 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->bits_hi != 8 || cfg->bits_lo != 4 || cfg->bits_w != 4) return STAMP_ERR_UNSUPPORTED;
@@ -58,7 +58,8 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
     levels = cfg->levels ? cfg->levels : full;
     if (levels > full) return STAMP_ERR_UNSUPPORTED;
   }
-  if (cfg->transform == STAMP_T_DCT2 && n > 4096) return STAMP_ERR_UNSUPPORTED;  // dense n x n matrix in scratch
+  if ((cfg->transform == STAMP_T_DCT2 || cfg->transform == STAMP_T_WHT) && n > 4096)
+    return STAMP_ERR_UNSUPPORTED;  // dense n x n matrix in scratch
   if (cfg->transform == STAMP_T_HAAR2D) {
     const int w = cfg->grid_w;
     if (w <= 0 || n % w != 0) return STAMP_ERR_INVALID_ARG;
@@ -132,7 +133,8 @@ static Workspace layout(const Problem& pb) {
   w.atop = off;     off += align256((M >> 3) * (size_t)pb.K * 4);
   w.top_ping = off; off += align256((M >> 6) * (size_t)pb.K * 4);
   w.top_pong = off; off += align256((M >> 9) * (size_t)pb.K * 4);
-  w.dctmat = off; off += align256(pb.transform == STAMP_T_DCT2 ? (size_t)pb.n * pb.n * 4 : 0);
+  const bool dense = pb.transform == STAMP_T_DCT2 || pb.transform == STAMP_T_WHT;
+  w.dctmat = off; off += align256(dense ? (size_t)pb.n * pb.n * 4 : 0);
   // the top table follows the M rows of a8 directly: the tiled route addresses it as rows M, M + 1, ...
   w.a8 = off;     off += M * (size_t)pb.K;
   w.a8top = off;  off += align256((M >> 8) * (size_t)pb.K) + 256;
@@ -144,7 +146,7 @@ static Workspace layout(const Problem& pb) {
   w.yttop = off;  off += align256((M >> 8) * (size_t)pb.N * 4);
   w.a8v = off;    off += align256((M >> 8) * (size_t)pb.N * 4);
   // bf16 terms of the DCT matrix and of its transpose (tensor-core DCT)
-  w.dctsplit = off; off += align256(pb.transform == STAMP_T_DCT2 ? (size_t)2 * 3 * DCT_N * DCT_N * 2 : 0);
+  w.dctsplit = off; off += align256(dense ? (size_t)2 * 3 * DCT_N * DCT_N * 2 : 0);
   w.total = off;
   return w;
 }
@@ -360,8 +362,12 @@ static int run_haar_passes(const void* in, bool in_bf16, int nseq, int Lin, int 
   return STAMP_OK;
 }
 
-static int make_dct_matrix(int n, float* mat, cudaStream_t st) {
-  k_dct_matrix<<<(unsigned)(((long)n * n + 255) / 256), 256, 0, st>>>(n, mat);
+// The dense n x n matrix of a block transform: DCT-II or sequency-ordered Walsh-Hadamard.
+static int make_dct_matrix(int transform, int n, float* mat, cudaStream_t st) {
+  if (transform == STAMP_T_WHT)
+    k_wht_matrix<<<(unsigned)(((long)n * n + 255) / 256), 256, 0, st>>>(n, ilog2(n), mat);
+  else
+    k_dct_matrix<<<(unsigned)(((long)n * n + 255) / 256), 256, 0, st>>>(n, mat);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
 }
@@ -397,9 +403,9 @@ static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, 
       default: return bf ? launch_haar2d_fwd<3>(pb, xb, T, rowmax, st) : launch_haar2d_fwd<3>(pb, xf, T, rowmax, st);
     }
   }
-  if (pb.transform == STAMP_T_DCT2) {
+  if (pb.transform == STAMP_T_DCT2 || pb.transform == STAMP_T_WHT) {
     if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
-    if (int rc = make_dct_matrix(pb.n, mat, st)) return rc;
+    if (int rc = make_dct_matrix(pb.transform, pb.n, mat, st)) return rc;
     const dim3 grid((unsigned)(pb.nseq * ((pb.n + 63) / 64)), (unsigned)((pb.K + 63) / 64));
     if (x_dtype == STAMP_BF16)
       k_dct_apply<false, __nv_bfloat16, float><<<grid, 256, 0, st>>>(mat, pb.n, static_cast<const __nv_bfloat16*>(X),
@@ -443,8 +449,8 @@ static int run_inverse_generic(const Problem& pb, const float* Yt, const float* 
       default: return bf ? launch_haar2d_inv<3>(pb, Yt, bias, yb, st) : launch_haar2d_inv<3>(pb, Yt, bias, yf, st);
     }
   }
-  if (pb.transform == STAMP_T_DCT2) {
-    if (int rc = make_dct_matrix(pb.n, mat, st)) return rc;
+  if (pb.transform == STAMP_T_DCT2 || pb.transform == STAMP_T_WHT) {
+    if (int rc = make_dct_matrix(pb.transform, pb.n, mat, st)) return rc;
     const dim3 grid((unsigned)(pb.nseq * ((pb.n + 63) / 64)), (unsigned)((pb.N + 63) / 64));
     if (y_dtype == STAMP_BF16)
       k_dct_apply<true, float, __nv_bfloat16><<<grid, 256, 0, st>>>(mat, pb.n, Yt, pb.N, static_cast<__nv_bfloat16*>(Y),
@@ -679,7 +685,7 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
 // Blockwise 256-point DCT-II on the tensor cores (bf16 activations).
 // ------------------------------------------------------------------------------------------
 static bool dct_tc_ok(const Problem& pb, int x_dtype) {
-  return pb.transform == STAMP_T_DCT2 && pb.n == DCT_N && x_dtype == STAMP_BF16;
+  return (pb.transform == STAMP_T_DCT2 || pb.transform == STAMP_T_WHT) && pb.n == DCT_N && x_dtype == STAMP_BF16;
 }
 
 // Transform + quantizer: row maxima in a first launch, codes (a8, logical order) and scales in a second.
@@ -687,7 +693,8 @@ static int run_quantize_dct_tc(const Problem& pb, const void* X, int8_t* a8, flo
                                const Workspace& wl, cudaStream_t st) {
   __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(base + wl.dctsplit);
   unsigned* rowmax = reinterpret_cast<unsigned*>(base + wl.rowmax);
-  k_dct_split_matrix<<<DCT_N * DCT_N / 256, 256, 0, st>>>(0, split);
+  const int wht = pb.transform == STAMP_T_WHT;
+  k_dct_split_matrix<<<DCT_N * DCT_N / 256, 256, 0, st>>>(0, wht, split);
   STAMP_CHECK_LAUNCH();
   if (cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
   CUtensorMap ta, tb;
@@ -703,6 +710,7 @@ static int run_quantize_dct_tc(const Problem& pb, const void* X, int8_t* a8, flo
   dp.rowmax = rowmax;
   dp.a8 = a8;
   dp.x_scale = x_scale;
+  dp.nterms = wht ? 1 : 3;
   if ((rc = launch_dct_tc<DCT_TC_MAX, 2, 1>(ta, tb, tb, dp, st))) return rc;
   return launch_dct_tc<DCT_TC_QUANT, 2, 1>(ta, tb, tb, dp, st);
 }
@@ -711,7 +719,8 @@ static int run_quantize_dct_tc(const Problem& pb, const void* X, int8_t* a8, flo
 static int run_inverse_dct_tc(const Problem& pb, const __nv_bfloat16* planes, const float* bias, void* Y, int y_dtype,
                               uint8_t* base, const Workspace& wl, cudaStream_t st) {
   __nv_bfloat16* split = reinterpret_cast<__nv_bfloat16*>(base + wl.dctsplit) + 3 * DCT_N * DCT_N;
-  k_dct_split_matrix<<<DCT_N * DCT_N / 256, 256, 0, st>>>(1, split);
+  const int wht = pb.transform == STAMP_T_WHT;
+  k_dct_split_matrix<<<DCT_N * DCT_N / 256, 256, 0, st>>>(1, wht, split);
   STAMP_CHECK_LAUNCH();
   CUtensorMap ta, tb0, tb1;
   int rc = make_tmap_bf16(split, 3 * DCT_N, DCT_N, &ta);
@@ -724,6 +733,7 @@ static int run_inverse_dct_tc(const Problem& pb, const __nv_bfloat16* planes, co
   dp.y = Y;
   dp.y_bf16 = (y_dtype == STAMP_BF16);
   dp.bias = bias;
+  dp.nterms = wht ? 2 : 3;
   return launch_dct_tc<DCT_TC_INVERSE, 1, 2>(ta, tb0, tb1, dp, st);
 }
 
@@ -932,7 +942,8 @@ int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float*
   const PassPlan pl = make_plan(pb.levels);
   const size_t ping_bytes = pl.npass > 1 ? align256(((size_t)pb.M >> pl.p[0]) * pb.N * 4) : 0;
   const size_t pong_bytes = pl.npass > 2 ? align256(((size_t)pb.M >> (pl.p[0] + pl.p[1])) * pb.N * 4) : 0;
-  const size_t mat_bytes = pb.transform == STAMP_T_DCT2 ? align256((size_t)pb.n * pb.n * 4) : 0;
+  const size_t mat_bytes =
+      (pb.transform == STAMP_T_DCT2 || pb.transform == STAMP_T_WHT) ? align256((size_t)pb.n * pb.n * 4) : 0;
   if (ping_bytes + pong_bytes + mat_bytes > (size_t)STAMP_NOALLOC_SCRATCH_BYTES) return STAMP_ERR_TOO_LARGE;
   uint8_t* base = nullptr;
   if ((rc = noalloc_scratch_base(&base))) return rc;

@@ -26,13 +26,14 @@ def _scale_rtol(cfg):
     """A scale is absmax / qmax of a transformed row, so it inherits the tolerance on T.  Haar
     coefficients see at most log2(n) fp32 roundings (1e-6 holds); a DCT coefficient is an fp32 sum
     of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised."""
-    return 1e-5 if cfg.transform == gen.T_DCT2 else 1e-6
+    return 1e-5 if cfg.transform in (gen.T_DCT2, gen.T_WHT) else 1e-6
 
 FULL = {
     "llm_mlp_up": gen.config_llm_up(),
     "dit_attn_proj": gen.config_dit_proj(),
     "llm_down_proj": gen.config_llm_down(),
     "dit_attn_proj_2d": gen.config_dit_proj_2d(),
+    "llm_down_proj_wht": gen.config_llm_down_wht(),
     "sweep_L512_D2048": gen.config_sweep(512, 2048),
     "sweep_L8192_D4096": gen.config_sweep(8192, 4096),
     "sweep_L32768_D8192": gen.config_sweep(32768, 8192),

@@ -21,7 +21,7 @@ def _scale_rtol(cfg):
     """A scale is absmax / qmax of a transformed row, so it inherits the tolerance on T.  Haar
     coefficients see at most log2(n) fp32 roundings (1e-6 holds); a DCT coefficient is an fp32 sum
     of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised."""
-    return 1e-5 if cfg.transform == gen.T_DCT2 else 1e-6
+    return 1e-5 if cfg.transform in (gen.T_DCT2, gen.T_WHT) else 1e-6
 
 
 @pytest.fixture(scope="module")
@@ -63,6 +63,9 @@ CASES = {
     "dct_blocks": gen.scaled(gen.config_llm_down(), B=2, L=512, K=384, N=136),
     # output width a multiple of 64: the layer's inverse DCT also runs on the tensor cores
     "dct_tensor_inverse": gen.scaled(gen.config_llm_down(), B=1, L=768, K=256, N=192),
+    # Walsh-Hadamard blocks: 256 tokens (tensor cores, one exact bf16 term) and a short block (general kernels)
+    "wht_blocks": gen.scaled(gen.config_llm_down_wht(), B=2, L=512, K=384, N=192),
+    "wht_short_block": gen.scaled(gen.config_llm_down_wht(), B=1, L=256, K=128, N=72, block=64, k_hi=4),
     "dct_short_block": gen.scaled(gen.config_llm_down(), B=1, L=256, K=128, N=64, block=32, k_hi=4),
     # fused inverse epilogue with 5 and 7 levels closed inside a 256-token tile (8 and 6 are covered above)
     "tile_depth5": gen.scaled(gen.config_dit_proj(), B=2, L=512, K=256, N=200, grid=0, block=256, levels=5, k_hi=8,
