@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
         for (int i = 0; i < G; i += 2 * st) {
           const float2 a = v[h][i], b2 = v[h][i + st];
           v[h][i] = __fadd2_rn(a, b2);
-          v[h][i + st] = __ffma2_rn(b2, cq_f2(-1.0f), a);
+          v[h][i + st] = ptx::fsub2_rn(a, b2);
         }
       }
     }

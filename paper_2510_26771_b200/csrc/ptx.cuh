@@ -22,6 +22,17 @@ __device__ __forceinline__ T* ptr_mad_wide(T* base, int a, int b) {
   return reinterpret_cast<T*>(r);
 }
 
+// Packed fp32x2 subtraction (there is an intrinsic for add, mul and fma only).
+__device__ __forceinline__ float2 fsub2_rn(float2 a, float2 b) {
+  uint64_t ra, rb, rd;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+  float2 r;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(rd));
+  return r;
+}
+
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(
