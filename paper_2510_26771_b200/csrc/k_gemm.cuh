@@ -15,8 +15,10 @@
 //              STAGES-deep shared-memory ring (one mbarrier pair per stage)
 //   warp 1     allocates TMEM; one elected thread issues tcgen05.mma kind::i8 (128 x BN x 32
 //              per instruction, four per 128-byte K block) into one of two accumulators
-//   warps 2-5  epilogue: tcgen05.ld the finished accumulator (the other one is being filled),
-//              de-quantize with per-token x per-channel scales, store
+//   warps 2-9  epilogue: tcgen05.ld the finished accumulator (the other one is being filled),
+//              de-quantize with per-token x per-channel scales, store.  A warp reaches only the 32
+//              TMEM lanes of its quarter (warp % 4), so two warps share a quarter and each drains
+//              half of the accumulator's columns
 // Every mbarrier wait is bounded; when one expires the CTA raises the device status word,
 // drains its outstanding copies, frees TMEM and returns.
 #pragma once
@@ -47,7 +49,8 @@ struct GemmParams {
 
 constexpr int GEMM_BM = 128;           // output channels per tile
 constexpr int GEMM_BK = 128;           // int8 per K block = one 128-byte swizzle row
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_EPI_THREADS = 256;   // two epilogue warps per TMEM lane quarter, each draining half the columns
+constexpr int GEMM_THREADS = 64 + GEMM_EPI_THREADS;
 constexpr long long GEMM_WAIT_LIMIT = 4000000000LL;  // SM clocks (~2 s) before a wait gives up
 
 template <int BN, int STAGES>
@@ -103,7 +106,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&tfull[a], 1);
-      ptx::mbar_init(&tempty[a], 128);
+      ptx::mbar_init(&tempty[a], GEMM_EPI_THREADS);
     }
     *abort_word = 0;
     ptx::fence_mbar_init();
@@ -207,7 +210,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32 * (warp % 4) ...
     const int row = quarter * 32 + lane;
-    const int ep_tid = threadIdx.x - 64;  // 0..127
+    const int half = (warp - 2) >> 2;     // which half of the accumulator's columns this warp drains
+    const int ep_tid = threadIdx.x - 64;  // 0..255
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
@@ -221,29 +225,24 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       const bool full_tile = (tok0 + BN <= p.m_tok);
       float* sxs = sx_stage + a * BN;
       float sw = 0.f;
-      float my_sx[BN / 128];
+      float my_sx = 0.f;
       if (EPI != EPI_RAW_I32) {
         if (ch_ok) sw = p.w_scale ? __ldg(p.w_scale + ch) : 1.0f;
         // fetch this tile's token scales while the accumulator is still being filled
-#pragma unroll
-        for (int i = 0; i < BN / 128; ++i) {
-          const int tok = tok0 + i * 128 + ep_tid;
-          my_sx[i] = (tok < p.m_tok) ? __ldg(p.x_scale + tok) : 0.f;
-        }
+        if (ep_tid < BN && tok0 + ep_tid < p.m_tok) my_sx = __ldg(p.x_scale + tok0 + ep_tid);
       }
-      // The four epilogue warps continue or stop TOGETHER: a warp whose wait ran out raises the abort
+      // The eight epilogue warps continue or stop TOGETHER: a warp whose wait ran out raises the abort
       // word, and everybody reads it behind the named barrier below -- no warp is left waiting at that
       // barrier for one that already gave up.  (The TMEM loads are warp-collective as well.)
       if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&tfull[a], acc_phase, abort_word, GEMM_WAIT_LIMIT)))
         *abort_word = 1;
       ptx::tc_fence_after();
       if (EPI != EPI_RAW_I32) {
-        // every epilogue thread has finished the previous tile that used accumulator `a` (all 128
-        // arrived on tempty[a] before tfull[a] could complete again), so its staging buffer is free
-#pragma unroll
-        for (int i = 0; i < BN / 128; ++i) sxs[i * 128 + ep_tid] = my_sx[i];
+        // every epilogue thread has finished the previous tile that used accumulator `a` (all of
+        // them arrived on tempty[a] before tfull[a] could complete again), so its staging buffer is free
+        if (ep_tid < BN) sxs[ep_tid] = my_sx;
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, %0;" ::"n"(GEMM_EPI_THREADS) : "memory");
       if (*abort_word != 0u) {
         ok = false;
         break;
@@ -289,16 +288,18 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
             for (int i = 0; i < 8; ++i) a5[i] = hd[i];
           }
         }
-        // ---- eight chunks of 32 tokens: slot 0 <- level-5 sum, 31 details, five synthesis levels
+        // ---- this warp's four chunks of 32 tokens: slot 0 <- level-5 sum, 31 details, five synthesis levels
+        const int c0 = half * 4;
         uint32_t r[2][32];
-        ptx::tmem_ld_32x32b_x32(taddr, r[0]);
+        ptx::tmem_ld_32x32b_x32(taddr + c0 * 32, r[0]);
 #pragma unroll
-        for (int chunk = 0; chunk < 8; ++chunk) {
+        for (int ci = 0; ci < 4; ++ci) {
+          const int chunk = c0 + ci;
           ptx::tmem_ld_wait();
-          if (chunk + 1 < 8) ptx::tmem_ld_32x32b_x32(taddr + (chunk + 1) * 32, r[(chunk + 1) & 1]);
-          const uint32_t(&rc)[32] = r[chunk & 1];
+          if (ci + 1 < 4) ptx::tmem_ld_32x32b_x32(taddr + (chunk + 1) * 32, r[(ci + 1) & 1]);
+          const uint32_t(&rc)[32] = r[ci & 1];
           float y[32];
-          y[0] = a5[chunk];
+          y[0] = half ? a5[4 + ci] : a5[ci];
 #pragma unroll
           for (int len = 1; len < 32; len <<= 1) {
 #pragma unroll
@@ -323,13 +324,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
           }
         }
       } else {
+      constexpr int NCH = BN / 64;   // chunks of 32 tokens per warp
+      const int c0 = half * NCH;
       uint32_t r[2][32];
-      ptx::tmem_ld_32x32b_x32(taddr, r[0]);
+      ptx::tmem_ld_32x32b_x32(taddr + c0 * 32, r[0]);
 #pragma unroll
-      for (int chunk = 0; chunk < BN / 32; ++chunk) {
+      for (int ci = 0; ci < NCH; ++ci) {
+        const int chunk = c0 + ci;
         ptx::tmem_ld_wait();
-        if (chunk + 1 < BN / 32) ptx::tmem_ld_32x32b_x32(taddr + (chunk + 1) * 32, r[(chunk + 1) & 1]);
-        const uint32_t(&rc)[32] = r[chunk & 1];
+        if (ci + 1 < NCH) ptx::tmem_ld_32x32b_x32(taddr + (chunk + 1) * 32, r[(ci + 1) & 1]);
+        const uint32_t(&rc)[32] = r[ci & 1];
         const int tbase = tok0 + chunk * 32;
         if (EPI == EPI_DEQUANT_F32) {
           float* out = static_cast<float*>(p.out) + (long)tbase * p.n_out + ch;
