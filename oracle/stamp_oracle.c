@@ -12,7 +12,8 @@
  *   - Activation quantizer, Background Sec. 2.1, first equation (integer quantization with
  *     per-token scale shared across features), in its symmetric form: zero-point 0, codes
  *     in [-(2^(b-1)-1), +(2^(b-1)-1)], scale = absmax / qmax so that nothing clips (the
- *     min-max, "no clipping error" range setting of the same section).
+ *     min-max, "no clipping error" range setting of the same section); and, selectable, in
+ *     the form the equation prints: unsigned codes with an integer zero point, s = range / (2^b - 1).
  *   - Two-level bit allocation (end of Sec. "Optimal bit allocation"): the first k_hi
  *     transformed tokens of each transform block use bits_hi, the rest bits_lo.
  *   - Sequence transforms (Sec. "Efficient Energy Concentration"): orthonormal multi-level
@@ -23,7 +24,9 @@
  * Pins (tests/test_oracle_pins.py): orthonormality, closed-form Haar rows, SciPy's
  * orthonormal DCT-II, energy preservation, exact reconstruction, identity of the
  * unquantized pipeline with X W^T, the bias form l = L 1, rounding/error bounds, the
- * printed effective bit-widths 4.0625 and 4.125, brute force on tiny shapes.
+ * printed effective bit-widths 4.0625 and 4.125, brute force on tiny shapes; for the zero-point
+ * quantizer a hand-computed row, the section's error bound d s^2 / 4, the nearest-level property by
+ * brute force, and the integer product against a float product of the de-quantized operands.
  * Conventions that no pin can fix (they are choices shared with the CUDA path by
  * specification; "parity unpinned" for these): the sign of the Haar detail rows, the
  * round-half-to-even tie rule, symmetric instead of zero-point codes.
@@ -424,6 +427,72 @@ int oracle_quantize_rows(const double* T, long rows, int K, const int32_t* bits_
   return 0;
 }
 
+/* ------------------------------------------------------------------------------------------
+ * Per-row asymmetric (zero-point) round-to-nearest quantizer: Sec. 2.1, first equation, as printed,
+ *   x_int = clamp(rne(x / s) + z, 0, 2^b - 1),      de-quantized value  s * (x_int - z),
+ * with the min-max range setting of the same section (the one under which its error bound holds):
+ *   s = range(x) / (2^b - 1),  range(x) = max_j x_j - min_j x_j,      z = rne(-min_j x_j / s).
+ * The printed scale formula of that passage is the reciprocal of the s used in the equation and in
+ * the bound; the reading taken here is the one consistent with both.  z is an integer (it is added
+ * to an integer code) and is not clamped to the code range: a row that does not straddle zero has
+ * z < 0 or z > 2^b - 1 and still uses all its codes.  |z| is limited to 2^30 so that it fits an
+ * int32 (only a row whose range is ~1e-7 of its offset gets there).  range == 0 (a constant row; the
+ * zero row of a padded sequence) takes s = 1.
+ * As in the symmetric quantizer, min, max, s and the rounding decision are taken in fp32.
+ * ------------------------------------------------------------------------------------------ */
+int oracle_quantize_rows_asym(const double* T, long rows, int K, const int32_t* bits_per_row, int period,
+                              float* scale, int32_t* zero, uint8_t* codes) {
+  if (period <= 0) return 1;
+#pragma omp parallel for schedule(static)
+  for (long r = 0; r < rows; ++r) {
+    const double* t = T + (size_t)r * K;
+    int bits = bits_per_row[r % period];
+    float top = (float)((1 << bits) - 1);
+    float mn = (float)t[0], mx = (float)t[0];
+    for (int j = 1; j < K; ++j) {
+      float v = (float)t[j];
+      if (v < mn) mn = v;
+      if (v > mx) mx = v;
+    }
+    float s = (mx - mn) / top;
+    if (!(s > 0.0f)) s = 1.0f;
+    float zf = rintf(-mn / s);
+    if (zf > 1073741824.0f) zf = 1073741824.0f;
+    if (zf < -1073741824.0f) zf = -1073741824.0f;
+    scale[r] = s;
+    zero[r] = (int32_t)zf;
+    for (int j = 0; j < K; ++j) {
+      float q = rintf((float)t[j] / s) + zf;
+      if (q > top) q = top;
+      if (q < 0.0f) q = 0.0f;
+      codes[(size_t)r * K + j] = (uint8_t)q;
+    }
+  }
+  return 0;
+}
+
+/* Integer matmul on zero-point codes: acc[m][n] = sum_k (q[m][k] - z[m]) * wq[n][k]  (the de-quantized
+ * activation of Sec. 2.1 is s (x_int - z); the scale is applied afterwards).  int64 accumulation,
+ * checked to fit int32 (returns 5 otherwise). */
+int oracle_gemm_zp_i32(const uint8_t* q, const int32_t* zero, const int8_t* wq, long M, int N, int K,
+                       int32_t* acc) {
+  int overflow = 0;
+#pragma omp parallel for schedule(static)
+  for (long m = 0; m < M; ++m)
+    for (int n = 0; n < N; ++n) {
+      int64_t s = 0;
+      const uint8_t* a = q + (size_t)m * K;
+      const int8_t* b = wq + (size_t)n * K;
+      for (int k = 0; k < K; ++k) s += ((int64_t)a[k] - (int64_t)zero[m]) * (int64_t)b[k];
+      if (s > INT32_MAX || s < INT32_MIN) {
+#pragma omp atomic write
+        overflow = 1;
+      }
+      acc[(size_t)m * N + n] = (int32_t)s;
+    }
+  return overflow ? 5 : 0;
+}
+
 /* float-input convenience for the weights (per output channel, Sec. "Set-up": a separate
  * scale for each weight output channel; round-to-nearest). */
 int oracle_quantize_rows_f32in(const float* W, long rows, int K, int bits, float* scale, int8_t* codes) {
@@ -509,17 +578,19 @@ int oracle_matmul_f64(const float* X, const float* W, long M, int N, int K, doub
  *   acc      [B*L, N]  int32  integer accumulators
  *   Yt       [B*L, N]  fp64   de-quantized output, transformed domain
  *   Y        [B*L, N]  fp64   final output
+ * act_asym != 0 selects the zero-point activation quantizer: q then holds UNSIGNED bytes, x_zero
+ * [B*L] receives the zero points (it may be null otherwise) and acc is the sum over (q - z) * wq.
  * Returns 0 on success.
  * ------------------------------------------------------------------------------------------ */
 int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B, int L, int K, int N,
                         int transform, int block, int levels, int k_hi, int bits_hi, int bits_lo,
                         int bits_w, double* T, float* x_scale, int8_t* q, float* w_scale, int8_t* wq,
-                        int32_t* acc, double* Yt, double* Y, int grid_w) {
+                        int32_t* acc, double* Yt, double* Y, int grid_w, int act_asym, int32_t* x_zero) {
   int n = block ? block : L;
   if (n <= 0 || L % n) return 1;
   long M = (long)B * L;
   int rc = 0;
-  int own_T = 0, own_xs = 0, own_q = 0, own_ws = 0, own_wq = 0, own_acc = 0, own_Yt = 0;
+  int own_T = 0, own_xs = 0, own_q = 0, own_ws = 0, own_wq = 0, own_acc = 0, own_Yt = 0, own_xz = 0;
   double* Lmat = NULL;
   int64_t* rp = NULL; int32_t* ci = NULL; double* cv = NULL;
   int32_t* bits = NULL;
@@ -530,6 +601,7 @@ int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B
   OWN(T, own_T, double, (size_t)M * K)
   OWN(x_scale, own_xs, float, M)
   OWN(q, own_q, int8_t, (size_t)M * K)
+  if (act_asym) { OWN(x_zero, own_xz, int32_t, M) }
   OWN(w_scale, own_ws, float, N)
   OWN(wq, own_wq, int8_t, (size_t)N * K)
   OWN(acc, own_acc, int32_t, (size_t)M * N)
@@ -563,7 +635,8 @@ int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B
   if (!bits) { rc = 3; goto done; }
   rc = oracle_bit_map(L, n, k_hi, bits_hi, bits_lo, bits);
   if (rc) goto done;
-  rc = oracle_quantize_rows(T, M, K, bits, L, x_scale, q);
+  rc = act_asym ? oracle_quantize_rows_asym(T, M, K, bits, L, x_scale, x_zero, (uint8_t*)q)
+                : oracle_quantize_rows(T, M, K, bits, L, x_scale, q);
   if (rc) goto done;
 
   /* quantized weights (static; untouched by the sequence transform) */
@@ -571,7 +644,8 @@ int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B
   if (rc) goto done;
 
   /* Y <- X W^T on the integer codes, then de-quantize */
-  rc = oracle_gemm_i32(q, wq, M, N, K, acc);
+  rc = act_asym ? oracle_gemm_zp_i32((const uint8_t*)q, x_zero, wq, M, N, K, acc)
+                : oracle_gemm_i32(q, wq, M, N, K, acc);
   if (rc) goto done;
   rc = oracle_dequant(acc, x_scale, w_scale, M, N, Yt);
   if (rc) goto done;
@@ -593,6 +667,7 @@ done:
   if (own_T) free(T);
   if (own_xs) free(x_scale);
   if (own_q) free(q);
+  if (own_xz) free(x_zero);
   if (own_ws) free(w_scale);
   if (own_wq) free(wq);
   if (own_acc) free(acc);

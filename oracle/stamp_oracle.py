@@ -117,6 +117,31 @@ def quantize_rows(T: np.ndarray, bits_per_row: np.ndarray):
     return codes, scale
 
 
+def quantize_rows_asym(T: np.ndarray, bits_per_row: np.ndarray):
+    """Per-row zero-point RTN quantizer (Sec. 2.1, first equation, min-max range).  Returns unsigned
+    codes [rows, K] uint8, scales [rows] float32 and integer zero points [rows] int32."""
+    T = np.ascontiguousarray(T, dtype=np.float64)
+    rows, K = T.shape
+    bits_per_row = np.ascontiguousarray(bits_per_row, dtype=np.int32)
+    scale = np.empty(rows, dtype=np.float32)
+    zero = np.empty(rows, dtype=np.int32)
+    codes = np.empty((rows, K), dtype=np.uint8)
+    _check(lib().oracle_quantize_rows_asym(_p(T), ctypes.c_long(rows), K, _p(bits_per_row), len(bits_per_row),
+                                           _p(scale), _p(zero), _p(codes)), "quantize_rows_asym")
+    return codes, scale, zero
+
+
+def gemm_zp_i32(q: np.ndarray, zero: np.ndarray, wq: np.ndarray) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    zero = np.ascontiguousarray(zero, dtype=np.int32)
+    wq = np.ascontiguousarray(wq, dtype=np.int8)
+    M, K = q.shape
+    N = wq.shape[0]
+    acc = np.empty((M, N), dtype=np.int32)
+    _check(lib().oracle_gemm_zp_i32(_p(q), _p(zero), _p(wq), ctypes.c_long(M), N, K, _p(acc)), "gemm_zp_i32")
+    return acc
+
+
 def quantize_weights(W: np.ndarray, bits: int = 4):
     W = np.ascontiguousarray(W, dtype=np.float32)
     N, K = W.shape
@@ -159,8 +184,12 @@ def matmul_f64(X: np.ndarray, W: np.ndarray) -> np.ndarray:
 
 def stamp_linear(X: np.ndarray, W: np.ndarray, bias: Optional[np.ndarray] = None, *, transform: int,
                  block: int = 0, levels: int = 0, k_hi: int = 64, bits_hi: int = 8, bits_lo: int = 4,
-                 bits_w: int = 4, grid_w: int = 0, want=("T", "x_scale", "q", "w_scale", "wq", "acc", "Yt", "Y")) -> Dict[str, np.ndarray]:
+                 bits_w: int = 4, grid_w: int = 0, asym: bool = False,
+                 want=("T", "x_scale", "q", "w_scale", "wq", "acc", "Yt", "Y")) -> Dict[str, np.ndarray]:
     """Run the whole layer; returns the stages named in `want`.
+
+    asym=True selects the zero-point activation quantizer: "q" is then uint8 and "x_zero" (int32 per
+    transformed token) is returned as well.
 
     X [B, L, K] float32 (values already rounded to the storage dtype), W [N, K] float32."""
     X = np.ascontiguousarray(X, dtype=np.float32)
@@ -170,7 +199,10 @@ def stamp_linear(X: np.ndarray, W: np.ndarray, bias: Optional[np.ndarray] = None
     M = B * L
     if bias is not None:
         bias = np.ascontiguousarray(bias, dtype=np.float32)
-    shapes = {"T": ((M, K), np.float64), "x_scale": ((M,), np.float32), "q": ((M, K), np.int8),
+    if asym and "x_scale" in want:
+        want = tuple(want) + ("x_zero",)
+    shapes = {"T": ((M, K), np.float64), "x_scale": ((M,), np.float32),
+              "q": ((M, K), np.uint8 if asym else np.int8), "x_zero": ((M,), np.int32),
               "w_scale": ((N,), np.float32), "wq": ((N, K), np.int8), "acc": ((M, N), np.int32),
               "Yt": ((M, N), np.float64), "Y": ((M, N), np.float64)}
     out = {k: np.empty(s, dtype=d) for k, (s, d) in shapes.items() if k in want}
@@ -178,6 +210,6 @@ def stamp_linear(X: np.ndarray, W: np.ndarray, bias: Optional[np.ndarray] = None
     rc = lib().oracle_stamp_linear(_p(X), _p(W), _p(bias), B, L, K, N, int(transform), int(block), int(levels),
                                    int(k_hi), int(bits_hi), int(bits_lo), int(bits_w), _p(g("T")),
                                    _p(g("x_scale")), _p(g("q")), _p(g("w_scale")), _p(g("wq")), _p(g("acc")),
-                                   _p(g("Yt")), _p(g("Y")), int(grid_w))
+                                   _p(g("Yt")), _p(g("Y")), int(grid_w), int(bool(asym)), _p(g("x_zero")))
     _check(rc, "stamp_linear")
     return out

@@ -499,3 +499,107 @@ def test_wht_layer_runs_blockwise(oracle):
     assert abs((out["T"] ** 2).sum() - (X.astype(np.float64) ** 2).sum()) <= 1e-10 * (X.astype(np.float64) ** 2).sum()
     ref = oracle.matmul_f64(X.reshape(-1, cfg.K), W)
     assert np.linalg.norm(out["Y"] - ref) / np.linalg.norm(ref) < 0.2
+
+
+# --------------------------------------------------------------------------------------
+# Zero-point (asymmetric) activation quantizer: Sec. 2.1, first equation as printed, min-max range
+# --------------------------------------------------------------------------------------
+
+def test_asym_quantizer_hand_case_and_constant_rows(oracle):
+    # 4 bits: range 3, s = 3/15 = 0.2, z = rne(1/0.2) = 5; x/s = -5, 0, 3, 10 (none near a tie)
+    T = np.array([[-1.0, 0.0, 0.6, 2.0],
+                  [0.0, 0.0, 0.0, 0.0],          # zero row: s = 1, z = 0, codes 0
+                  [3.0, 3.0, 3.0, 3.0]])         # constant row: s = 1, z = -3, codes 0, de-quantizes to 3
+    q, s, z = oracle.quantize_rows_asym(T, np.array([4], dtype=np.int32))
+    assert q.dtype == np.uint8 and s.dtype == np.float32 and z.dtype == np.int32
+    assert q[0].tolist() == [0, 5, 8, 15] and z[0] == 5 and s[0] == np.float32(3.0) / np.float32(15.0)
+    assert not q[1].any() and s[1] == 1.0 and z[1] == 0
+    assert not q[2].any() and s[2] == 1.0 and z[2] == -3
+    # integers -100 .. 155 at 8 bits: s = 1, z = 100, codes = value + 100, exact
+    T = np.arange(-100, 156, dtype=np.float64)[None, ::-1].copy()
+    q, s, z = oracle.quantize_rows_asym(T, np.array([8], dtype=np.int32))
+    assert s[0] == 1.0 and z[0] == 100 and np.array_equal(q[0].astype(int), T[0].astype(int) + 100)
+    # a row that does not straddle zero keeps an out-of-range zero point and still uses every code
+    T = np.linspace(10.0, 25.0, 16)[None, :]
+    q, s, z = oracle.quantize_rows_asym(T, np.array([4], dtype=np.int32))
+    assert z[0] == -10 and q[0].tolist() == list(range(16))
+
+
+def test_asym_quantizer_bound_and_nearest_level(oracle):
+    rng = np.random.default_rng(12)
+    rows, K = 48, 80
+    T = rng.standard_normal((rows, K)) * rng.lognormal(0, 1.5, size=(rows, 1)) + rng.standard_normal((rows, 1)) * 3
+    bits = np.where(np.arange(rows) < 10, 8, 4).astype(np.int32)
+    q, s, z = oracle.quantize_rows_asym(T, bits)
+    top = (2 ** bits - 1)
+    assert np.all(q.astype(int) <= top[:, None])
+    rng_row = T.max(axis=1) - T.min(axis=1)
+    assert np.allclose(s, rng_row / top, rtol=1e-6)                       # s = range / (2^b - 1)
+    assert np.all(np.abs(z + T.min(axis=1) / s) <= 0.5 + 1e-3)            # z = rne(-min / s)
+    # the minimum maps to code 0, the maximum to the top code (one below on a rounding coincidence)
+    assert np.all(q[np.arange(rows), T.argmin(axis=1)] == 0)
+    qtop = q[np.arange(rows), T.argmax(axis=1)].astype(int)
+    assert np.all(qtop >= top - 1) and np.mean(qtop == top) > 0.9
+    sd = s.astype(np.float64)[:, None]
+    deq = sd * (q.astype(np.float64) - z[:, None])
+    err = deq - T
+    # the section's bound: ||Q(x) - x||^2 <= d s^2 / 4 = d range^2 / (4 (2^b - 1)^2); the clamp of a top code
+    # that rounded one past the range costs at most one extra half step on that element
+    assert np.all(np.abs(err) <= sd * (0.5 + 1e-5) + sd * (q == top[:, None]) * 0.5)
+    e2 = np.sum(np.where(q == top[:, None], 0.0, err * err), axis=1)
+    assert np.all(e2 <= K * (rng_row / top) ** 2 / 4 * (1 + 1e-5))
+    # brute force: every code is the level nearest to its value among all 2^b levels
+    for r in range(rows):
+        levels = sd[r, 0] * (np.arange(top[r] + 1, dtype=np.float64) - z[r])
+        best = np.abs(T[r][:, None] - levels[None, :]).min(axis=1)
+        assert np.all(np.abs(err[r]) <= best * (1 + 1e-4) + 1e-6 * sd[r, 0])
+
+
+def test_asym_beats_symmetric_on_one_sided_rows(oracle):
+    # rows in [0, 1): the symmetric quantizer spends half its codes on values that never occur
+    rng = np.random.default_rng(13)
+    T = rng.random((16, 256))
+    bits = np.full(1, 4, dtype=np.int32)
+    qa, sa, za = oracle.quantize_rows_asym(T, bits)
+    qs, ss = oracle.quantize_rows(T, bits)
+    ea = np.sum((sa.astype(np.float64)[:, None] * (qa.astype(np.float64) - za[:, None]) - T) ** 2)
+    es = np.sum((ss.astype(np.float64)[:, None] * qs - T) ** 2)
+    assert ea < es / 3.5          # twice the resolution (15 steps over 1 vs 7): about 4.6x less squared error
+
+
+def test_asym_integer_product_equals_product_of_dequantized_operands(oracle):
+    rng = np.random.default_rng(14)
+    M, K, N = 24, 64, 20
+    T = rng.standard_normal((M, K)) + rng.standard_normal((M, 1)) * 2
+    bits = np.where(np.arange(M) < 4, 8, 4).astype(np.int32)
+    q, s, z = oracle.quantize_rows_asym(T, bits)
+    wq, sw = oracle.quantize_weights(rng.standard_normal((N, K)).astype(np.float32))
+    acc = oracle.gemm_zp_i32(q, z, wq)
+    Yt = oracle.dequant(acc, s, sw)
+    xhat = s.astype(np.float64)[:, None] * (q.astype(np.float64) - z[:, None])       # s (x_int - z)
+    what = sw.astype(np.float64)[:, None] * wq.astype(np.float64)
+    ref = xhat @ what.T
+    assert np.abs(Yt - ref).max() <= 1e-12 * np.abs(ref).max()
+    # and the sum splits into the plain code product minus z times the weight row sums
+    plain = q.astype(np.int64) @ wq.astype(np.int64).T
+    assert np.array_equal(acc, plain - z.astype(np.int64)[:, None] * wq.astype(np.int64).sum(axis=1)[None, :])
+
+
+def test_asym_layer_composes_and_is_closer_than_symmetric_on_shifted_activations(oracle):
+    cfg = gen.scaled(gen.config_llm_up(), B=1, L=256, K=128, N=96)
+    X, W = gen.make_activation(cfg), gen.make_weight(cfg)
+    X = (X + 0.75 * np.abs(X).mean()).astype(np.float32)       # a per-feature offset the transform concentrates in row 0
+    kw = dict(transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi)
+    out = oracle.stamp_linear(X, W, None, asym=True, **kw)
+    assert out["q"].dtype == np.uint8 and out["x_zero"].shape == (cfg.L,)
+    bits = oracle.bit_map(cfg.L, cfg.L, cfg.k_hi)
+    q, s, z = oracle.quantize_rows_asym(out["T"], bits)
+    assert np.array_equal(q, out["q"]) and np.array_equal(z, out["x_zero"]) and np.array_equal(s, out["x_scale"])
+    assert np.array_equal(out["acc"], oracle.gemm_zp_i32(q, z, out["wq"]))
+    Lm = oracle.transform_matrix(cfg.transform, cfg.L, cfg.levels)
+    assert np.abs(out["Y"] - Lm.T @ out["Yt"]).max() <= 1e-12 * np.abs(out["Y"]).max()
+    ref = oracle.matmul_f64(X.reshape(-1, cfg.K), W)
+    sym = oracle.stamp_linear(X, W, None, **kw, want=("Y",))
+    ea = np.linalg.norm(out["Y"] - ref) / np.linalg.norm(ref)
+    es = np.linalg.norm(sym["Y"] - ref) / np.linalg.norm(ref)
+    assert ea < es and ea < 0.2
