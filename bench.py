@@ -136,7 +136,7 @@ def cpu_oracle_sample(cfg, seconds_target=15.0):
     def run(ncol):
         Wc = gen.make_weight(cfg, np.arange(ncol))
         t0 = time.perf_counter()
-        orc.stamp_linear(X, Wc, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi, grid_w=cfg.grid,
+        orc.stamp_linear(X, Wc, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi, grid_w=cfg.grid, asym=cfg.zero_point,
                          want=("Y",))
         return time.perf_counter() - t0
     # two probes separate the fixed cost (transform + quantizer) from the per-channel cost (GEMM, inverse)
@@ -166,7 +166,7 @@ def run_reference(args, cfg):
     base, (X, W, ncols) = cpu_oracle_sample(cfg, seconds_target=8.0)
 
     def step():
-        orc.stamp_linear(X, W, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi, grid_w=cfg.grid,
+        orc.stamp_linear(X, W, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi, grid_w=cfg.grid, asym=cfg.zero_point,
                          want=("Y",))
     for _ in range(min(args.warmup, 1)):
         step()
@@ -224,7 +224,7 @@ def main():
     peaks = measured_peaks()
 
     # ---- inputs: generated on the host, resident in HBM before the timed region ----
-    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid)
+    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid, zero_point=cfg.zero_point)
     B, L, K, N, M = cfg.B, cfg.L, cfg.K, cfg.N, cfg.M
     x_t = torch.bfloat16 if cfg.dtype == gen.BF16 else torch.float32
     y_t = torch.bfloat16 if args.out_dtype == "bf16" else torch.float32

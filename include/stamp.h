@@ -88,6 +88,15 @@ typedef struct {
   int32_t act_gran;  /* STAMP_G_PER_TOKEN   (scales shared across features, Sec. 2.1)          */
   int32_t w_gran;    /* STAMP_G_PER_CHANNEL (one scale per output channel, Sec. "Set-up")      */
   int32_t grid_w;    /* STAMP_T_HAAR2D: width of the patch grid a block's tokens form; else 0  */
+  int32_t act_zero_point; /* 0: symmetric activation codes (zero point 0, range +-(2^(b-1) - 1)).
+                        1: the zero-point form Sec. 2.1's first equation prints, min-max range:
+                           s = (max_j t_j - min_j t_j) / (2^b - 1)  (1 for a constant row),
+                           z = rne(-min_j t_j / s),  x_int = clamp(rne(t / s) + z, 0, 2^b - 1).
+                           Codes are STORED as c = x_int - 2^(b-1) in the same signed byte / nibble
+                           formats as the symmetric ones, and the zero point handed out is that of
+                           the stored code, zc = z - 2^(b-1):  t ~ s * (c - zc).  Every transform is
+                           accepted; the layer then runs as separate transform, quantize, GEMM and
+                           inverse kernels.                                                       */
 } stamp_config;
 
 /* Bytes of scratch any call below may need for this problem size (the maximum over the calls). */
@@ -119,6 +128,8 @@ int stamp_prepare_weights(const stamp_config* cfg, const void* wq_packed, int N,
  *   q_lo     [B * (L-n_hi), K/2]  packed 4-bit codes of the remaining tokens in logical
  *            order (low nibble = even k)                                             out
  *   x_scale  [B, L]      float, per transformed token (logical order)                out
+ *            With cfg->act_zero_point = 1 the buffer holds 2 * B * L words: the B * L scales, then the
+ *            B * L zero points zc of the stored codes as int32.
  */
 int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, void* q_hi,
                    void* q_lo, float* x_scale, void* ws, size_t ws_bytes, void* stream);
@@ -128,6 +139,9 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
  *   Yt[m, n] = (sum_k q[m,k] * wq[n,k]) * x_scale[m] * w_scale[n],   int32 accumulation on the
  * tensor cores.  Output stays in the transformed token domain.
  *   q_hi, q_lo, x_scale : as written by stamp_quantize                               in
+ *            With cfg->act_zero_point = 1 (x_scale then carries the zero points zc as well)
+ *              Yt[m, n] = (sum_k c[m,k] * wq[n,k] - zc[m] * sum_k wq[n,k]) * x_scale[m] * w_scale[n],
+ *            the same sum over (c - zc) * wq with the constant term taken out of the product.
  *   w, w_format, w_scale: weight codes (stamp_weight_format) and per-channel scales  in
  *   Yt       [B, L, N]   float                                                       out
  */

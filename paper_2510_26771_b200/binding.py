@@ -29,14 +29,15 @@ EXPORTS = (
 
 class StampConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("transform", "block", "levels", "k_hi", "bits_hi", "bits_lo",
-                                              "bits_w", "act_gran", "w_gran", "grid_w")]
+                                              "bits_w", "act_gran", "w_gran", "grid_w", "act_zero_point")]
 
 
 def make_config(transform: int, block: int = 0, levels: int = 0, k_hi: int = 64, bits_hi: int = 8,
-                bits_lo: int = 4, bits_w: int = 4, grid_w: int = 0) -> StampConfig:
-    """grid_w: width of the patch grid for T_HAAR2D (0 for the other transforms)."""
+                bits_lo: int = 4, bits_w: int = 4, grid_w: int = 0, zero_point: bool = False) -> StampConfig:
+    """grid_w: width of the patch grid for T_HAAR2D (0 for the other transforms); zero_point: activation
+    codes with a per-token zero point and min-max range instead of the symmetric ones."""
     return StampConfig(transform, block, levels, k_hi, bits_hi, bits_lo, bits_w, G_PER_TOKEN, G_PER_CHANNEL,
-                       grid_w if transform == T_HAAR2D else 0)
+                       grid_w if transform == T_HAAR2D else 0, 1 if zero_point else 0)
 
 
 class StampError(RuntimeError):
@@ -132,11 +133,18 @@ def stamp_quantize(cfg: StampConfig, X: torch.Tensor, ws: torch.Tensor):
     nh = n_hi_rows(cfg, B, L)
     q_hi = torch.empty((max(nh, 1), K), dtype=torch.int8, device=X.device)
     q_lo = torch.empty((max(B * L - nh, 1), K // 2), dtype=torch.uint8, device=X.device)
-    x_scale = torch.empty((B, L), dtype=torch.float32, device=X.device)
+    # zero-point codes: the scales, then the zero points of the stored codes as int32 words (split_zero_points)
+    x_scale = torch.empty((2, B, L) if cfg.act_zero_point else (B, L), dtype=torch.float32, device=X.device)
     wp, wb = _ws_args(ws)
     _check(lib().stamp_quantize(ctypes.byref(cfg), _ptr(X), _dtype_code(X), B, L, K, _ptr(q_hi), _ptr(q_lo),
                                 _ptr(x_scale), wp, wb, _stream()), "stamp_quantize")
     return q_hi, q_lo, x_scale
+
+
+def split_zero_points(x_scale: torch.Tensor):
+    """The two halves of stamp_quantize's scale buffer in zero-point mode: scales [B, L] float32 and the zero
+    points of the stored codes [B, L] int32."""
+    return x_scale[0], x_scale[1].view(torch.int32)
 
 
 def stamp_linear(cfg: StampConfig, q_hi, q_lo, x_scale, w, w_format: int, w_scale, B: int, L: int, K: int, N: int,

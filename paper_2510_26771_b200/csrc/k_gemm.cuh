@@ -27,7 +27,8 @@
 
 namespace stamp {
 
-enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1, EPI_HAAR_F32 = 2, EPI_HAAR_BF16 = 3, EPI_DEQUANT_BF16X2 = 4 };
+enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1, EPI_HAAR_F32 = 2, EPI_HAAR_BF16 = 3, EPI_DEQUANT_BF16X2 = 4,
+                    EPI_DEQUANT_ZP_F32 = 5 };
 
 struct GemmParams {
   int n_out;               // output channels (MMA M extent)
@@ -45,6 +46,10 @@ struct GemmParams {
   const float* a8v;        // [m_tok / 256, n_out] level-8 approximation of every tile when the transform
                            // has more than 8 levels (orthonormal scaling), else nullptr
   const float* bias;       // [n_out] or nullptr
+  // EPI_DEQUANT_ZP_F32: zero-point codes (Sec. 2.1, first equation):  out = (acc - x_zero[tok] * w_sum[ch])
+  // * x_scale[tok] * w_scale[ch], the bracket in 64-bit integers
+  const int* x_zero;       // [m_tok] zero point of every token's stored codes
+  const int* w_sum;        // [n_out] sum over k of the weight codes of a channel
 };
 
 constexpr int GEMM_BM = 128;           // output channels per tile
@@ -62,7 +67,8 @@ struct GemmSmem {
   // full[STAGES], empty[STAGES], tfull[2], tempty[2], then tmem base + abort word
   static constexpr int NUM_BARS = 2 * STAGES + 4;
   static constexpr int SX_OFFSET = BAR_OFFSET + NUM_BARS * 8 + 16;  // token scales of the tile being drained
-  static constexpr int TOTAL = SX_OFFSET + 2 * BN * 4;   // one buffer per accumulator
+  static constexpr int ZP_OFFSET = SX_OFFSET + 2 * BN * 4;  // token zero points, same arrangement
+  static constexpr int TOTAL = ZP_OFFSET + 2 * BN * 4;   // one buffer per accumulator
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for 1024-byte alignment of the ring
 };
 
@@ -91,6 +97,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile uint32_t* abort_word = tmem_slot + 1;
   float* sx_stage = reinterpret_cast<float*>(smem + SM::SX_OFFSET);
+  int* zp_stage = reinterpret_cast<int*>(smem + SM::ZP_OFFSET);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -225,11 +232,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       const bool full_tile = (tok0 + BN <= p.m_tok);
       float* sxs = sx_stage + a * BN;
       float sw = 0.f;
+      int* zps = zp_stage + a * BN;
       float my_sx = 0.f;
+      int my_zp = 0, wsum = 0;
       if (EPI != EPI_RAW_I32) {
         if (ch_ok) sw = p.w_scale ? __ldg(p.w_scale + ch) : 1.0f;
         // fetch this tile's token scales while the accumulator is still being filled
-        if (ep_tid < BN && tok0 + ep_tid < p.m_tok) my_sx = __ldg(p.x_scale + tok0 + ep_tid);
+        if (ep_tid < BN && tok0 + ep_tid < p.m_tok) {
+          my_sx = __ldg(p.x_scale + tok0 + ep_tid);
+          if (EPI == EPI_DEQUANT_ZP_F32) my_zp = __ldg(p.x_zero + tok0 + ep_tid);
+        }
+        if (EPI == EPI_DEQUANT_ZP_F32 && ch_ok) wsum = __ldg(p.w_sum + ch);
       }
       // The eight epilogue warps continue or stop TOGETHER: a warp whose wait ran out raises the abort
       // word, and everybody reads it behind the named barrier below -- no warp is left waiting at that
@@ -240,7 +253,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       if (EPI != EPI_RAW_I32) {
         // every epilogue thread has finished the previous tile that used accumulator `a` (all of
         // them arrived on tempty[a] before tfull[a] could complete again), so its staging buffer is free
-        if (ep_tid < BN) sxs[ep_tid] = my_sx;
+        if (ep_tid < BN) {
+          sxs[ep_tid] = my_sx;
+          if (EPI == EPI_DEQUANT_ZP_F32) zps[ep_tid] = my_zp;
+        }
       }
       asm volatile("bar.sync 1, %0;" ::"n"(GEMM_EPI_THREADS) : "memory");
       if (*abort_word != 0u) {
@@ -347,6 +363,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
               if (tbase + j < p.m_tok && ch_ok)
                 out[(long)j * p.n_out] = static_cast<float>(static_cast<int>(rc[j])) * sxs[chunk * 32 + j] * sw;
           }
+        } else if (EPI == EPI_DEQUANT_ZP_F32) {
+          float* out = static_cast<float*>(p.out) + (long)tbase * p.n_out + ch;
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (tbase + j < p.m_tok && ch_ok) {
+              const long long v = static_cast<long long>(static_cast<int>(rc[j])) -
+                                  static_cast<long long>(zps[chunk * 32 + j]) * wsum;
+              out[(long)j * p.n_out] = __ll2float_rn(v) * sxs[chunk * 32 + j] * sw;
+            }
         } else if (EPI == EPI_DEQUANT_BF16X2) {
           __nv_bfloat16* hi = static_cast<__nv_bfloat16*>(p.out) + (long)tbase * p.n_out + ch;
           __nv_bfloat16* lo = hi + (long)p.m_tok * p.n_out;

@@ -204,6 +204,92 @@ __global__ void __launch_bounds__(256) k_quant_rows(const float* __restrict__ T,
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Row quantizer in the zero-point form the first equation of Sec. 2.1 prints, min-max range:
+//   s = (max - min) / (2^b - 1)  (1 when the row is constant),  z = rne(-min / s),
+//   x_int = clamp(rne(t / s) + z, 0, 2^b - 1).
+// Codes are STORED offset by half the code range, c = x_int - 2^(b-1), so that they use the same
+// signed byte / nibble formats (and the same signed tensor-core operand) as the symmetric codes; the
+// zero point written out is that of the stored code, zc = z - 2^(b-1), and t ~ s * (c - zc).
+// One CTA per materialised row; the row is read twice (min/max, then codes), the second time from L2.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_quant_rows_zp(const float* __restrict__ T, int K, int n, int k_hi,
+                                                       int8_t* __restrict__ a8, int8_t* __restrict__ q_hi,
+                                                       uint8_t* __restrict__ q_lo, float* __restrict__ x_scale,
+                                                       int* __restrict__ x_zero) {
+  __shared__ float red_mn[8], red_mx[8];
+  const long r = blockIdx.x;
+  const long s = r / n;
+  const int i = static_cast<int>(r - s * n);
+  const bool hi = i < k_hi;
+  const int half = hi ? 128 : 8;
+  const int top = 2 * half - 1;
+  const float4* src = reinterpret_cast<const float4*>(T + r * (long)K);
+  float mn = __int_as_float(0x7f800000), mx = -mn;
+  for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) {
+    const float4 t = src[k4];
+    mn = fminf(fminf(mn, t.x), fminf(t.y, fminf(t.z, t.w)));
+    mx = fmaxf(fmaxf(mx, t.x), fmaxf(t.y, fmaxf(t.z, t.w)));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  if ((threadIdx.x & 31) == 0) {
+    red_mn[threadIdx.x >> 5] = mn;
+    red_mx[threadIdx.x >> 5] = mx;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    mn = fminf(mn, red_mn[w]);
+    mx = fmaxf(mx, red_mx[w]);
+  }
+  float scale = __fdiv_rn(mx - mn, static_cast<float>(top));
+  if (!(scale > 0.f)) scale = 1.0f;
+  const float inv = __fdiv_rn(1.0f, scale);
+  float zf = rintf(__fdiv_rn(-mn, scale));
+  zf = fminf(fmaxf(zf, -1073741824.0f), 1073741824.0f);
+  const int z = static_cast<int>(zf);
+  if (threadIdx.x == 0) {
+    x_scale[r] = scale;
+    x_zero[r] = z - half;
+  }
+  char4* dst8 = a8 ? reinterpret_cast<char4*>(a8 + r * (long)K) : nullptr;
+  char4* dsth = (q_hi && hi) ? reinterpret_cast<char4*>(q_hi + (s * k_hi + i) * (long)K) : nullptr;
+  uint16_t* dstl =
+      (q_lo && !hi) ? reinterpret_cast<uint16_t*>(q_lo + (s * (n - k_hi) + (i - k_hi)) * (long)(K / 2)) : nullptr;
+  for (int k4 = threadIdx.x; k4 < K / 4; k4 += blockDim.x) {
+    const float4 t = src[k4];
+    int q0 = __float2int_rn(div_by_scale(t.x, scale, inv)) + z, q1 = __float2int_rn(div_by_scale(t.y, scale, inv)) + z;
+    int q2 = __float2int_rn(div_by_scale(t.z, scale, inv)) + z, q3 = __float2int_rn(div_by_scale(t.w, scale, inv)) + z;
+    q0 = max(0, min(top, q0)) - half;
+    q1 = max(0, min(top, q1)) - half;
+    q2 = max(0, min(top, q2)) - half;
+    q3 = max(0, min(top, q3)) - half;
+    const char4 c = make_char4((signed char)q0, (signed char)q1, (signed char)q2, (signed char)q3);
+    if (dst8) dst8[k4] = c;
+    if (dsth) dsth[k4] = c;
+    if (dstl)
+      dstl[k4] = static_cast<uint16_t>((q0 & 0xF) | ((q1 & 0xF) << 4) | ((q2 & 0xF) << 8) | ((q3 & 0xF) << 12));
+  }
+}
+
+// Sum of every row of an int8 matrix [rows, K] (the weight row sums of the zero-point correction
+//   sum_k (c - zc) w = sum_k c w  -  zc * sum_k w).  One warp per row.
+__global__ void __launch_bounds__(256) k_row_sums_i8(const int8_t* __restrict__ w8, int rows, int K,
+                                                     int* __restrict__ out) {
+  const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const int* src = reinterpret_cast<const int*>(w8 + (long)r * K);
+  int acc = 0;
+  for (int k4 = threadIdx.x & 31; k4 < K / 4; k4 += 32) acc = __dp4a(src[k4], 0x01010101, acc);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) out[r] = acc;
+}
+
 // Sign-extend the two nibbles of a byte.
 __device__ __forceinline__ int nib_lo(uint32_t b) { return (static_cast<int>(b << 28)) >> 28; }
 __device__ __forceinline__ int nib_hi(uint32_t b) { return (static_cast<int>(b << 24)) >> 28; }

@@ -46,6 +46,7 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
   if (cfg->transform != STAMP_T_HAAR2D && cfg->grid_w != 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->bits_hi != 8 || cfg->bits_lo != 4 || cfg->bits_w != 4) return STAMP_ERR_UNSUPPORTED;
   if (cfg->act_gran != STAMP_G_PER_TOKEN || cfg->w_gran != STAMP_G_PER_CHANNEL) return STAMP_ERR_UNSUPPORTED;
+  if (cfg->act_zero_point != 0 && cfg->act_zero_point != 1) return STAMP_ERR_INVALID_ARG;
   const int n = cfg->block ? cfg->block : L;
   if (!is_pow2(n) || L % n != 0) return STAMP_ERR_UNSUPPORTED;
   if (cfg->k_hi > n) return STAMP_ERR_INVALID_ARG;
@@ -76,6 +77,7 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
   out->levels = levels;
   out->k_hi = cfg->k_hi;
   out->grid_w = cfg->grid_w;
+  out->act_zp = cfg->act_zero_point;
   out->nseq = B * (L / n);
   out->M = (long)B * L;
   out->qmax_hi = (1 << (cfg->bits_hi - 1)) - 1;
@@ -113,7 +115,7 @@ static PassPlan make_plan(int levels) {
 // Workspace layout (one layout for all calls of a problem size).
 // ------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, dctsplit, total;
+  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, dctsplit, xzero, wsum, total;
 };
 static Workspace layout(const Problem& pb) {
   Workspace w{};
@@ -147,6 +149,9 @@ static Workspace layout(const Problem& pb) {
   w.a8v = off;    off += align256((M >> 8) * (size_t)pb.N * 4);
   // bf16 terms of the DCT matrix and of its transpose (tensor-core DCT)
   w.dctsplit = off; off += align256(dense ? (size_t)2 * 3 * DCT_N * DCT_N * 2 : 0);
+  // zero-point activation codes: per-token zero points and the weight row sums of the correction term
+  w.xzero = off;  off += align256(pb.act_zp ? M * 4 : 0);
+  w.wsum = off;   off += align256(pb.act_zp ? (size_t)pb.N * 4 : 0);
   w.total = off;
   return w;
 }
@@ -281,7 +286,8 @@ static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const Gem
 // acc/out[tok, ch] from int8 operands a8 [M, K], w8 [N, K].
 static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K, const float* x_scale,
                        const float* w_scale, void* out, int epi, cudaStream_t st, const float* bias = nullptr,
-                       const float* a8v = nullptr, int depth = 0) {
+                       const float* a8v = nullptr, int depth = 0, const int* x_zero = nullptr,
+                       const int* w_sum = nullptr) {
   GemmParams gp{};
   gp.n_out = N;
   gp.m_tok = (int)M;
@@ -293,6 +299,8 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
   gp.bias = bias;
   gp.a8v = a8v;
   gp.depth = depth;
+  gp.x_zero = x_zero;
+  gp.w_sum = w_sum;
   CUtensorMap tw, tx;
   int rc = make_tmap_i8(w8, N, K, GEMM_BM, &tw);
   if (rc) return rc;
@@ -307,6 +315,11 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
   if (epi == EPI_DEQUANT_BF16X2)
     return wide ? launch_gemm_t<256, 4, EPI_DEQUANT_BF16X2>(tw, tx, gp, st)
                 : launch_gemm_t<128, 6, EPI_DEQUANT_BF16X2>(tw, tx, gp, st);
+  if (epi == EPI_DEQUANT_ZP_F32) {
+    if (!x_zero || !w_sum) return STAMP_ERR_INVALID_ARG;
+    return wide ? launch_gemm_t<256, 4, EPI_DEQUANT_ZP_F32>(tw, tx, gp, st)
+                : launch_gemm_t<128, 6, EPI_DEQUANT_ZP_F32>(tw, tx, gp, st);
+  }
   if (wide) {
     if (epi == EPI_DEQUANT_F32) return launch_gemm_t<256, 4, EPI_DEQUANT_F32>(tw, tx, gp, st);
     return launch_gemm_t<256, 4, EPI_RAW_I32>(tw, tx, gp, st);
@@ -498,6 +511,21 @@ static int run_quant_rows(const Problem& pb, const float* T, const unsigned* row
   const long rows = (long)pb.nseq * n_src;
   k_quant_rows<<<(unsigned)rows, 256, 0, st>>>(T, rowmax, pb.K, n_src, pb.n, pb.k_hi, pb.qmax_hi, pb.qmax_lo, a8,
                                                static_cast<int8_t*>(q_hi), static_cast<uint8_t*>(q_lo), x_scale);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// Zero-point codes from materialised T (all rows of every block).
+static int run_quant_rows_zp(const Problem& pb, const float* T, int8_t* a8, void* q_hi, void* q_lo, float* x_scale,
+                             int* x_zero, cudaStream_t st) {
+  k_quant_rows_zp<<<(unsigned)pb.M, 256, 0, st>>>(T, pb.K, pb.n, pb.k_hi, a8, static_cast<int8_t*>(q_hi),
+                                                   static_cast<uint8_t*>(q_lo), x_scale, x_zero);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+static int run_weight_row_sums(const int8_t* w8, int N, int K, int* w_sum, cudaStream_t st) {
+  k_row_sums_i8<<<(unsigned)((N + 7) / 8), 256, 0, st>>>(w8, N, K, w_sum);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
 }
@@ -878,6 +906,12 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   uint8_t* base = static_cast<uint8_t*>(ws);
   float* T = reinterpret_cast<float*>(base + w.T);
   unsigned* rowmax = reinterpret_cast<unsigned*>(base + w.rowmax);
+  if (pb.act_zp) {
+    rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
+                               reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st);
+    if (rc) return rc;
+    return run_quant_rows_zp(pb, T, nullptr, q_hi, q_lo, x_scale, reinterpret_cast<int*>(x_scale + pb.M), st);
+  }
   CqChoice cc;
   if ((pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc))
     return run_quantize_cq(pb, cc, X, x_dtype, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
@@ -912,6 +946,12 @@ int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, co
   if ((rc = run_unpack_codes(pb, q_hi, q_lo, a8, st))) return rc;
   const int8_t* w8 = nullptr;
   if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
+  if (pb.act_zp) {
+    int* w_sum = reinterpret_cast<int*>(base + wl.wsum);
+    if ((rc = run_weight_row_sums(w8, N, K, w_sum, st))) return rc;
+    return launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, Yt, EPI_DEQUANT_ZP_F32, st, nullptr, nullptr, 0,
+                       reinterpret_cast<const int*>(x_scale + pb.M), w_sum);
+  }
   return launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, Yt, EPI_DEQUANT_F32, st);
 }
 
@@ -971,6 +1011,21 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
   float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
   float* yt = reinterpret_cast<float*>(base + wl.yt);
+  if (pb.act_zp) {
+    // zero-point codes: transform, min-max quantizer, GEMM with the zero-point term in its epilogue, inverse
+    int* x_zero = reinterpret_cast<int*>(base + wl.xzero);
+    int* w_sum = reinterpret_cast<int*>(base + wl.wsum);
+    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
+      return rc;
+    if ((rc = run_quant_rows_zp(pb, T, a8, nullptr, nullptr, x_scale, x_zero, st))) return rc;
+    const int8_t* w8z = nullptr;
+    if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8z, st))) return rc;
+    if ((rc = run_weight_row_sums(w8z, N, K, w_sum, st))) return rc;
+    if ((rc = launch_gemm(a8, w8z, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_ZP_F32, st, nullptr, nullptr, 0, x_zero,
+                          w_sum)))
+      return rc;
+    return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
+  }
   CqChoice cc;
   const bool have_cq = (pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc);
   if (have_cq && pb.transform == STAMP_T_HAAR && pb.levels >= 5 && pb.n % 256 == 0) {

@@ -49,6 +49,7 @@ class LayerConfig:
     w_std: float = 0.02
     grid: int = 0              # patch-grid side for the GRF recipe
     length_scale: float = 8.0
+    zero_point: bool = False   # activation codes with a per-token zero point (min-max range)
 
     @property
     def M(self) -> int:
@@ -194,6 +195,11 @@ def config_llm_down_wht() -> LayerConfig:
     return dataclasses.replace(config_llm_down(), name="llm_down_proj_wht", transform=T_WHT)
 
 
+def config_llm_up_zp() -> LayerConfig:
+    """The MLP up-projection workload with zero-point (asymmetric, min-max) activation codes."""
+    return dataclasses.replace(config_llm_up(), name="llm_mlp_up_zp", zero_point=True)
+
+
 def config_dit_proj_2d() -> LayerConfig:
     """The DiT projection with the paper's own LVM transform: 3-level 2-D Haar over the 64 x 64 patch grid,
     whose 64 low-pass tokens are the 8-bit ones."""
@@ -218,7 +224,8 @@ def config_sweep(L: int, D: int, levels: int = 0) -> LayerConfig:
 
 
 def named_configs() -> dict:
-    return {c.name: c for c in (config_tiny(), config_llm_up(), config_dit_proj(), config_llm_down(), config_dit_proj_2d(), config_llm_down_wht())}
+    return {c.name: c for c in (config_tiny(), config_llm_up(), config_dit_proj(), config_llm_down(), config_dit_proj_2d(), config_llm_down_wht(),
+                                config_llm_up_zp())}
 
 
 def scaled(cfg: LayerConfig, **kw) -> LayerConfig:

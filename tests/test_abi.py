@@ -36,7 +36,11 @@ def test_status_strings(st):
 
 
 def test_config_struct_matches_header(st):
-    assert ctypes.sizeof(st.StampConfig) == 40
+    assert ctypes.sizeof(st.StampConfig) == 44      # eleven int32 fields
+    header = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "stamp.h")).read()
+    body = header[header.index("typedef struct {"):header.index("} stamp_config;")]
+    names = re.findall(r"int32_t\s+(\w+);", body)
+    assert names == [n for n, _ in st.StampConfig._fields_]
 
 
 def test_host_side_validation(st):

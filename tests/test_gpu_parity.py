@@ -150,6 +150,107 @@ def test_stagewise_parity(st, oracle, name):
     assert st.stamp_last_device_status() == 0
 
 
+ZP_CASES = {
+    # full-depth Haar with ragged tiles, blockwise DCT and Walsh-Hadamard, the patch-grid Haar, no transform
+    "zp_haar": gen.scaled(gen.config_llm_up(), B=2, L=512, K=384, N=392, k_hi=16),
+    "zp_haar_fp32_blocks": gen.scaled(gen.config_tiny(), B=1, L=256, K=128, N=72, block=64, levels=3, k_hi=8),
+    "zp_dct": gen.scaled(gen.config_llm_down(), B=1, L=512, K=256, N=136),
+    "zp_wht": gen.scaled(gen.config_llm_down_wht(), B=1, L=256, K=128, N=64, block=64, k_hi=4),
+    "zp_haar2d": gen.scaled(gen.config_dit_proj_2d(), B=1, L=1024, K=256, N=128, grid=32, levels=3, k_hi=16),
+    "zp_identity": gen.scaled(gen.config_sweep(512, 2048), L=256, K=256, N=128, transform=gen.T_IDENTITY, k_hi=8),
+}
+
+
+@pytest.mark.parametrize("name", list(ZP_CASES))
+def test_zero_point_stagewise_parity(st, oracle, name):
+    """Zero-point activation codes (Sec. 2.1, first equation, min-max range) against the oracle.  The library
+    stores codes and zero points offset by half the code range; the oracle keeps the unsigned ones."""
+    import torch
+    cfg = ZP_CASES[name]
+    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid, zero_point=True)
+    X, W, bias = gen.make_activation(cfg), gen.make_weight(cfg), gen.make_bias(cfg)
+    # a per-feature offset, so that rows (above all the low-pass ones) are far from symmetric about zero
+    X = gen.round_to_bf16((X + 0.5 * np.abs(X).mean()).astype(np.float32)) if cfg.dtype == 1 else (X + 0.5).astype(np.float32)
+    ref = oracle.stamp_linear(X, W, bias, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi,
+                              grid_w=cfg.grid, asym=True)
+    B, L, K, N = cfg.B, cfg.L, cfg.K, cfg.N
+    M = B * L
+    Xd, Wd = H.to_device(X, cfg.dtype), H.to_device(W, cfg.dtype)
+    bd = torch.from_numpy(bias).cuda()
+    ws = st.alloc_workspace(c, B, L, K, N)
+    half = np.where((np.arange(M) % cfg.block_len) < cfg.k_hi, 128, 8).astype(np.int64)
+
+    # scales, zero points, codes
+    q_hi, q_lo, xbuf = st.stamp_quantize(c, Xd, ws)
+    xs, zc = st.split_zero_points(xbuf)
+    xs, zc = xs.cpu().numpy().reshape(-1), zc.cpu().numpy().reshape(-1).astype(np.int64)
+    codes = st.stamp_debug_unpack_codes(c, q_hi, q_lo, B, L, K).cpu().numpy().reshape(-1, K).astype(np.int64)
+    assert np.allclose(xs, ref["x_scale"], rtol=2 * _scale_rtol(cfg), atol=0)
+    dz = zc + half - ref["x_zero"]
+    # a zero point is a rounded quotient: within fp32 error of a tie it may come out one off, and the row's
+    # codes move with it -- compare such rows through the centred codes c - zc = x_int - z
+    assert np.abs(dz).max() <= 1 and np.count_nonzero(dz) <= max(1, M // 100), (np.abs(dz).max(), np.count_nonzero(dz))
+    same = dz == 0
+    bad, worst = H.code_mismatch((codes + half[:, None])[same], ref["q"][same].astype(np.int64))
+    print(f"[{name}] zero-point code mismatches: {bad} of {codes.size} (max |diff| {worst}); rows with z off by one: "
+          f"{np.count_nonzero(dz)}")
+    assert worst <= 1 and bad <= _allowed(codes.size), (bad, worst, codes.size)
+    centred = codes - zc[:, None]
+    centred_ref = ref["q"].astype(np.int64) - ref["x_zero"].astype(np.int64)[:, None]
+    assert np.abs(centred - centred_ref).max() <= 1
+    assert codes.min() >= -128 and codes.max() <= 127 and np.all(np.abs(codes[half == 8]) <= 8)
+
+    # integer GEMM on the oracle's codes in the stored (offset) form: the plain code product, bit-identical
+    oc = (ref["q"].astype(np.int64) - half[:, None]).astype(np.int8)
+    ozc = (ref["x_zero"].astype(np.int64) - half).astype(np.int32)
+    oq_hi, oq_lo = H.pack_codes(oc, cfg.block_len, cfg.k_hi)
+    oqh, oql = torch.from_numpy(oq_hi).cuda(), torch.from_numpy(oq_lo).cuda()
+    ow8 = torch.from_numpy(ref["wq"]).cuda()
+    acc = st.stamp_debug_gemm_i32(c, oqh, oql, ow8, st.W_INT8, B, L, K, N, ws).cpu().numpy()
+    assert np.array_equal(acc, oracle.gemm_i32(oc, ref["wq"]))
+
+    # de-quantized transformed-domain output with the zero-point term, from the oracle's codes, scales, zero points
+    oxbuf = torch.empty((2, B, L), dtype=torch.float32, device="cuda")
+    oxbuf[0].copy_(torch.from_numpy(ref["x_scale"]).reshape(B, L))
+    oxbuf[1].view(torch.int32).copy_(torch.from_numpy(ozc).reshape(B, L))
+    ows = torch.from_numpy(ref["w_scale"]).cuda()
+    owq = torch.from_numpy(H.pack_nibbles(ref["wq"])).cuda()
+    for wfmt, wbuf in ((st.W_PACKED4, owq), (st.W_INT8, ow8)):
+        Yt = st.stamp_linear(c, oqh, oql, oxbuf, wbuf, wfmt, ows, B, L, K, N, ws).cpu().numpy().reshape(-1, N)
+        assert H.rel_fro(Yt, ref["Yt"]) <= 1e-6
+
+    # whole layer: chained calls and the one-call form
+    wq, wsc = st.stamp_quantize_weights(c, Wd)
+    w8 = st.stamp_prepare_weights(c, wq)
+    Yt2 = st.stamp_linear(c, q_hi, q_lo, xbuf, wq, st.W_PACKED4, wsc, B, L, K, N, ws)
+    Y2 = st.stamp_inverse(c, Yt2, bd, ws).cpu().numpy().reshape(-1, N)
+    assert H.rel_fro(Y2, ref["Y"]) <= Y_TOL
+    for wfmt, wbuf in ((st.W_PACKED4, wq), (st.W_INT8, w8)):
+        Y3 = st.stamp_linear_fused(c, Xd, wbuf, wfmt, wsc, bd, ws).cpu().numpy().reshape(-1, N)
+        assert H.rel_fro(Y3, ref["Y"]) <= Y_TOL
+    assert st.stamp_last_device_status() == 0
+    # what the zero point buys on these one-sided rows: closer to the unquantized product than symmetric codes
+    plain = oracle.matmul_f64(X.reshape(-1, K), W) + bias[None, :]
+    sym = _oracle_all(oracle, cfg, X, W, bias, want=("Y",))["Y"]
+    assert H.rel_fro(Y3, plain) < H.rel_fro(sym, plain)
+
+
+def test_zero_point_constant_and_zero_rows(st):
+    """No transform, rows that are constant: scale 1, stored code -2^(b-1) everywhere, zero point -rne(value) - 2^(b-1)."""
+    import torch
+    c = st.make_config(st.T_IDENTITY, 0, 0, 2, zero_point=True)
+    ws = st.alloc_workspace(c, 1, 4, 128, 8)
+    X = torch.zeros((1, 4, 128), device="cuda")
+    X[0, 1] = 3.0
+    X[0, 3] = -2.0
+    q_hi, q_lo, xbuf = st.stamp_quantize(c, X, ws)
+    xs, zc = st.split_zero_points(xbuf)
+    codes = st.stamp_debug_unpack_codes(c, q_hi, q_lo, 1, 4, 128).cpu().numpy().reshape(4, 128)
+    assert torch.all(xs == 1.0)
+    assert zc.cpu().numpy().reshape(-1).tolist() == [-128, -3 - 128, -8, 2 - 8]
+    assert np.all(codes[:2] == -128) and np.all(codes[2:] == -8)
+
+
 def test_transform_then_inverse_is_identity(st):
     """Quantizers off: L^T (L X) = X on the device (uses the activation as its own 'output')."""
     import torch
