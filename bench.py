@@ -35,7 +35,7 @@ FALLBACK_BF16_TFLOPS = 1590.0
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None until
 # a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {"llm_mlp_up": 54303232 + 13345280}   # profiles/k_gemm_i8_haar_epilogue_llm_mlp_up.txt
+NCU_TRAFFIC_BYTES = {"llm_mlp_up": 54400000 + 14459392}   # profiles/k_gemm_i8_haar_epilogue_llm_mlp_up.txt
 
 
 def workloads():
@@ -149,7 +149,7 @@ def cpu_oracle_sample(cfg, seconds_target=15.0):
     W = gen.make_weight(cfg, np.arange(ncols))
     t0 = time.perf_counter()
     orc.stamp_linear(X, W, None, transform=cfg.transform, block=cfg.block, levels=cfg.levels, k_hi=cfg.k_hi,
-                     want=("Y",))
+                     grid_w=cfg.grid, asym=cfg.zero_point, want=("Y",))
     dt = time.perf_counter() - t0
     tops = 2.0 * cfg.M * ncols * cfg.K / dt / 1e12
     return {"value": tops, "unit": "TOPS", "cores": orc.num_threads(), "kind": "oracle",
@@ -357,16 +357,37 @@ def main():
         pass
 
     # ---- end to end: host buffers, copies inside the timed region, through the C ABI ----
-    ws_h = torch.empty(st.stamp_workspace_bytes_host(c, B, L, K, N, st._dtype_code(X_host), 1 if y_t == torch.bfloat16 else 0),
-                       dtype=torch.uint8, device="cuda")
-    Y_host = torch.empty((B, L, N), dtype=y_t).pin_memory()
-    e2e_steps = max(5, min(steps, 100))
+    # Two calls are kept in flight, on two streams with a workspace and a pinned result buffer each, so that
+    # one step's result copy (device to host) overlaps the next step's input copy (host to device): the link is
+    # full duplex.  Every step still copies its X in and its Y out inside the timed region.
+    ws_bytes_h = st.stamp_workspace_bytes_host(c, B, L, K, N, st._dtype_code(X_host), 1 if y_t == torch.bfloat16 else 0)
+    lanes = [(torch.cuda.Stream(), torch.empty(ws_bytes_h, dtype=torch.uint8, device="cuda"),
+              torch.empty((B, L, N), dtype=y_t).pin_memory()) for _ in range(2)]
+    e2e_steps = max(6, min(steps, 100))
 
-    def e2e_step(i):
-        st.stamp_linear_fused_host(c, X_host, Ws[i % n_w], st.W_INT8, w_scale, bias, Y_host, ws_h)
-    e2e_ms = time_loop(e2e_step, e2e_steps)
+    def e2e_loop(iters):
+        main = torch.cuda.current_stream()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(main)
+        for lane in lanes:
+            lane[0].wait_event(a)
+        for i in range(iters):
+            stream, ws_h, Y_host = lanes[i % 2]
+            with torch.cuda.stream(stream):
+                st.stamp_linear_fused_host(c, X_host, Ws[i % n_w], st.W_INT8, w_scale, bias, Y_host, ws_h)
+        for lane in lanes:
+            done = torch.cuda.Event()
+            done.record(lane[0])
+            main.wait_event(done)
+        b.record(main)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters
+
+    e2e_loop(4)
+    e2e_ms = e2e_loop(e2e_steps)
     e2e = {"value": ops / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": x_bytes,
-           "d2h_bytes_per_step": y_bytes, "ms_per_step": e2e_ms}
+           "d2h_bytes_per_step": y_bytes, "ms_per_step": e2e_ms, "in_flight": 2}
+    del lanes
 
     i8_peak = peaks["bf16_sustained"] * NOMINAL_I8_OVER_BF16
     gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
