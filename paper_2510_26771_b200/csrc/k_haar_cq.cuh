@@ -53,6 +53,10 @@ struct CqParams {
   long a8_top_row;  // codes of the rows of levels > 8 (logical order inside a block) go to rows a8_top_row + i of a8
   float* sx_top;    // [M / 256]    their scales
   float* sx_epi;    // [M]          scale * 2^(-j/2) of every tile row, indexed like a8
+  // Optional: a region (the layer's weight codes) to pull towards L2 while this launch and the small
+  // launches after it leave HBM idle; the kernels that follow read it from there.  pf_bytes % 16 == 0.
+  const uint8_t* pf_base;
+  long pf_bytes;
 };
 
 constexpr float CQ_MAGIC = 12582912.0f;            // 1.5 * 2^23
@@ -149,6 +153,15 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
   }
   // every CTA of the cluster has initialised its barriers before anyone posts to them
   ptx::cluster_sync();
+  if (p.pf_bytes > 0 && tid >= 480) {   // the last warp: fire-and-forget hints, 8 KB each
+    constexpr long PF_CHUNK = 8192;
+    const long nchunk = (p.pf_bytes + PF_CHUNK - 1) / PF_CHUNK;
+    for (long c = (long)blockIdx.x * 32 + lane; c < nchunk; c += (long)gridDim.x * 32) {
+      const long off = c * PF_CHUNK;
+      const long left = p.pf_bytes - off;
+      ptx::prefetch_l2_bulk(p.pf_base + off, static_cast<uint32_t>(left < PF_CHUNK ? left : PF_CHUNK));
+    }
+  }
   ptx::grid_dependency_wait();   // the input rows may come from the previous launch
 
   // warp 0 brings one group's rows of this strip into a ring stage: lane r copies token row r

@@ -217,6 +217,11 @@ __host__ __device__ constexpr uint32_t make_i8_idesc(int m, int n) {
 // Blocks until the grids this one depends on have completed and their writes are visible.  A no-op
 // for a launch without the programmatic-serialization attribute.  Everything before it (barrier
 // set-up, TMEM allocation) may overlap the tail of the previous kernel.
+// Hint: bring `bytes` (a multiple of 16, 16-byte aligned start) of global memory into L2; nothing waits on it.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* gptr, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
+}
+
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ---------------------------------------------------------------- clusters
