@@ -28,7 +28,7 @@
 namespace stamp {
 
 enum GemmEpilogue { EPI_DEQUANT_F32 = 0, EPI_RAW_I32 = 1, EPI_HAAR_F32 = 2, EPI_HAAR_BF16 = 3, EPI_DEQUANT_BF16X2 = 4,
-                    EPI_DEQUANT_ZP_F32 = 5 };
+                    EPI_DEQUANT_ZP_F32 = 5, EPI_HAAR2D_F32 = 6, EPI_HAAR2D_BF16 = 7 };
 
 struct GemmParams {
   int n_out;               // output channels (MMA M extent)
@@ -50,6 +50,12 @@ struct GemmParams {
   // * x_scale[tok] * w_scale[ch], the bracket in 64-bit integers
   const int* x_zero;       // [m_tok] zero point of every token's stored codes
   const int* w_sum;        // [n_out] sum over k of the weight codes of a channel
+  // EPI_HAAR2D_*: the token operand is in the patch order of the 2-D Haar quantize kernel (64 consecutive rows
+  // = the coefficients of one 8 x 8 patch of the token grid in synthesis order), x_scale holds scale * 2^-l, and
+  // the epilogue applies the three-level inverse 2-D Haar transform of the tile's four patches, w_scale and the
+  // bias before storing Y at the patches' raster positions.
+  int grid_w;              // width of the token grid of a transform block
+  int n_block;             // tokens per transform block (grid_w x height)
 };
 
 constexpr int GEMM_BM = 128;           // output channels per tile
@@ -264,8 +270,65 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
         break;
       }
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(a * BN);
-      if constexpr (EPI == EPI_HAAR_F32 || EPI == EPI_HAAR_BF16) {
-        static_assert(EPI < EPI_HAAR_F32 || BN == 256, "the fused inverse works on 256-token tiles");
+      if constexpr (EPI == EPI_HAAR2D_F32 || EPI == EPI_HAAR2D_BF16) {
+        static_assert(BN == 256, "four 8 x 8 patches per tile");
+        float bch = 0.f;
+        if (ch_ok && p.bias) bch = __ldg(p.bias + ch);
+        const int pw = p.grid_w >> 3;        // patches per grid row
+        const int ppb = p.n_block >> 6;      // patches per transform block
+#pragma unroll 1
+        for (int pp = 0; pp < 2; ++pp) {     // this warp's two patches
+          const int pcol = (half * 2 + pp) * 64;
+          uint32_t r0[32], r1[32];
+          ptx::tmem_ld_32x32b_x32(taddr + pcol, r0);
+          ptx::tmem_ld_32x32b_x32(taddr + pcol + 32, r1);
+          ptx::tmem_ld_wait();
+          const float* sxp = sxs + pcol;
+          // column idx of the patch: 0 = LL_3, then per level l (3, 2, 1) the cells' (LH, HL, HH) triples from
+          // column 4^(3-l) on; the scales carry 2^-l, so the synthesis is additions only
+          auto val = [&](int idx) -> float {
+            const uint32_t u = idx < 32 ? r0[idx & 31] : r1[idx & 31];
+            return static_cast<float>(static_cast<int>(u)) * sxp[idx];
+          };
+          float v[8][8];
+          v[0][0] = val(0);
+#pragma unroll
+          for (int l = 3; l >= 1; --l) {
+            const int st = 1 << (l - 1);
+            const int base = 1 << (2 * (3 - l));
+#pragma unroll
+            for (int y = 0; y < 8; y += 2 * st)
+#pragma unroll
+              for (int x = 0; x < 8; x += 2 * st) {
+                const int idx = base + 3 * ((y >> l) * (8 >> l) + (x >> l));
+                const float ll = v[y][x], lh = val(idx), hl = val(idx + 1), hh = val(idx + 2);
+                const float s0 = ll + lh, s1 = ll - lh, s2 = hl + hh, s3 = hl - hh;
+                v[y][x] = s0 + s2;
+                v[y][x + st] = s1 + s3;
+                v[y + st][x] = s0 - s2;
+                v[y + st][x + st] = s1 - s3;
+              }
+          }
+          if (ch_ok) {
+            const int pt = tok_t * 4 + half * 2 + pp;
+            const int blk = pt / ppb;
+            const int pi = pt - blk * ppb;
+            const int py = pi / pw, px = pi - py * pw;
+            const long o = ((long)blk * p.n_block + (long)(py * 8) * p.grid_w + px * 8) * p.n_out + ch;
+#pragma unroll
+            for (int y = 0; y < 8; ++y)
+#pragma unroll
+              for (int x = 0; x < 8; ++x) {
+                const long oo = o + ((long)y * p.grid_w + x) * p.n_out;
+                if constexpr (EPI == EPI_HAAR2D_F32)
+                  static_cast<float*>(p.out)[oo] = fmaf(v[y][x], sw, bch);
+                else
+                  static_cast<__nv_bfloat16*>(p.out)[oo] = __float2bfloat16_rn(fmaf(v[y][x], sw, bch));
+              }
+          }
+        }
+      } else if constexpr (EPI == EPI_HAAR_F32 || EPI == EPI_HAAR_BF16) {
+        static_assert(BN == 256, "the fused inverse works on 256-token tiles");
         // ---- the tile's eight coarse values (column 32 q), synthesised down to the level-5 sums
         float hd[8];
         {

@@ -13,6 +13,7 @@
 // the row quantizer reads them.  LV <= 3.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace stamp {
 
@@ -23,11 +24,45 @@ __device__ __forceinline__ int haar2d_row(int n, int w, int l, int band, int gy,
   return (band + 1) * q + gy * (w >> l) + gx;
 }
 
+// What a forward launch does with the coefficients.
+//   H2D_STORE_T  write fp32 T to its logical rows (+ row maxima when asked): the general route
+//   H2D_MAX      row maxima only: first launch of the fused route
+//   H2D_QUANT    second launch of the fused route: recompute the patch (its input is still in L2), quantize with
+//                scale = rowmax / qmax (Sec. 2.1, first equation, symmetric) and write int8 codes in PATCH order:
+//                row 64 * patch + idx of a8, idx = 0 for the patch's LL_3 value and 4^(3-l) + 3 * cell + band for
+//                the level-l detail of `band` in the patch's cell (row-major) -- the order in which the GEMM's
+//                fused inverse epilogue synthesises a patch from 64 consecutive accumulator columns.  LV == 3.
+enum Haar2dMode { H2D_STORE_T = 0, H2D_MAX = 1, H2D_QUANT = 2 };
+
+struct Haar2dQuant {
+  int8_t* a8;            // [M, K] codes, patch order                                              out
+  float* sx_epi;         // [M] scale * 2^-l of every a8 row (the synthesis then needs additions only)  out
+  const float* x_scale;  // [M] scale of every logical row (k_haar2d_row_scales)                    in
+  const float* x_inv;    // [M] its reciprocal                                                      in
+  float qmax_hi, qmax_lo;
+  int k_hi;
+};
+
+// Per logical row: scale = rowmax / qmax (IEEE fp32 division; 1 for a zero row) and 1 / scale.
+__global__ void __launch_bounds__(256) k_haar2d_row_scales(const unsigned* __restrict__ rowmax, long M, int n, int k_hi,
+                                                           float qmax_hi, float qmax_lo, float* __restrict__ x_scale,
+                                                           float* __restrict__ x_inv) {
+  const long r = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= M) return;
+  const float qmax = static_cast<int>(r % n) < k_hi ? qmax_hi : qmax_lo;
+  const float amax = __uint_as_float(rowmax[r]);
+  const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
+  x_scale[r] = scale;
+  x_inv[r] = __fdiv_rn(1.0f, scale);
+}
+
 //   in      [nblk, n, K]  TIn        T  [nblk * n, K] float     rowmax [nblk * n] uint bits or nullptr
-template <int LV, typename TIn>
+template <int LV, typename TIn, int MODE>
 __global__ void __launch_bounds__(128) k_haar2d_fwd(const TIn* __restrict__ in, int n, int w, long npatch, int K,
-                                                     float* __restrict__ T, unsigned* __restrict__ rowmax) {
+                                                     float* __restrict__ T, unsigned* __restrict__ rowmax,
+                                                     const Haar2dQuant hq) {
   constexpr int S = 1 << LV;
+  static_assert(MODE != H2D_QUANT || LV == 3, "patch order is defined for 8 x 8 patches");
   const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
   if (c >= K) return;  // whole warps only: K/2 is a multiple of 32
   const int pw = w / S, ph = (n / w) / S;   // patches per grid row / column
@@ -43,29 +78,195 @@ __global__ void __launch_bounds__(128) k_haar2d_fwd(const TIn* __restrict__ in, 
       for (int x = 0; x < S; ++x) v[y][x] = load2(src + ((long)y * w + x) * K);
     float* Tb = T + (blk * n) * (long)K + c;
     unsigned* rm = rowmax ? rowmax + blk * n : nullptr;
-    auto emit = [&](int row, float2 t) {
-      store2(Tb + (long)row * K, t.x, t.y);
-      if (rm) {
-        const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(t.x), absbits(t.y)));
-        if ((threadIdx.x & 31) == 0) atomicMax(rm + row, m);
+    // row: logical row inside the block; idx: position inside the patch (H2D_QUANT); l: level of the coefficient
+    auto emit = [&](int row, int idx, int l, float2 t) {
+      if (MODE == H2D_STORE_T) store2(Tb + (long)row * K, t.x, t.y);
+      if (MODE != H2D_QUANT) {
+        if (rm) {
+          const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(t.x), absbits(t.y)));
+          if ((threadIdx.x & 31) == 0) atomicMax(rm + row, m);
+        }
+      } else {
+        const float qmax = row < hq.k_hi ? hq.qmax_hi : hq.qmax_lo;
+        const float scale = __ldg(hq.x_scale + blk * n + row);
+        const float inv = __ldg(hq.x_inv + blk * n + row);
+        const float q0 = fminf(fmaxf(rintf(fmaf(fmaf(-(t.x * inv), scale, t.x), inv, t.x * inv)), -qmax), qmax);
+        const float q1 = fminf(fmaxf(rintf(fmaf(fmaf(-(t.y * inv), scale, t.y), inv, t.y * inv)), -qmax), qmax);
+        const long arow = pt * (S * S) + idx;
+        *reinterpret_cast<char2*>(hq.a8 + arow * K + c) =
+            make_char2(static_cast<signed char>(static_cast<int>(q0)), static_cast<signed char>(static_cast<int>(q1)));
+        if (c == 0) hq.sx_epi[arow] = scale * (1.0f / static_cast<float>(1 << l));
       }
     };
 #pragma unroll
     for (int l = 1; l <= LV; ++l) {
       const int st = 1 << (l - 1);
+      const int base = 1 << (2 * (LV - l));   // LL values of this level inside the patch: the details follow them
 #pragma unroll
       for (int y = 0; y < S; y += 2 * st)
 #pragma unroll
         for (int x = 0; x < S; x += 2 * st) {
           const float2 a = v[y][x], b = v[y][x + st], cc = v[y + st][x], d = v[y + st][x + st];
           const int gy = (py * S + y) >> l, gx = (px * S + x) >> l;
+          const int idx = base + 3 * ((y >> l) * (S >> l) + (x >> l));
           v[y][x] = make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y)));
-          emit(haar2d_row(n, w, l, 0, gy, gx), make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-          emit(haar2d_row(n, w, l, 1, gy, gx), make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
-          emit(haar2d_row(n, w, l, 2, gy, gx), make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
+          emit(haar2d_row(n, w, l, 0, gy, gx), idx, l, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
+          emit(haar2d_row(n, w, l, 1, gy, gx), idx + 1, l, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+          emit(haar2d_row(n, w, l, 2, gy, gx), idx + 2, l, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
         }
     }
-    emit(haar2d_row(n, w, LV, -1, py, px), v[0][0]);
+    emit(haar2d_row(n, w, LV, -1, py, px), 0, LV, v[0][0]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Fused three-level 2-D Haar transform + quantizer, one CTA per 8 x 8 patch.
+// Every coefficient of the three levels is a function of one patch only, and so is its row of the
+// transformed activation across the K channels: the CTA stages the patch's 64 tokens x K channels in
+// shared memory once, computes the coefficients twice from there -- first for the 64 row maxima
+// (warp reductions + shared-memory atomics), then, with the scales known, for the codes -- and writes
+// codes and scales in the patch order described at Haar2dMode.  X is read from HBM once and T is never
+// materialised.  Needs 64 * K * sizeof(TIn) bytes of shared memory (K <= 1792 for bf16).
+// A thread owns two adjacent channels and walks the patch quadrant by quadrant (16 tokens in registers).
+// ------------------------------------------------------------------------------------------
+
+struct Haar2dPatchParams {
+  const void* in;        // [nblk, n, K]
+  int n, w, K, k_hi;
+  float qmax_hi, qmax_lo;
+  int8_t* a8;            // [M, K] patch order
+  float* sx_epi;         // [M] patch order, scale * 2^-l
+  float* x_scale;        // [M] logical order
+  const uint8_t* pf_base; // optional region (the layer's weight codes) to pull towards L2 for the GEMM that follows
+  long pf_bytes;          // multiple of 16, 0 for none
+};
+
+// One sweep over a staged patch xs [64 tokens][K] for the channel pair starting at c: emit(idx, value) is called
+// once per coefficient, idx in the patch order described at Haar2dMode.
+template <typename TIn, typename F>
+__device__ __forceinline__ void haar2d_patch_sweep(const TIn* xs, int K, int c, F&& emit) {
+    // (the quadrant loop stays rolled: unrolled, the compiler hoists all 64 loads and spills)
+    float2 ll2_0 = make_float2(0.f, 0.f), ll2_1 = ll2_0, ll2_2 = ll2_0, ll2_3 = ll2_0;
+#pragma unroll 1
+    for (int q = 0; q < 4; ++q) {             // quadrant (qy, qx) of 4 x 4 tokens
+      const int qy = q >> 1, qx = q & 1;
+      float2 v[4][4];
+#pragma unroll
+      for (int y = 0; y < 4; ++y)
+#pragma unroll
+        for (int x = 0; x < 4; ++x) v[y][x] = load2(xs + (long)((qy * 4 + y) * 8 + qx * 4 + x) * K + c);
+      float2 ll1[2][2];
+#pragma unroll
+      for (int cy = 0; cy < 2; ++cy)
+#pragma unroll
+        for (int cx = 0; cx < 2; ++cx) {      // level 1: cell (2 qy + cy, 2 qx + cx) of the patch's 4 x 4 cells
+          const float2 a = v[2 * cy][2 * cx], b = v[2 * cy][2 * cx + 1], cc = v[2 * cy + 1][2 * cx], d = v[2 * cy + 1][2 * cx + 1];
+          const int idx = 16 + 3 * ((2 * qy + cy) * 4 + (2 * qx + cx));
+          ll1[cy][cx] = make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y)));
+          emit(idx, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
+          emit(idx + 1, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+          emit(idx + 2, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
+        }
+      {                                       // level 2: cell (qy, qx) of the patch's 2 x 2 cells
+        const float2 a = ll1[0][0], b = ll1[0][1], cc = ll1[1][0], d = ll1[1][1];
+        const int idx = 4 + 3 * q;
+        const float2 s4 = make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y)));
+        if (q == 0) ll2_0 = s4;
+        if (q == 1) ll2_1 = s4;
+        if (q == 2) ll2_2 = s4;
+        if (q == 3) ll2_3 = s4;
+        emit(idx, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
+        emit(idx + 1, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+        emit(idx + 2, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
+      }
+    }
+    {                                         // level 3
+      const float2 a = ll2_0, b = ll2_1, cc = ll2_2, d = ll2_3;
+      emit(0, make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y))));
+      emit(1, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
+      emit(2, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+      emit(3, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
+    }
+}
+
+template <typename TIn, int H2P_THREADS>
+__global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haar2dPatchParams p) {
+  extern __shared__ __align__(16) uint8_t h2p_smem[];
+  __shared__ unsigned s_max[64];
+  __shared__ float s_scale[64], s_inv[64], s_qmax[64];
+  TIn* xs = reinterpret_cast<TIn*>(h2p_smem);      // [64 tokens (patch raster)][K]
+  const int K = p.K, n = p.n, w = p.w;
+  const int pw = w >> 3, ppb = n >> 6;
+  const long pt = blockIdx.x;
+  const long blk = pt / ppb;
+  const int pi = static_cast<int>(pt - blk * ppb);
+  const int py = pi / pw, px = pi - py * pw;
+  const int tid = threadIdx.x;
+  if (tid < 64) s_max[tid] = 0u;
+  if (p.pf_bytes > 0 && tid < 32) {   // fire-and-forget hints, 8 KB each
+    const long nchunk = (p.pf_bytes + 8191) / 8192;
+    for (long ck = (long)blockIdx.x * 32 + tid; ck < nchunk; ck += (long)gridDim.x * 32) {
+      const long left = p.pf_bytes - ck * 8192;
+      ptx::prefetch_l2_bulk(p.pf_base + ck * 8192, static_cast<uint32_t>(left < 8192 ? left : 8192));
+    }
+  }
+  // stage: patch row y is 8 consecutive tokens = 8 K contiguous elements
+  {
+    const int vec_per_row = 8 * K * (int)sizeof(TIn) / 16;
+    const TIn* src0 = static_cast<const TIn*>(p.in) + (blk * n + (long)(py * 8) * w + px * 8) * K;
+#pragma unroll 1
+    for (int y = 0; y < 8; ++y) {
+      const uint4* src = reinterpret_cast<const uint4*>(src0 + (long)y * w * K);
+      uint4* dst = reinterpret_cast<uint4*>(xs + (long)y * 8 * K);
+      for (int i = tid; i < vec_per_row; i += H2P_THREADS) dst[i] = __ldg(src + i);
+    }
+  }
+  __syncthreads();
+
+  // ---- pass 1: row maxima.  Whole warps only enter (K / 2 is a multiple of 32).
+  for (int c2 = tid; c2 < K / 2; c2 += H2P_THREADS)
+    haar2d_patch_sweep(xs, K, 2 * c2, [&](int idx, float2 t) {
+      const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(t.x), absbits(t.y)));
+      if ((tid & 31) == 0) atomicMax(&s_max[idx], m);
+    });
+  __syncthreads();
+  if (tid < 64) {
+    // coefficient idx of the patch -> level, band, cell -> logical row of the block
+    int l, band, cy, cx;
+    if (tid == 0) {
+      l = 3; band = -1; cy = 0; cx = 0;
+    } else {
+      l = tid < 4 ? 3 : (tid < 16 ? 2 : 1);
+      const int e = tid - (1 << (2 * (3 - l)));
+      const int cell = e / 3;
+      band = e - 3 * cell;
+      cy = cell >> (3 - l);
+      cx = cell & ((1 << (3 - l)) - 1);
+    }
+    const int gy = (py << (3 - l)) + cy, gx = (px << (3 - l)) + cx;
+    const int row = haar2d_row(n, w, l, band, gy, gx);
+    const float qmax = row < p.k_hi ? p.qmax_hi : p.qmax_lo;
+    const float amax = __uint_as_float(s_max[tid]);
+    const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
+    s_scale[tid] = scale;
+    s_inv[tid] = __fdiv_rn(1.0f, scale);
+    s_qmax[tid] = qmax;
+    p.x_scale[blk * n + row] = scale;
+    p.sx_epi[pt * 64 + tid] = scale * (1.0f / static_cast<float>(1 << l));
+  }
+  __syncthreads();
+  // ---- pass 2: codes
+  int8_t* a8p = p.a8 + pt * 64 * (long)K;
+  for (int c2 = tid; c2 < K / 2; c2 += H2P_THREADS) {
+    const int c = 2 * c2;
+    haar2d_patch_sweep(xs, K, c, [&](int idx, float2 t) {
+      const float scale = s_scale[idx], inv = s_inv[idx], qmax = s_qmax[idx];
+      const float a0 = t.x * inv, a1 = t.y * inv;
+      const float q0 = fminf(fmaxf(rintf(fmaf(fmaf(-a0, scale, t.x), inv, a0)), -qmax), qmax);
+      const float q1 = fminf(fmaxf(rintf(fmaf(fmaf(-a1, scale, t.y), inv, a1)), -qmax), qmax);
+      *reinterpret_cast<char2*>(a8p + (long)idx * K + c) =
+          make_char2(static_cast<signed char>(static_cast<int>(q0)), static_cast<signed char>(static_cast<int>(q1)));
+    });
   }
 }
 

@@ -287,7 +287,7 @@ static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const Gem
 static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K, const float* x_scale,
                        const float* w_scale, void* out, int epi, cudaStream_t st, const float* bias = nullptr,
                        const float* a8v = nullptr, int depth = 0, const int* x_zero = nullptr,
-                       const int* w_sum = nullptr) {
+                       const int* w_sum = nullptr, int grid_w = 0, int n_block = 0) {
   GemmParams gp{};
   gp.n_out = N;
   gp.m_tok = (int)M;
@@ -301,6 +301,8 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
   gp.depth = depth;
   gp.x_zero = x_zero;
   gp.w_sum = w_sum;
+  gp.grid_w = grid_w;
+  gp.n_block = n_block;
   CUtensorMap tw, tx;
   int rc = make_tmap_i8(w8, N, K, GEMM_BM, &tw);
   if (rc) return rc;
@@ -315,6 +317,11 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
   if (epi == EPI_DEQUANT_BF16X2)
     return wide ? launch_gemm_t<256, 4, EPI_DEQUANT_BF16X2>(tw, tx, gp, st)
                 : launch_gemm_t<128, 6, EPI_DEQUANT_BF16X2>(tw, tx, gp, st);
+  if (epi == EPI_HAAR2D_F32 || epi == EPI_HAAR2D_BF16) {
+    if (!wide || M % 256 != 0 || grid_w < 8 || grid_w % 8 != 0 || n_block % (8 * grid_w) != 0) return STAMP_ERR_UNSUPPORTED;
+    if (epi == EPI_HAAR2D_F32) return launch_gemm_t<256, 4, EPI_HAAR2D_F32>(tw, tx, gp, st);
+    return launch_gemm_t<256, 4, EPI_HAAR2D_BF16>(tw, tx, gp, st);
+  }
   if (epi == EPI_DEQUANT_ZP_F32) {
     if (!x_zero || !w_sum) return STAMP_ERR_INVALID_ARG;
     return wide ? launch_gemm_t<256, 4, EPI_DEQUANT_ZP_F32>(tw, tx, gp, st)
@@ -386,13 +393,54 @@ static int make_dct_matrix(int transform, int n, float* mat, cudaStream_t st) {
 }
 
 // T = L X (Haar, identity or blockwise DCT-II), fp32, logical order; optionally the per-row |T| maxima.
-template <int LV, typename TIn>
-static int launch_haar2d_fwd(const Problem& pb, const TIn* X, float* T, unsigned* rowmax, cudaStream_t st) {
+template <int LV, typename TIn, int MODE = H2D_STORE_T>
+static int launch_haar2d_fwd(const Problem& pb, const TIn* X, float* T, unsigned* rowmax, cudaStream_t st,
+                             const Haar2dQuant& hq = Haar2dQuant{}) {
   const long npatch = pb.M >> (2 * LV);
   dim3 grid((pb.K / 2 + 127) / 128, (unsigned)(npatch < 32768 ? npatch : 32768));
-  k_haar2d_fwd<LV, TIn><<<grid, 128, 0, st>>>(X, pb.n, pb.grid_w, npatch, pb.K, T, rowmax);
+  k_haar2d_fwd<LV, TIn, MODE><<<grid, 128, 0, st>>>(X, pb.n, pb.grid_w, npatch, pb.K, T, rowmax, hq);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
+}
+
+template <typename TIn, int THREADS>
+static int launch_haar2d_patch(const Haar2dPatchParams& pp, long npatch, size_t smem, cudaStream_t st) {
+  auto kern = k_haar2d_patch_quant<TIn, THREADS>;
+  static size_t attr_smem = 0;
+  if (smem > attr_smem) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return STAMP_ERR_CUDA;
+    attr_smem = smem;
+  }
+  kern<<<(unsigned)npatch, THREADS, smem, st>>>(pp);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// Fused route of the three-level 2-D Haar transform: codes and scales in patch order.  One CTA per patch when a
+// patch (64 tokens x K channels) fits in shared memory; otherwise row maxima, scales, then codes in three launches.
+template <typename TIn>
+static int run_quantize_haar2d_patch(const Problem& pb, const TIn* X, unsigned* rowmax, float* x_scale, float* x_inv,
+                                     int8_t* a8, float* sx_epi, const int8_t* w8, cudaStream_t st) {
+  const size_t smem = (size_t)64 * pb.K * sizeof(TIn);
+  if (smem <= 224 * 1024) {
+    Haar2dPatchParams pp{X, pb.n, pb.grid_w, pb.K, pb.k_hi, (float)pb.qmax_hi, (float)pb.qmax_lo, a8, sx_epi, x_scale,
+                         nullptr, 0};
+    if ((size_t)pb.N * pb.K <= (size_t)24 << 20) {   // small weight matrix: have it in L2 when the GEMM starts
+      pp.pf_base = reinterpret_cast<const uint8_t*>(w8);
+      pp.pf_bytes = (long)pb.N * pb.K;
+    }
+    // a thread owns a channel pair: 576 threads when the pairs fill them exactly (1152 channels), else 512
+    if ((pb.K / 2) % 576 == 0) return launch_haar2d_patch<TIn, 576>(pp, pb.M >> 6, smem, st);
+    return launch_haar2d_patch<TIn, 512>(pp, pb.M >> 6, smem, st);
+  }
+  if (cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+  if (int rc = launch_haar2d_fwd<3, TIn, H2D_MAX>(pb, X, nullptr, rowmax, st)) return rc;
+  k_haar2d_row_scales<<<(unsigned)((pb.M + 255) / 256), 256, 0, st>>>(rowmax, pb.M, pb.n, pb.k_hi, (float)pb.qmax_hi,
+                                                                      (float)pb.qmax_lo, x_scale, x_inv);
+  STAMP_CHECK_LAUNCH();
+  Haar2dQuant hq{a8, sx_epi, x_scale, x_inv, (float)pb.qmax_hi, (float)pb.qmax_lo, pb.k_hi};
+  return launch_haar2d_fwd<3, TIn, H2D_QUANT>(pb, X, nullptr, rowmax, st, hq);
 }
 template <int LV, typename TOut>
 static int launch_haar2d_inv(const Problem& pb, const float* Yt, const float* bias, TOut* Y, cudaStream_t st) {
@@ -1029,6 +1077,21 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
                           w_sum)))
       return rc;
     return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
+  }
+  if (pb.transform == STAMP_T_HAAR2D && pb.levels == 3 && pb.M % 256 == 0) {
+    // Fused route of the paper's LVM transform: two passes over X (row maxima; codes in patch order, the second
+    // pass reading X from L2), then the GEMM whose epilogue inverts the four 8 x 8 patches of its 256-token tile.
+    float* x_inv = T;               // the fp32 T of the general route is not materialised here: reuse its space
+    float* sx_epi = T + pb.M;
+    const int8_t* w8p = nullptr;
+    if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8p, st))) return rc;
+    if (x_dtype == STAMP_BF16)
+      rc = run_quantize_haar2d_patch(pb, static_cast<const __nv_bfloat16*>(X), rowmax, x_scale, x_inv, a8, sx_epi, w8p, st);
+    else
+      rc = run_quantize_haar2d_patch(pb, static_cast<const float*>(X), rowmax, x_scale, x_inv, a8, sx_epi, w8p, st);
+    if (rc) return rc;
+    return launch_gemm(a8, w8p, pb.M, N, K, sx_epi, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR2D_BF16 : EPI_HAAR2D_F32,
+                       st, bias, nullptr, 0, nullptr, nullptr, pb.grid_w, pb.n);
   }
   CqChoice cc;
   const bool have_cq = (pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc);

@@ -25,7 +25,10 @@ Y_TOL = 1e-3
 def _scale_rtol(cfg):
     """A scale is absmax / qmax of a transformed row, so it inherits the tolerance on T.  Haar
     coefficients see at most log2(n) fp32 roundings (1e-6 holds); a DCT coefficient is an fp32 sum
-    of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised."""
+    of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised.  A 2-D Haar
+    coefficient of level l is the result of 3 l fp32 additions (9 roundings for 3 levels): 2e-6."""
+    if cfg.transform == gen.T_HAAR2D:
+        return 2e-6
     return 1e-5 if cfg.transform in (gen.T_DCT2, gen.T_WHT) else 1e-6
 
 FULL = {

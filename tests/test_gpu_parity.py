@@ -20,7 +20,10 @@ Y_TOL = 1e-3
 def _scale_rtol(cfg):
     """A scale is absmax / qmax of a transformed row, so it inherits the tolerance on T.  Haar
     coefficients see at most log2(n) fp32 roundings (1e-6 holds); a DCT coefficient is an fp32 sum
-    of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised."""
+    of n products, whose error grows like sqrt(n) ulp, so only the 1e-5 of T itself is promised.  A 2-D Haar
+    coefficient of level l is the result of 3 l fp32 additions (9 roundings for 3 levels): 2e-6."""
+    if cfg.transform == gen.T_HAAR2D:
+        return 2e-6
     return 1e-5 if cfg.transform in (gen.T_DCT2, gen.T_WHT) else 1e-6
 
 
@@ -74,6 +77,11 @@ CASES = {
     # 2-D Haar over the patch grid: square and oblong grids, one to three levels
     "haar2d_3": gen.scaled(gen.config_dit_proj_2d(), B=2, L=1024, K=256, N=136, grid=32, levels=3, k_hi=16),
     "haar2d_1": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=128, N=64, grid=16, levels=1, k_hi=64),
+    # oblong grid (32 wide, 16 high), fp32 input, ragged channel tile: the fused patch-order route again
+    "haar2d_oblong": gen.scaled(gen.config_dit_proj_2d(), B=3, L=512, K=128, N=72, grid=32, levels=3, k_hi=8,
+                                dtype=gen.F32, recipe="ar1"),
+    # a patch (64 tokens x 2048 channels) that does not fit in shared memory: row maxima and codes in separate launches
+    "haar2d_wide_k": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=2048, N=64, grid=16, levels=3, k_hi=4),
     # two levels only: no cluster tree, approximation rows quantized by the same kernel
     "two_levels": gen.scaled(gen.config_dit_proj(), B=2, L=256, K=1152, N=128, grid=16, levels=2, k_hi=64),
 }
