@@ -193,7 +193,9 @@ template <typename TIn, int H2P_THREADS>
 __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haar2dPatchParams p) {
   extern __shared__ __align__(16) uint8_t h2p_smem[];
   __shared__ unsigned s_max[64];
-  __shared__ float s_scale[64], s_inv[64], s_qmax[64];
+  __shared__ float4 s_tab[64];                      // {scale, 1 / scale, qmax, -} per coefficient of the patch
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ uint32_t s_abort;
   TIn* xs = reinterpret_cast<TIn*>(h2p_smem);      // [64 tokens (patch raster)][K]
   const int K = p.K, n = p.n, w = p.w;
   const int pw = w >> 3, ppb = n >> 6;
@@ -210,18 +212,26 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
       ptx::prefetch_l2_bulk(p.pf_base + ck * 8192, static_cast<uint32_t>(left < 8192 ? left : 8192));
     }
   }
-  // stage: patch row y is 8 consecutive tokens = 8 K contiguous elements
-  {
-    const int vec_per_row = 8 * K * (int)sizeof(TIn) / 16;
-    const TIn* src0 = static_cast<const TIn*>(p.in) + (blk * n + (long)(py * 8) * w + px * 8) * K;
-#pragma unroll 1
-    for (int y = 0; y < 8; ++y) {
-      const uint4* src = reinterpret_cast<const uint4*>(src0 + (long)y * w * K);
-      uint4* dst = reinterpret_cast<uint4*>(xs + (long)y * 8 * K);
-      for (int i = tid; i < vec_per_row; i += H2P_THREADS) dst[i] = __ldg(src + i);
-    }
+  // stage: patch row y is 8 consecutive tokens = 8 K contiguous elements -> eight bulk copies on one mbarrier
+  if (tid == 0) {
+    s_abort = 0;
+    ptx::mbar_init(&s_bar, 1);
+    ptx::fence_mbar_init();
   }
   __syncthreads();
+  if (tid == 0) {
+    const uint32_t row_bytes = 8u * static_cast<uint32_t>(K) * static_cast<uint32_t>(sizeof(TIn));
+    const TIn* src0 = static_cast<const TIn*>(p.in) + (blk * n + (long)(py * 8) * w + px * 8) * K;
+    ptx::mbar_arrive_expect_tx(&s_bar, 8u * row_bytes);
+#pragma unroll 1
+    for (int y = 0; y < 8; ++y) ptx::bulk_load(xs + (long)y * 8 * K, src0 + (long)y * w * K, row_bytes, &s_bar);
+  }
+  if (!ptx::mbar_wait_bounded(&s_bar, 0u, &s_abort, 2000000000LL)) {
+    // the copies did not land within about a second: record it and leave the patch unwritten
+    s_abort = 1;
+    raise_device_status(STAMP_ERR_TIMEOUT);
+    return;
+  }
 
   // ---- pass 1: row maxima.  Whole warps only enter (K / 2 is a multiple of 32).
   for (int c2 = tid; c2 < K / 2; c2 += H2P_THREADS)
@@ -248,9 +258,7 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
     const float qmax = row < p.k_hi ? p.qmax_hi : p.qmax_lo;
     const float amax = __uint_as_float(s_max[tid]);
     const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
-    s_scale[tid] = scale;
-    s_inv[tid] = __fdiv_rn(1.0f, scale);
-    s_qmax[tid] = qmax;
+    s_tab[tid] = make_float4(scale, __fdiv_rn(1.0f, scale), qmax, 0.f);
     p.x_scale[blk * n + row] = scale;
     p.sx_epi[pt * 64 + tid] = scale * (1.0f / static_cast<float>(1 << l));
   }
@@ -260,12 +268,13 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
   for (int c2 = tid; c2 < K / 2; c2 += H2P_THREADS) {
     const int c = 2 * c2;
     haar2d_patch_sweep(xs, K, c, [&](int idx, float2 t) {
-      const float scale = s_scale[idx], inv = s_inv[idx], qmax = s_qmax[idx];
-      const float a0 = t.x * inv, a1 = t.y * inv;
-      const float q0 = fminf(fmaxf(rintf(fmaf(fmaf(-a0, scale, t.x), inv, a0)), -qmax), qmax);
-      const float q1 = fminf(fmaxf(rintf(fmaf(fmaf(-a1, scale, t.y), inv, a1)), -qmax), qmax);
-      *reinterpret_cast<char2*>(a8p + (long)idx * K + c) =
-          make_char2(static_cast<signed char>(static_cast<int>(q0)), static_cast<signed char>(static_cast<int>(q1)));
+      const float4 tb = s_tab[idx];               // scale, 1 / scale, qmax
+      const float a0 = t.x * tb.y, a1 = t.y * tb.y;
+      // clamp, then round to nearest even by adding 1.5 * 2^23: the code is the low byte of the sum's bit pattern
+      const float q0 = fminf(fmaxf(fmaf(fmaf(-a0, tb.x, t.x), tb.y, a0), -tb.z), tb.z) + 12582912.0f;
+      const float q1 = fminf(fmaxf(fmaf(fmaf(-a1, tb.x, t.y), tb.y, a1), -tb.z), tb.z) + 12582912.0f;
+      *reinterpret_cast<uint16_t*>(a8p + (long)idx * K + c) =
+          static_cast<uint16_t>(__byte_perm(__float_as_uint(q0), __float_as_uint(q1), 0x0040));
     });
   }
 }
