@@ -50,6 +50,7 @@ struct GemmParams {
   // * x_scale[tok] * w_scale[ch], the bracket in 64-bit integers
   const int* x_zero;       // [m_tok] zero point of every token's stored codes
   const int* w_sum;        // [n_out] sum over k of the weight codes of a channel
+  // (x_zero / w_sum may also be given to EPI_HAAR2D_*: the same term is then taken out before the synthesis.)
   // EPI_HAAR2D_*: the token operand is in the patch order of the 2-D Haar quantize kernel (64 consecutive rows
   // = the coefficients of one 8 x 8 patch of the token grid in synthesis order), x_scale holds scale * 2^-l, and
   // the epilogue applies the three-level inverse 2-D Haar transform of the tile's four patches, w_scale and the
@@ -239,6 +240,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       float* sxs = sx_stage + a * BN;
       float sw = 0.f;
       int* zps = zp_stage + a * BN;
+      // zero-point codes: always in the de-quantize epilogue made for them, on request in the 2-D Haar ones
+      const bool with_zp = (EPI == EPI_DEQUANT_ZP_F32) ||
+                           ((EPI == EPI_HAAR2D_F32 || EPI == EPI_HAAR2D_BF16) && p.x_zero != nullptr);
       float my_sx = 0.f;
       int my_zp = 0, wsum = 0;
       if (EPI != EPI_RAW_I32) {
@@ -246,9 +250,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
         // fetch this tile's token scales while the accumulator is still being filled
         if (ep_tid < BN && tok0 + ep_tid < p.m_tok) {
           my_sx = __ldg(p.x_scale + tok0 + ep_tid);
-          if (EPI == EPI_DEQUANT_ZP_F32) my_zp = __ldg(p.x_zero + tok0 + ep_tid);
+          if (with_zp) my_zp = __ldg(p.x_zero + tok0 + ep_tid);
         }
-        if (EPI == EPI_DEQUANT_ZP_F32 && ch_ok) wsum = __ldg(p.w_sum + ch);
+        if (with_zp && ch_ok) wsum = __ldg(p.w_sum + ch);
       }
       // The eight epilogue warps continue or stop TOGETHER: a warp whose wait ran out raises the abort
       // word, and everybody reads it behind the named barrier below -- no warp is left waiting at that
@@ -261,7 +265,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
         // them arrived on tempty[a] before tfull[a] could complete again), so its staging buffer is free
         if (ep_tid < BN) {
           sxs[ep_tid] = my_sx;
-          if (EPI == EPI_DEQUANT_ZP_F32) zps[ep_tid] = my_zp;
+          if (with_zp) zps[ep_tid] = my_zp;
         }
       }
       asm volatile("bar.sync 1, %0;" ::"n"(GEMM_EPI_THREADS) : "memory");
@@ -284,10 +288,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
           ptx::tmem_ld_32x32b_x32(taddr + pcol + 32, r1);
           ptx::tmem_ld_wait();
           const float* sxp = sxs + pcol;
+          const int* zpp = zps + pcol;
           // column idx of the patch: 0 = LL_3, then per level l (3, 2, 1) the cells' (LH, HL, HH) triples from
           // column 4^(3-l) on; the scales carry 2^-l, so the synthesis is additions only
           auto val = [&](int idx) -> float {
             const uint32_t u = idx < 32 ? r0[idx & 31] : r1[idx & 31];
+            if (with_zp)   // (acc - zc * sum_k w) in 64-bit integers, as in EPI_DEQUANT_ZP_F32
+              return __ll2float_rn(static_cast<long long>(static_cast<int>(u)) -
+                                   static_cast<long long>(zpp[idx]) * wsum) * sxp[idx];
             return static_cast<float>(static_cast<int>(u)) * sxp[idx];
           };
           float v[8][8];

@@ -137,6 +137,7 @@ struct Haar2dPatchParams {
   int8_t* a8;            // [M, K] patch order
   float* sx_epi;         // [M] patch order, scale * 2^-l
   float* x_scale;        // [M] logical order
+  int* zp_epi;           // [M] patch order: zero point of every row's stored codes (zero-point variant only)
   const uint8_t* pf_base; // optional region (the layer's weight codes) to pull towards L2 for the GEMM that follows
   long pf_bytes;          // multiple of 16, 0 for none
 };
@@ -189,11 +190,22 @@ __device__ __forceinline__ void haar2d_patch_sweep(const TIn* xs, int K, int c, 
     }
 }
 
-template <typename TIn, int H2P_THREADS>
+// Order-preserving map of a float onto a signed integer (for integer min / max reductions), and back.
+__device__ __forceinline__ int float_order_key(float v) {
+  const int b = __float_as_int(v);
+  return b >= 0 ? b : b ^ 0x7fffffff;
+}
+__device__ __forceinline__ float float_from_order_key(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff); }
+
+// ZP = false: symmetric codes (scale = absmax / qmax).  ZP = true: the zero-point form of Sec. 2.1's first
+// equation with min-max range, codes and zero points stored offset by half the code range (see k_quant_rows_zp).
+template <typename TIn, int H2P_THREADS, bool ZP>
 __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haar2dPatchParams p) {
   extern __shared__ __align__(16) uint8_t h2p_smem[];
-  __shared__ unsigned s_max[64];
+  __shared__ unsigned s_max[64];                    // |t| maxima as bit patterns; ZP: maxima as order keys
+  __shared__ int s_min[64];                         // ZP: minima as order keys
   __shared__ float4 s_tab[64];                      // {scale, 1 / scale, qmax, -} per coefficient of the patch
+                                                    // ZP: {scale, 1 / scale, top code, zero point} (last two as int bits)
   __shared__ __align__(8) uint64_t s_bar;
   __shared__ uint32_t s_abort;
   TIn* xs = reinterpret_cast<TIn*>(h2p_smem);      // [64 tokens (patch raster)][K]
@@ -204,7 +216,10 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
   const int pi = static_cast<int>(pt - blk * ppb);
   const int py = pi / pw, px = pi - py * pw;
   const int tid = threadIdx.x;
-  if (tid < 64) s_max[tid] = 0u;
+  if (tid < 64) {
+    s_max[tid] = ZP ? 0x80000000u : 0u;   // ZP: INT_MIN as the identity of the signed maximum
+    s_min[tid] = 0x7fffffff;
+  }
   if (p.pf_bytes > 0 && tid < 32) {   // fire-and-forget hints, 8 KB each
     const long nchunk = (p.pf_bytes + 8191) / 8192;
     for (long ck = (long)blockIdx.x * 32 + tid; ck < nchunk; ck += (long)gridDim.x * 32) {
@@ -236,8 +251,18 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
   // ---- pass 1: row maxima.  Whole warps only enter (K / 2 is a multiple of 32).
   for (int c2 = tid; c2 < K / 2; c2 += H2P_THREADS)
     haar2d_patch_sweep(xs, K, 2 * c2, [&](int idx, float2 t) {
-      const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(t.x), absbits(t.y)));
-      if ((tid & 31) == 0) atomicMax(&s_max[idx], m);
+      if (!ZP) {
+        const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(t.x), absbits(t.y)));
+        if ((tid & 31) == 0) atomicMax(&s_max[idx], m);
+      } else {
+        const int k0 = float_order_key(t.x), k1 = float_order_key(t.y);
+        const int hi = __reduce_max_sync(0xffffffffu, max(k0, k1));
+        const int lo = __reduce_min_sync(0xffffffffu, min(k0, k1));
+        if ((tid & 31) == 0) {
+          atomicMax(reinterpret_cast<int*>(&s_max[idx]), hi);
+          atomicMin(&s_min[idx], lo);
+        }
+      }
     });
   __syncthreads();
   if (tid < 64) {
@@ -255,10 +280,24 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
     }
     const int gy = (py << (3 - l)) + cy, gx = (px << (3 - l)) + cx;
     const int row = haar2d_row(n, w, l, band, gy, gx);
-    const float qmax = row < p.k_hi ? p.qmax_hi : p.qmax_lo;
-    const float amax = __uint_as_float(s_max[tid]);
-    const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
-    s_tab[tid] = make_float4(scale, __fdiv_rn(1.0f, scale), qmax, 0.f);
+    float scale;
+    if (!ZP) {
+      const float qmax = row < p.k_hi ? p.qmax_hi : p.qmax_lo;
+      const float amax = __uint_as_float(s_max[tid]);
+      scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
+      s_tab[tid] = make_float4(scale, __fdiv_rn(1.0f, scale), qmax, 0.f);
+    } else {
+      const int half = row < p.k_hi ? 128 : 8;
+      const int top = 2 * half - 1;
+      const float mx = float_from_order_key(static_cast<int>(s_max[tid])), mn = float_from_order_key(s_min[tid]);
+      scale = __fdiv_rn(mx - mn, static_cast<float>(top));
+      if (!(scale > 0.f)) scale = 1.0f;
+      float zf = rintf(__fdiv_rn(-mn, scale));
+      zf = fminf(fmaxf(zf, -1073741824.0f), 1073741824.0f);
+      const int z = static_cast<int>(zf);
+      s_tab[tid] = make_float4(scale, __fdiv_rn(1.0f, scale), __int_as_float(top), __int_as_float(z));
+      p.zp_epi[pt * 64 + tid] = z - half;
+    }
     p.x_scale[blk * n + row] = scale;
     p.sx_epi[pt * 64 + tid] = scale * (1.0f / static_cast<float>(1 << l));
   }
@@ -270,11 +309,20 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
     haar2d_patch_sweep(xs, K, c, [&](int idx, float2 t) {
       const float4 tb = s_tab[idx];               // scale, 1 / scale, qmax
       const float a0 = t.x * tb.y, a1 = t.y * tb.y;
-      // clamp, then round to nearest even by adding 1.5 * 2^23: the code is the low byte of the sum's bit pattern
-      const float q0 = fminf(fmaxf(fmaf(fmaf(-a0, tb.x, t.x), tb.y, a0), -tb.z), tb.z) + 12582912.0f;
-      const float q1 = fminf(fmaxf(fmaf(fmaf(-a1, tb.x, t.y), tb.y, a1), -tb.z), tb.z) + 12582912.0f;
-      *reinterpret_cast<uint16_t*>(a8p + (long)idx * K + c) =
-          static_cast<uint16_t>(__byte_perm(__float_as_uint(q0), __float_as_uint(q1), 0x0040));
+      const float r0 = fmaf(fmaf(-a0, tb.x, t.x), tb.y, a0), r1 = fmaf(fmaf(-a1, tb.x, t.y), tb.y, a1);   // t / scale
+      if (!ZP) {
+        // clamp, then round to nearest even by adding 1.5 * 2^23: the code is the low byte of the sum's bit pattern
+        const float q0 = fminf(fmaxf(r0, -tb.z), tb.z) + 12582912.0f;
+        const float q1 = fminf(fmaxf(r1, -tb.z), tb.z) + 12582912.0f;
+        *reinterpret_cast<uint16_t*>(a8p + (long)idx * K + c) =
+            static_cast<uint16_t>(__byte_perm(__float_as_uint(q0), __float_as_uint(q1), 0x0040));
+      } else {
+        const int top = __float_as_int(tb.z), z = __float_as_int(tb.w), half = (top + 1) >> 1;
+        const int q0 = max(0, min(top, __float2int_rn(r0) + z)) - half;
+        const int q1 = max(0, min(top, __float2int_rn(r1) + z)) - half;
+        *reinterpret_cast<uint16_t*>(a8p + (long)idx * K + c) =
+            static_cast<uint16_t>(__byte_perm(static_cast<unsigned>(q0), static_cast<unsigned>(q1), 0x0040));
+      }
     });
   }
 }

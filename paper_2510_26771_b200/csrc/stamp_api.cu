@@ -403,9 +403,9 @@ static int launch_haar2d_fwd(const Problem& pb, const TIn* X, float* T, unsigned
   return STAMP_OK;
 }
 
-template <typename TIn, int THREADS>
+template <typename TIn, int THREADS, bool ZP>
 static int launch_haar2d_patch(const Haar2dPatchParams& pp, long npatch, size_t smem, cudaStream_t st) {
-  auto kern = k_haar2d_patch_quant<TIn, THREADS>;
+  auto kern = k_haar2d_patch_quant<TIn, THREADS, ZP>;
   static size_t attr_smem = 0;
   if (smem > attr_smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -421,19 +421,24 @@ static int launch_haar2d_patch(const Haar2dPatchParams& pp, long npatch, size_t 
 // patch (64 tokens x K channels) fits in shared memory; otherwise row maxima, scales, then codes in three launches.
 template <typename TIn>
 static int run_quantize_haar2d_patch(const Problem& pb, const TIn* X, unsigned* rowmax, float* x_scale, float* x_inv,
-                                     int8_t* a8, float* sx_epi, const int8_t* w8, cudaStream_t st) {
+                                     int8_t* a8, float* sx_epi, int* zp_epi, const int8_t* w8, cudaStream_t st) {
   const size_t smem = (size_t)64 * pb.K * sizeof(TIn);
   if (smem <= 224 * 1024) {
     Haar2dPatchParams pp{X, pb.n, pb.grid_w, pb.K, pb.k_hi, (float)pb.qmax_hi, (float)pb.qmax_lo, a8, sx_epi, x_scale,
-                         nullptr, 0};
+                         zp_epi, nullptr, 0};
     if ((size_t)pb.N * pb.K <= (size_t)24 << 20) {   // small weight matrix: have it in L2 when the GEMM starts
       pp.pf_base = reinterpret_cast<const uint8_t*>(w8);
       pp.pf_bytes = (long)pb.N * pb.K;
     }
     // a thread owns a channel pair: 576 threads when the pairs fill them exactly (1152 channels), else 512
-    if ((pb.K / 2) % 576 == 0) return launch_haar2d_patch<TIn, 576>(pp, pb.M >> 6, smem, st);
-    return launch_haar2d_patch<TIn, 512>(pp, pb.M >> 6, smem, st);
+    if (pb.act_zp) {
+      if ((pb.K / 2) % 576 == 0) return launch_haar2d_patch<TIn, 576, true>(pp, pb.M >> 6, smem, st);
+      return launch_haar2d_patch<TIn, 512, true>(pp, pb.M >> 6, smem, st);
+    }
+    if ((pb.K / 2) % 576 == 0) return launch_haar2d_patch<TIn, 576, false>(pp, pb.M >> 6, smem, st);
+    return launch_haar2d_patch<TIn, 512, false>(pp, pb.M >> 6, smem, st);
   }
+  if (pb.act_zp) return STAMP_ERR_UNSUPPORTED;   // the caller takes the general zero-point route
   if (cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
   if (int rc = launch_haar2d_fwd<3, TIn, H2D_MAX>(pb, X, nullptr, rowmax, st)) return rc;
   k_haar2d_row_scales<<<(unsigned)((pb.M + 255) / 256), 256, 0, st>>>(rowmax, pb.M, pb.n, pb.k_hi, (float)pb.qmax_hi,
@@ -1063,6 +1068,30 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
   float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
   float* yt = reinterpret_cast<float*>(base + wl.yt);
+  const bool patch_fits = (size_t)64 * K * (x_dtype == STAMP_BF16 ? 2 : 4) <= 224 * 1024;
+  if (pb.transform == STAMP_T_HAAR2D && pb.levels == 3 && pb.M % 256 == 0 && (!pb.act_zp || patch_fits)) {
+    // Fused route of the paper's LVM transform: one CTA per 8 x 8 patch finds the row maxima (or minima and maxima,
+    // for zero-point codes) and writes codes in patch order; the GEMM's epilogue inverts the four patches of its
+    // 256-token tile.
+    float* x_inv = T;               // the fp32 T of the general route is not materialised here: reuse its space
+    float* sx_epi = T + pb.M;
+    int* zp_epi = reinterpret_cast<int*>(T + 2 * pb.M);
+    const int8_t* w8p = nullptr;
+    if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8p, st))) return rc;
+    int* w_sum = nullptr;
+    if (pb.act_zp) {
+      w_sum = reinterpret_cast<int*>(base + wl.wsum);
+      if ((rc = run_weight_row_sums(w8p, N, K, w_sum, st))) return rc;
+    }
+    if (x_dtype == STAMP_BF16)
+      rc = run_quantize_haar2d_patch(pb, static_cast<const __nv_bfloat16*>(X), rowmax, x_scale, x_inv, a8, sx_epi, zp_epi,
+                                     w8p, st);
+    else
+      rc = run_quantize_haar2d_patch(pb, static_cast<const float*>(X), rowmax, x_scale, x_inv, a8, sx_epi, zp_epi, w8p, st);
+    if (rc) return rc;
+    return launch_gemm(a8, w8p, pb.M, N, K, sx_epi, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR2D_BF16 : EPI_HAAR2D_F32,
+                       st, bias, nullptr, 0, pb.act_zp ? zp_epi : nullptr, w_sum, pb.grid_w, pb.n);
+  }
   if (pb.act_zp) {
     // zero-point codes: transform, min-max quantizer, GEMM with the zero-point term in its epilogue, inverse
     int* x_zero = reinterpret_cast<int*>(base + wl.xzero);
@@ -1077,21 +1106,6 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
                           w_sum)))
       return rc;
     return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
-  }
-  if (pb.transform == STAMP_T_HAAR2D && pb.levels == 3 && pb.M % 256 == 0) {
-    // Fused route of the paper's LVM transform: two passes over X (row maxima; codes in patch order, the second
-    // pass reading X from L2), then the GEMM whose epilogue inverts the four 8 x 8 patches of its 256-token tile.
-    float* x_inv = T;               // the fp32 T of the general route is not materialised here: reuse its space
-    float* sx_epi = T + pb.M;
-    const int8_t* w8p = nullptr;
-    if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8p, st))) return rc;
-    if (x_dtype == STAMP_BF16)
-      rc = run_quantize_haar2d_patch(pb, static_cast<const __nv_bfloat16*>(X), rowmax, x_scale, x_inv, a8, sx_epi, w8p, st);
-    else
-      rc = run_quantize_haar2d_patch(pb, static_cast<const float*>(X), rowmax, x_scale, x_inv, a8, sx_epi, w8p, st);
-    if (rc) return rc;
-    return launch_gemm(a8, w8p, pb.M, N, K, sx_epi, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR2D_BF16 : EPI_HAAR2D_F32,
-                       st, bias, nullptr, 0, nullptr, nullptr, pb.grid_w, pb.n);
   }
   CqChoice cc;
   const bool have_cq = (pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc);

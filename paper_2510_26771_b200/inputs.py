@@ -206,6 +206,12 @@ def config_dit_proj_2d() -> LayerConfig:
     return dataclasses.replace(config_dit_proj(), name="dit_attn_proj_2d", transform=T_HAAR2D, levels=3)
 
 
+def config_dit_proj_2d_zp() -> LayerConfig:
+    """The paper's LVM activation setting in full: 3-level 2-D Haar over the patch grid, 64 low-pass tokens at
+    8 bits, zero-point (asymmetric, min-max) codes."""
+    return dataclasses.replace(config_dit_proj_2d(), name="dit_attn_proj_2d_zp", zero_point=True)
+
+
 def config_llm_down() -> LayerConfig:
     return LayerConfig("llm_down_proj", B=4, L=4096, K=14336, N=4096, dtype=BF16, transform=T_DCT2,
                        block=256, levels=0, k_hi=16, seed=3, recipe="ar1_student", rho=0.9,
@@ -225,7 +231,7 @@ def config_sweep(L: int, D: int, levels: int = 0) -> LayerConfig:
 
 def named_configs() -> dict:
     return {c.name: c for c in (config_tiny(), config_llm_up(), config_dit_proj(), config_llm_down(), config_dit_proj_2d(), config_llm_down_wht(),
-                                config_llm_up_zp())}
+                                config_llm_up_zp(), config_dit_proj_2d_zp())}
 
 
 def scaled(cfg: LayerConfig, **kw) -> LayerConfig:

@@ -38,6 +38,7 @@ FULL = {
     "dit_attn_proj_2d": gen.config_dit_proj_2d(),
     "llm_down_proj_wht": gen.config_llm_down_wht(),
     "llm_mlp_up_zp": gen.config_llm_up_zp(),
+    "dit_attn_proj_2d_zp": gen.config_dit_proj_2d_zp(),
     "sweep_L512_D2048": gen.config_sweep(512, 2048),
     "sweep_L8192_D4096": gen.config_sweep(8192, 4096),
     "sweep_L32768_D8192": gen.config_sweep(32768, 8192),
