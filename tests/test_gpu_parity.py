@@ -320,3 +320,28 @@ def test_edge_cases(st, oracle):
     Xz = torch.zeros((1, cfg.L, cfg.K), device="cuda")
     q_hi, q_lo, xs = st.stamp_quantize(c, Xz, ws)
     assert torch.all(xs == 1.0) and not q_hi.any() and not q_lo.any()
+
+
+def test_zero_activations_give_the_bias_on_every_route(st):
+    """All-zero input: every row has scale 1 (range 0) and codes 0 (stored -2^(b-1) with zero points), so the
+    layer returns the bias exactly -- on the fused Haar route (with rows above the GEMM tiles), the fused 2-D
+    route with symmetric and with zero-point codes, the tensor-core DCT route and the general zero-point route."""
+    import torch
+    routes = {
+        "haar_tiled": (gen.scaled(gen.config_llm_up(), B=1, L=1024, K=256, N=136), False),
+        "haar2d_patch": (gen.scaled(gen.config_dit_proj_2d(), B=1, L=1024, K=256, N=136, grid=32, k_hi=16), False),
+        "haar2d_patch_zp": (gen.scaled(gen.config_dit_proj_2d(), B=1, L=1024, K=256, N=136, grid=32, k_hi=16), True),
+        "dct_tensor": (gen.scaled(gen.config_llm_down(), B=1, L=512, K=256, N=192), False),
+        "haar_zp_general": (gen.scaled(gen.config_llm_up(), B=1, L=512, K=256, N=136), True),
+    }
+    for name, (cfg, zp) in routes.items():
+        c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid, zero_point=zp)
+        W, bias = gen.make_weight(cfg), gen.make_bias(cfg)
+        wq, wsc = st.stamp_quantize_weights(c, H.to_device(W, cfg.dtype))
+        bd = torch.from_numpy(bias).cuda()
+        ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+        Xz = torch.zeros((cfg.B, cfg.L, cfg.K), dtype=torch.bfloat16, device="cuda")
+        Y = st.stamp_linear_fused(c, Xz, wq, st.W_PACKED4, wsc, bd, ws)
+        assert torch.equal(Y.reshape(-1, cfg.N), bd.expand(cfg.M, cfg.N)), name
+        assert st.stamp_last_device_status() == 0
+
