@@ -4,7 +4,10 @@
 // 8 bits).  A transform block of n tokens is a grid of h = n / w rows by w columns in raster order.
 // One level maps every 2 x 2 cell (a b / c d) to
 //     LL = (a + b + c + d) / 2    LH = (a - b + c - d) / 2    HL = (a + b - c - d) / 2    HH = (a - b - c + d) / 2
-// (orthonormal; all factors are powers of two) and recurses on the LL grid.  Output order:
+// (orthonormal; all factors are powers of two) and recurses on the LL grid.  The details are evaluated as sums of
+// DIFFERENCES of neighbours, e.g. HL = ((a - c) + (b - d)) / 2: on activations with a large common offset the
+// differences are exact in fp32 and the result keeps its relative accuracy, which (a + b) - (c + d) would lose.
+// Output order:
 //     [LL_l | LH_l | HL_l | HH_l | LH_(l-1) | HL_(l-1) | HH_(l-1) | ... | LH_1 | HL_1 | HH_1],
 // each band in raster order of its (h >> level) x (w >> level) grid.
 //
@@ -111,7 +114,7 @@ __global__ void __launch_bounds__(128) k_haar2d_fwd(const TIn* __restrict__ in, 
           const int idx = base + 3 * ((y >> l) * (S >> l) + (x >> l));
           v[y][x] = make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y)));
           emit(haar2d_row(n, w, l, 0, gy, gx), idx, l, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-          emit(haar2d_row(n, w, l, 1, gy, gx), idx + 1, l, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+          emit(haar2d_row(n, w, l, 1, gy, gx), idx + 1, l, make_float2(0.5f * ((a.x - cc.x) + (b.x - d.x)), 0.5f * ((a.y - cc.y) + (b.y - d.y))));
           emit(haar2d_row(n, w, l, 2, gy, gx), idx + 2, l, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
         }
     }
@@ -165,7 +168,7 @@ __device__ __forceinline__ void haar2d_patch_sweep(const TIn* xs, int K, int c, 
           const int idx = 16 + 3 * ((2 * qy + cy) * 4 + (2 * qx + cx));
           ll1[cy][cx] = make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y)));
           emit(idx, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-          emit(idx + 1, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+          emit(idx + 1, make_float2(0.5f * ((a.x - cc.x) + (b.x - d.x)), 0.5f * ((a.y - cc.y) + (b.y - d.y))));
           emit(idx + 2, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
         }
       {                                       // level 2: cell (qy, qx) of the patch's 2 x 2 cells
@@ -177,7 +180,7 @@ __device__ __forceinline__ void haar2d_patch_sweep(const TIn* xs, int K, int c, 
         if (q == 2) ll2_2 = s4;
         if (q == 3) ll2_3 = s4;
         emit(idx, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-        emit(idx + 1, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+        emit(idx + 1, make_float2(0.5f * ((a.x - cc.x) + (b.x - d.x)), 0.5f * ((a.y - cc.y) + (b.y - d.y))));
         emit(idx + 2, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
       }
     }
@@ -185,7 +188,7 @@ __device__ __forceinline__ void haar2d_patch_sweep(const TIn* xs, int K, int c, 
       const float2 a = ll2_0, b = ll2_1, cc = ll2_2, d = ll2_3;
       emit(0, make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y))));
       emit(1, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-      emit(2, make_float2(0.5f * ((a.x + b.x) - (cc.x + d.x)), 0.5f * ((a.y + b.y) - (cc.y + d.y))));
+      emit(2, make_float2(0.5f * ((a.x - cc.x) + (b.x - d.x)), 0.5f * ((a.y - cc.y) + (b.y - d.y))));
       emit(3, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
     }
 }

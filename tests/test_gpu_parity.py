@@ -80,6 +80,12 @@ CASES = {
     # oblong grid (32 wide, 16 high), fp32 input, ragged channel tile: the fused patch-order route again
     "haar2d_oblong": gen.scaled(gen.config_dit_proj_2d(), B=3, L=512, K=128, N=72, grid=32, levels=3, k_hi=8,
                                 dtype=gen.F32, recipe="ar1"),
+    # the widest patches that still fit in shared memory: 1792 bf16 channels, 896 fp32 channels (224 KB each)
+    "haar2d_max_bf16": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=1792, N=64, grid=16, levels=3, k_hi=4),
+    # (an AR(1) field: the smooth random field of the patch-grid recipe, kept in fp32, has HH rows 1e6 times
+    #  smaller than the values they are differences of, beyond what fp32 butterflies resolve to 1e-5 of the row)
+    "haar2d_max_fp32": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=896, N=64, grid=16, levels=3, k_hi=4,
+                                  dtype=gen.F32, recipe="ar1"),
     # a patch (64 tokens x 2048 channels) that does not fit in shared memory: row maxima and codes in separate launches
     "haar2d_wide_k": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=2048, N=64, grid=16, levels=3, k_hi=4),
     # two levels only: no cluster tree, approximation rows quantized by the same kernel
