@@ -351,3 +351,31 @@ def test_zero_activations_give_the_bias_on_every_route(st):
         assert torch.equal(Y.reshape(-1, cfg.N), bd.expand(cfg.M, cfg.N)), name
         assert st.stamp_last_device_status() == 0
 
+
+def test_fused_call_can_be_captured_in_a_cuda_graph(st):
+    """The one-call layer makes no synchronising call and allocates nothing, so a stream capture records it
+    (dependent launches included) and the replayed graph gives the same output as the direct call."""
+    import torch
+    for cfg in (gen.scaled(gen.config_llm_up(), B=1, L=1024, K=256, N=264),
+                gen.scaled(gen.config_dit_proj_2d(), B=1, L=1024, K=256, N=136, grid=32, k_hi=16)):
+        c = _cfg_struct(st, cfg)
+        X, W, bias = gen.make_activation(cfg), gen.make_weight(cfg), gen.make_bias(cfg)
+        Xd, Wd, bd = H.to_device(X, cfg.dtype), H.to_device(W, cfg.dtype), torch.from_numpy(bias).cuda()
+        wq, wsc = st.stamp_quantize_weights(c, Wd)
+        w8 = st.stamp_prepare_weights(c, wq)
+        ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+        want = st.stamp_linear_fused(c, Xd, w8, st.W_INT8, wsc, bd, ws, out_dtype=torch.bfloat16).clone()
+        out = torch.zeros_like(want)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                st.stamp_linear_fused(c, Xd, w8, st.W_INT8, wsc, bd, ws, out=out)
+        for _ in range(3):
+            out.zero_()
+            graph.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(out, want)
+        assert st.stamp_last_device_status() == 0
+
