@@ -190,7 +190,7 @@ int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float*
 /*
  * The whole Algorithm in one call: Y = L^-1( Q(L X) Q(W)^T ) + bias.  Intermediates (codes,
  * scales, transformed-domain output) live in the workspace only.
-  * The call enqueues kernels on `stream` only (no synchronisation, no allocation): it may be recorded in a CUDA
+ * The call enqueues kernels on `stream` only (no synchronisation, no allocation): it may be recorded in a CUDA
  * graph by stream capture once it has run once outside a capture (function attributes are set on first use).
  */
 int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, const void* w, int w_format,
