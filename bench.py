@@ -196,6 +196,9 @@ def main():
     ap.add_argument("--impl", default="native", choices=("native", "reference"))
     ap.add_argument("--workload", default="llm_mlp_up")
     ap.add_argument("--out-dtype", default="bf16", choices=("bf16", "f32"))
+    ap.add_argument("--levels", type=int, default=None,
+                    help="override the workload's Haar level count (0 = full depth) and, with --k-hi, its 8-bit rows")
+    ap.add_argument("--k-hi", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true",
                     help="timed region only (no side measurements, no CPU baseline): for profiler captures")
@@ -203,6 +206,10 @@ def main():
                     help="with --quick: the call each step makes (the whole layer, or one of its passes alone)")
     args = ap.parse_args()
     cfg = workloads()[args.workload]
+    if args.levels is not None:
+        cfg = gen.scaled(cfg, levels=args.levels)
+    if args.k_hi is not None:
+        cfg = gen.scaled(cfg, k_hi=args.k_hi)
 
     if args.impl == "reference":
         run_reference(args, cfg)
