@@ -146,51 +146,64 @@ struct Haar2dPatchParams {
 };
 
 // One sweep over a staged patch xs [64 tokens][K] for the channel pair starting at c: emit(idx, value) is called
-// once per coefficient, idx in the patch order described at Haar2dMode.
+// once per coefficient, idx in the patch order described at Haar2dMode.  The values are UN-NORMALISED: 2^l times
+// the level-l coefficient (sums and differences only, two channels per packed fp32x2 instruction; the factor is an
+// exact power of two that the caller folds into its scales).
+struct Haar2dCell {
+  float2 ll, lh, hl, hh;
+};
+__device__ __forceinline__ Haar2dCell haar2d_cell(float2 a, float2 b, float2 c, float2 d) {
+  const float2 s0 = __fadd2_rn(a, b), s1 = ptx::fsub2_rn(a, b), s2 = __fadd2_rn(c, d), s3 = ptx::fsub2_rn(c, d);
+  Haar2dCell r;
+  r.ll = __fadd2_rn(s0, s2);
+  r.lh = __fadd2_rn(s1, s3);
+  r.hl = __fadd2_rn(ptx::fsub2_rn(a, c), ptx::fsub2_rn(b, d));   // differences of neighbours first
+  r.hh = ptx::fsub2_rn(s1, s3);
+  return r;
+}
 template <typename TIn, typename F>
 __device__ __forceinline__ void haar2d_patch_sweep(const TIn* xs, int K, int c, F&& emit) {
-    // (the quadrant loop stays rolled: unrolled, the compiler hoists all 64 loads and spills)
-    float2 ll2_0 = make_float2(0.f, 0.f), ll2_1 = ll2_0, ll2_2 = ll2_0, ll2_3 = ll2_0;
+  // (the quadrant loop stays rolled: unrolled, the compiler hoists all 64 loads and spills)
+  float2 ll2_0 = make_float2(0.f, 0.f), ll2_1 = ll2_0, ll2_2 = ll2_0, ll2_3 = ll2_0;
 #pragma unroll 1
-    for (int q = 0; q < 4; ++q) {             // quadrant (qy, qx) of 4 x 4 tokens
-      const int qy = q >> 1, qx = q & 1;
-      float2 v[4][4];
+  for (int q = 0; q < 4; ++q) {             // quadrant (qy, qx) of 4 x 4 tokens
+    const int qy = q >> 1, qx = q & 1;
+    float2 v[4][4];
 #pragma unroll
-      for (int y = 0; y < 4; ++y)
+    for (int y = 0; y < 4; ++y)
 #pragma unroll
-        for (int x = 0; x < 4; ++x) v[y][x] = load2(xs + (long)((qy * 4 + y) * 8 + qx * 4 + x) * K + c);
-      float2 ll1[2][2];
+      for (int x = 0; x < 4; ++x) v[y][x] = load2(xs + (long)((qy * 4 + y) * 8 + qx * 4 + x) * K + c);
+    float2 ll1[2][2];
 #pragma unroll
-      for (int cy = 0; cy < 2; ++cy)
+    for (int cy = 0; cy < 2; ++cy)
 #pragma unroll
-        for (int cx = 0; cx < 2; ++cx) {      // level 1: cell (2 qy + cy, 2 qx + cx) of the patch's 4 x 4 cells
-          const float2 a = v[2 * cy][2 * cx], b = v[2 * cy][2 * cx + 1], cc = v[2 * cy + 1][2 * cx], d = v[2 * cy + 1][2 * cx + 1];
-          const int idx = 16 + 3 * ((2 * qy + cy) * 4 + (2 * qx + cx));
-          ll1[cy][cx] = make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y)));
-          emit(idx, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-          emit(idx + 1, make_float2(0.5f * ((a.x - cc.x) + (b.x - d.x)), 0.5f * ((a.y - cc.y) + (b.y - d.y))));
-          emit(idx + 2, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
-        }
-      {                                       // level 2: cell (qy, qx) of the patch's 2 x 2 cells
-        const float2 a = ll1[0][0], b = ll1[0][1], cc = ll1[1][0], d = ll1[1][1];
-        const int idx = 4 + 3 * q;
-        const float2 s4 = make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y)));
-        if (q == 0) ll2_0 = s4;
-        if (q == 1) ll2_1 = s4;
-        if (q == 2) ll2_2 = s4;
-        if (q == 3) ll2_3 = s4;
-        emit(idx, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-        emit(idx + 1, make_float2(0.5f * ((a.x - cc.x) + (b.x - d.x)), 0.5f * ((a.y - cc.y) + (b.y - d.y))));
-        emit(idx + 2, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
+      for (int cx = 0; cx < 2; ++cx) {      // level 1: cell (2 qy + cy, 2 qx + cx) of the patch's 4 x 4 cells
+        const Haar2dCell r = haar2d_cell(v[2 * cy][2 * cx], v[2 * cy][2 * cx + 1], v[2 * cy + 1][2 * cx], v[2 * cy + 1][2 * cx + 1]);
+        const int idx = 16 + 3 * ((2 * qy + cy) * 4 + (2 * qx + cx));
+        ll1[cy][cx] = r.ll;
+        emit(idx, r.lh);
+        emit(idx + 1, r.hl);
+        emit(idx + 2, r.hh);
       }
+    {                                       // level 2: cell (qy, qx) of the patch's 2 x 2 cells
+      const Haar2dCell r = haar2d_cell(ll1[0][0], ll1[0][1], ll1[1][0], ll1[1][1]);
+      const int idx = 4 + 3 * q;
+      if (q == 0) ll2_0 = r.ll;
+      if (q == 1) ll2_1 = r.ll;
+      if (q == 2) ll2_2 = r.ll;
+      if (q == 3) ll2_3 = r.ll;
+      emit(idx, r.lh);
+      emit(idx + 1, r.hl);
+      emit(idx + 2, r.hh);
     }
-    {                                         // level 3
-      const float2 a = ll2_0, b = ll2_1, cc = ll2_2, d = ll2_3;
-      emit(0, make_float2(0.5f * ((a.x + b.x) + (cc.x + d.x)), 0.5f * ((a.y + b.y) + (cc.y + d.y))));
-      emit(1, make_float2(0.5f * ((a.x - b.x) + (cc.x - d.x)), 0.5f * ((a.y - b.y) + (cc.y - d.y))));
-      emit(2, make_float2(0.5f * ((a.x - cc.x) + (b.x - d.x)), 0.5f * ((a.y - cc.y) + (b.y - d.y))));
-      emit(3, make_float2(0.5f * ((a.x - b.x) - (cc.x - d.x)), 0.5f * ((a.y - b.y) - (cc.y - d.y))));
-    }
+  }
+  {                                         // level 3
+    const Haar2dCell r = haar2d_cell(ll2_0, ll2_1, ll2_2, ll2_3);
+    emit(0, r.ll);
+    emit(1, r.lh);
+    emit(2, r.hl);
+    emit(3, r.hh);
+  }
 }
 
 // Order-preserving map of a float onto a signed integer (for integer min / max reductions), and back.
@@ -207,8 +220,9 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
   extern __shared__ __align__(16) uint8_t h2p_smem[];
   __shared__ unsigned s_max[64];                    // |t| maxima as bit patterns; ZP: maxima as order keys
   __shared__ int s_min[64];                         // ZP: minima as order keys
-  __shared__ float4 s_tab[64];                      // {scale, 1 / scale, qmax, -} per coefficient of the patch
-                                                    // ZP: {scale, 1 / scale, top code, zero point} (last two as int bits)
+  // per coefficient of the patch, for the un-normalised values of the sweep (2^l times the coefficient):
+  // {-scale * 2^l, 2^-l / scale, qmax, -};  ZP: {-scale * 2^l, 2^-l / scale, top code, zero point} (last two as int bits)
+  __shared__ float4 s_tab[64];
   __shared__ __align__(8) uint64_t s_bar;
   __shared__ uint32_t s_abort;
   TIn* xs = reinterpret_cast<TIn*>(h2p_smem);      // [64 tokens (patch raster)][K]
@@ -284,25 +298,27 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
     const int gy = (py << (3 - l)) + cy, gx = (px << (3 - l)) + cx;
     const int row = haar2d_row(n, w, l, band, gy, gx);
     float scale;
+    const float up = static_cast<float>(1 << l), down = 1.0f / up;   // the sweep's values carry the factor 2^l
     if (!ZP) {
       const float qmax = row < p.k_hi ? p.qmax_hi : p.qmax_lo;
-      const float amax = __uint_as_float(s_max[tid]);
+      const float amax = __uint_as_float(s_max[tid]) * down;
       scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
-      s_tab[tid] = make_float4(scale, __fdiv_rn(1.0f, scale), qmax, 0.f);
+      s_tab[tid] = make_float4(-scale * up, __fdiv_rn(1.0f, scale) * down, qmax, 0.f);
     } else {
       const int half = row < p.k_hi ? 128 : 8;
       const int top = 2 * half - 1;
-      const float mx = float_from_order_key(static_cast<int>(s_max[tid])), mn = float_from_order_key(s_min[tid]);
+      const float mx = float_from_order_key(static_cast<int>(s_max[tid])) * down;
+      const float mn = float_from_order_key(s_min[tid]) * down;
       scale = __fdiv_rn(mx - mn, static_cast<float>(top));
       if (!(scale > 0.f)) scale = 1.0f;
       float zf = rintf(__fdiv_rn(-mn, scale));
       zf = fminf(fmaxf(zf, -1073741824.0f), 1073741824.0f);
       const int z = static_cast<int>(zf);
-      s_tab[tid] = make_float4(scale, __fdiv_rn(1.0f, scale), __int_as_float(top), __int_as_float(z));
+      s_tab[tid] = make_float4(-scale * up, __fdiv_rn(1.0f, scale) * down, __int_as_float(top), __int_as_float(z));
       p.zp_epi[pt * 64 + tid] = z - half;
     }
     p.x_scale[blk * n + row] = scale;
-    p.sx_epi[pt * 64 + tid] = scale * (1.0f / static_cast<float>(1 << l));
+    p.sx_epi[pt * 64 + tid] = scale * down;
   }
   __syncthreads();
   // ---- pass 2: codes
@@ -310,9 +326,12 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
   for (int c2 = tid; c2 < K / 2; c2 += H2P_THREADS) {
     const int c = 2 * c2;
     haar2d_patch_sweep(xs, K, c, [&](int idx, float2 t) {
-      const float4 tb = s_tab[idx];               // scale, 1 / scale, qmax
-      const float a0 = t.x * tb.y, a1 = t.y * tb.y;
-      const float r0 = fmaf(fmaf(-a0, tb.x, t.x), tb.y, a0), r1 = fmaf(fmaf(-a1, tb.x, t.y), tb.y, a1);   // t / scale
+      const float4 tb = s_tab[idx];
+      // t / scale by reciprocal and one Newton step, both channels per instruction
+      const float2 ninv = make_float2(tb.y, tb.y);
+      const float2 a = __fmul2_rn(t, ninv);
+      const float2 r = __ffma2_rn(__ffma2_rn(a, make_float2(tb.x, tb.x), t), ninv, a);
+      const float r0 = r.x, r1 = r.y;
       if (!ZP) {
         // clamp, then round to nearest even by adding 1.5 * 2^23: the code is the low byte of the sum's bit pattern
         const float q0 = fminf(fmaxf(r0, -tb.z), tb.z) + 12582912.0f;
