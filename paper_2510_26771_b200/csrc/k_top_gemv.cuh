@@ -19,7 +19,7 @@ constexpr int TOPG_CH_PER_WARP = 4;
 // R = total top rows (nseq * rows_per_block), rows_per_block = 2^top_levels.
 //   codes [R, K] int8, x_scale [R], w8 [n_out, K] int8, a8v [R, n_out] float
 template <int R>
-__global__ void __launch_bounds__(TOPG_THREADS, (R <= 8 ? 3 : 2)) k_top_gemv(const int8_t* __restrict__ codes,
+__global__ void __launch_bounds__(TOPG_THREADS, (R <= 4 ? 3 : (R <= 8 ? 4 : 2))) k_top_gemv(const int8_t* __restrict__ codes,
                                                            const float* __restrict__ x_scale,
                                                            const int8_t* __restrict__ w8, int K, int n_out,
                                                            int top_levels, float* __restrict__ a8v) {
@@ -39,21 +39,23 @@ __global__ void __launch_bounds__(TOPG_THREADS, (R <= 8 ? 3 : 2)) k_top_gemv(con
   for (int c = 0; c < TOPG_CH_PER_WARP; ++c)
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[c][r] = 0;
-  // Two 512-byte steps of every channel per iteration: the kernel is bound by the weight bytes in flight per SM
-  // (four channels x two 16-byte loads per lane), not by arithmetic; four channels per warp keep the shared-memory
-  // reads of the codes (R x 16 bytes per lane and step) at twice the weight bytes instead of four times.
-  for (int k0 = lane * 16; k0 < K; k0 += 2 * 32 * 16) {
-    const bool second = k0 + 32 * 16 < K;
-    uint4 w[TOPG_CH_PER_WARP][2];
+  // The kernel is bound by the weight bytes in flight per SM, not by arithmetic.  With few rows (R <= 4) the
+  // accumulators leave room for two 512-byte steps of every channel per iteration (eight 16-byte loads per lane in
+  // flight: measured 0.077 -> 0.060 ms per layer step at R = 2, K = 8192); from R = 8 on one step per iteration is
+  // as fast or faster (the second set of loads would cost occupancy).
+  constexpr int NSTEP = (R <= 4) ? 2 : 1;
+  for (int k0 = lane * 16; k0 < K; k0 += NSTEP * 32 * 16) {
+    const bool second = NSTEP == 2 && k0 + 32 * 16 < K;
+    uint4 w[TOPG_CH_PER_WARP][NSTEP];
 #pragma unroll
     for (int c = 0; c < TOPG_CH_PER_WARP; ++c) {
       const int ch = min(ch0 + c, n_out - 1);   // a ragged last group re-reads the last channel, stores are guarded
       const uint4* wp = reinterpret_cast<const uint4*>(w8 + (long)ch * K + k0);
       w[c][0] = __ldg(wp);
-      w[c][1] = second ? __ldg(wp + 32) : make_uint4(0u, 0u, 0u, 0u);
+      if (NSTEP == 2) w[c][NSTEP - 1] = second ? __ldg(wp + 32) : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < NSTEP; ++u) {
       if (u == 1 && !second) break;
 #pragma unroll
       for (int r = 0; r < R; ++r) {
