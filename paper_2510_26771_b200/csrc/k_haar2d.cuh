@@ -141,6 +141,11 @@ struct Haar2dPatchParams {
   float* sx_epi;         // [M] patch order, scale * 2^-l
   float* x_scale;        // [M] logical order
   int* zp_epi;           // [M] patch order: zero point of every row's stored codes (zero-point variant only)
+  // zero-point variant: the weight row sums of the correction term (sum over k of w8[n, k]) are taken here as well,
+  // one row per warp, while the patch's copies are in flight (saves a launch); rs_rows = 0 for none
+  const int8_t* rs_w8;   // [rs_rows, K]
+  int rs_rows;
+  int* rs_out;           // [rs_rows]
   const uint8_t* pf_base; // optional region (the layer's weight codes) to pull towards L2 for the GEMM that follows
   long pf_bytes;          // multiple of 16, 0 for none
 };
@@ -257,6 +262,17 @@ __global__ void __launch_bounds__(H2P_THREADS, 1) k_haar2d_patch_quant(const Haa
     ptx::mbar_arrive_expect_tx(&s_bar, 8u * row_bytes);
 #pragma unroll 1
     for (int y = 0; y < 8; ++y) ptx::bulk_load(xs + (long)y * 8 * K, src0 + (long)y * w * K, row_bytes, &s_bar);
+  }
+  if (ZP && p.rs_rows > 0) {
+    constexpr int nwarp = H2P_THREADS / 32;
+    for (int r = blockIdx.x * nwarp + (tid >> 5); r < p.rs_rows; r += gridDim.x * nwarp) {
+      const int* src = reinterpret_cast<const int*>(p.rs_w8 + (long)r * K);
+      int acc = 0;
+      for (int k4 = tid & 31; k4 < K / 4; k4 += 32) acc = __dp4a(__ldg(src + k4), 0x01010101, acc);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if ((tid & 31) == 0) p.rs_out[r] = acc;
+    }
   }
   if (!ptx::mbar_wait_bounded(&s_bar, 0u, &s_abort, 2000000000LL)) {
     // the copies did not land within about a second: record it and leave the patch unwritten

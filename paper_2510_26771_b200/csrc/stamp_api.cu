@@ -421,11 +421,12 @@ static int launch_haar2d_patch(const Haar2dPatchParams& pp, long npatch, size_t 
 // patch (64 tokens x K channels) fits in shared memory; otherwise row maxima, scales, then codes in three launches.
 template <typename TIn>
 static int run_quantize_haar2d_patch(const Problem& pb, const TIn* X, unsigned* rowmax, float* x_scale, float* x_inv,
-                                     int8_t* a8, float* sx_epi, int* zp_epi, const int8_t* w8, cudaStream_t st) {
+                                     int8_t* a8, float* sx_epi, int* zp_epi, const int8_t* w8, int* w_sum,
+                                     cudaStream_t st) {
   const size_t smem = (size_t)64 * pb.K * sizeof(TIn);
   if (smem <= 224 * 1024) {
     Haar2dPatchParams pp{X, pb.n, pb.grid_w, pb.K, pb.k_hi, (float)pb.qmax_hi, (float)pb.qmax_lo, a8, sx_epi, x_scale,
-                         zp_epi, nullptr, 0};
+                         zp_epi, pb.act_zp ? w8 : nullptr, pb.act_zp ? pb.N : 0, w_sum, nullptr, 0};
     if ((size_t)pb.N * pb.K <= (size_t)24 << 20) {   // small weight matrix: have it in L2 when the GEMM starts
       pp.pf_base = reinterpret_cast<const uint8_t*>(w8);
       pp.pf_bytes = (long)pb.N * pb.K;
@@ -1078,16 +1079,14 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     int* zp_epi = reinterpret_cast<int*>(T + 2 * pb.M);
     const int8_t* w8p = nullptr;
     if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8p, st))) return rc;
-    int* w_sum = nullptr;
-    if (pb.act_zp) {
-      w_sum = reinterpret_cast<int*>(base + wl.wsum);
-      if ((rc = run_weight_row_sums(w8p, N, K, w_sum, st))) return rc;
-    }
+    // (zero-point codes: the patch kernel also takes the weight row sums of the correction term)
+    int* w_sum = pb.act_zp ? reinterpret_cast<int*>(base + wl.wsum) : nullptr;
     if (x_dtype == STAMP_BF16)
       rc = run_quantize_haar2d_patch(pb, static_cast<const __nv_bfloat16*>(X), rowmax, x_scale, x_inv, a8, sx_epi, zp_epi,
-                                     w8p, st);
+                                     w8p, w_sum, st);
     else
-      rc = run_quantize_haar2d_patch(pb, static_cast<const float*>(X), rowmax, x_scale, x_inv, a8, sx_epi, zp_epi, w8p, st);
+      rc = run_quantize_haar2d_patch(pb, static_cast<const float*>(X), rowmax, x_scale, x_inv, a8, sx_epi, zp_epi, w8p,
+                                     w_sum, st);
     if (rc) return rc;
     return launch_gemm(a8, w8p, pb.M, N, K, sx_epi, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR2D_BF16 : EPI_HAAR2D_F32,
                        st, bias, nullptr, 0, pb.act_zp ? zp_epi : nullptr, w_sum, pb.grid_w, pb.n);
