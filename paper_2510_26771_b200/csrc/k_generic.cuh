@@ -212,12 +212,26 @@ __global__ void __launch_bounds__(256) k_quant_rows(const float* __restrict__ T,
 // signed byte / nibble formats (and the same signed tensor-core operand) as the symmetric codes; the
 // zero point written out is that of the stored code, zc = z - 2^(b-1), and t ~ s * (c - zc).
 // One CTA per materialised row; the row is read twice (min/max, then codes), the second time from L2.
+// CTAs past the `rows` token rows take the weight row sums of the correction term instead (eight weight rows per
+// CTA, one per warp: rs_out[j] = sum_k rs_w8[j, k]), so that the two independent reads share one launch.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_quant_rows_zp(const float* __restrict__ T, int K, int n, int k_hi,
+__global__ void __launch_bounds__(256) k_quant_rows_zp(const float* __restrict__ T, long rows, int K, int n, int k_hi,
                                                        int8_t* __restrict__ a8, int8_t* __restrict__ q_hi,
                                                        uint8_t* __restrict__ q_lo, float* __restrict__ x_scale,
-                                                       int* __restrict__ x_zero) {
+                                                       int* __restrict__ x_zero, const int8_t* __restrict__ rs_w8,
+                                                       int rs_rows, int* __restrict__ rs_out) {
   __shared__ float red_mn[8], red_mx[8];
+  if (blockIdx.x >= rows) {
+    const int j = static_cast<int>(blockIdx.x - rows) * 8 + (threadIdx.x >> 5);
+    if (j >= rs_rows) return;
+    const int* src = reinterpret_cast<const int*>(rs_w8 + (long)j * K);
+    int acc = 0;
+    for (int k4 = threadIdx.x & 31; k4 < K / 4; k4 += 32) acc = __dp4a(__ldg(src + k4), 0x01010101, acc);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0) rs_out[j] = acc;
+    return;
+  }
   const long r = blockIdx.x;
   const long s = r / n;
   const int i = static_cast<int>(r - s * n);

@@ -570,10 +570,14 @@ static int run_quant_rows(const Problem& pb, const float* T, const unsigned* row
 }
 
 // Zero-point codes from materialised T (all rows of every block).
+// (w8 / w_sum given: the same launch also takes the weight row sums, in CTAs of its own.)
 static int run_quant_rows_zp(const Problem& pb, const float* T, int8_t* a8, void* q_hi, void* q_lo, float* x_scale,
-                             int* x_zero, cudaStream_t st) {
-  k_quant_rows_zp<<<(unsigned)pb.M, 256, 0, st>>>(T, pb.K, pb.n, pb.k_hi, a8, static_cast<int8_t*>(q_hi),
-                                                   static_cast<uint8_t*>(q_lo), x_scale, x_zero);
+                             int* x_zero, cudaStream_t st, const int8_t* w8 = nullptr, int* w_sum = nullptr) {
+  const int rs_rows = (w8 && w_sum) ? pb.N : 0;
+  k_quant_rows_zp<<<(unsigned)(pb.M + (rs_rows + 7) / 8), 256, 0, st>>>(T, pb.M, pb.K, pb.n, pb.k_hi, a8,
+                                                                         static_cast<int8_t*>(q_hi),
+                                                                         static_cast<uint8_t*>(q_lo), x_scale, x_zero, w8,
+                                                                         rs_rows, w_sum);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
 }
@@ -1097,10 +1101,9 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     int* w_sum = reinterpret_cast<int*>(base + wl.wsum);
     if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
       return rc;
-    if ((rc = run_quant_rows_zp(pb, T, a8, nullptr, nullptr, x_scale, x_zero, st))) return rc;
     const int8_t* w8z = nullptr;
     if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8z, st))) return rc;
-    if ((rc = run_weight_row_sums(w8z, N, K, w_sum, st))) return rc;
+    if ((rc = run_quant_rows_zp(pb, T, a8, nullptr, nullptr, x_scale, x_zero, st, w8z, w_sum))) return rc;
     if ((rc = launch_gemm(a8, w8z, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_ZP_F32, st, nullptr, nullptr, 0, x_zero,
                           w_sum)))
       return rc;
