@@ -399,8 +399,20 @@ int oracle_bit_map(int L, int n, int k_hi, int bits_hi, int bits_lo, int32_t* bi
  * step; low-precision inputs (bf16 activations and weights) land EXACTLY on rounding
  * boundaries often (whenever absmax has a mantissa divisible by qmax), so the precision in
  * which the tie is seen decides the code, and fp32 is the precision of the scale itself.
+ * The other reading -- the quotient t_j / (double)scale evaluated and rounded in fp64 -- can be
+ * selected with oracle_set_rounding_decision(1); tests/test_oracle_pins.py counts how many codes
+ * the two readings disagree on for the named configurations.
  * bits_per_row has `period` entries and row r uses bits_per_row[r % period].
  * ------------------------------------------------------------------------------------------ */
+static int g_decide_fp64 = 0;
+
+/* 0 (default): rounding decision on the fp32 quotient; 1: on the fp64 quotient.  Returns the old value. */
+int oracle_set_rounding_decision(int fp64) {
+  int old = g_decide_fp64;
+  g_decide_fp64 = fp64 ? 1 : 0;
+  return old;
+}
+
 int oracle_quantize_rows(const double* T, long rows, int K, const int32_t* bits_per_row, int period,
                          float* scale, int8_t* codes) {
   if (period <= 0) return 1;
@@ -418,7 +430,7 @@ int oracle_quantize_rows(const double* T, long rows, int K, const int32_t* bits_
     if (!(s > 0.0f)) s = 1.0f; /* amax so small that the fp32 scale underflowed */
     scale[r] = s;
     for (int j = 0; j < K; ++j) {
-      float q = rintf((float)t[j] / s);
+      float q = g_decide_fp64 ? (float)nearbyint(t[j] / (double)s) : rintf((float)t[j] / s);
       if (q > qmaxf) q = qmaxf;
       if (q < -qmaxf) q = -qmaxf;
       codes[(size_t)r * K + j] = (int8_t)q;

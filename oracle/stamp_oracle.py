@@ -105,6 +105,12 @@ def bit_map(L: int, n: int, k_hi: int, bits_hi: int = 8, bits_lo: int = 4) -> np
     return bits
 
 
+def set_rounding_decision(fp64: bool) -> bool:
+    """Precision in which the symmetric quantizer takes its rounding decision: the fp32 quotient
+    (default) or the fp64 quotient.  Returns the previous setting."""
+    return bool(lib().oracle_set_rounding_decision(int(bool(fp64))))
+
+
 def quantize_rows(T: np.ndarray, bits_per_row: np.ndarray):
     """Per-row symmetric RTN quantizer.  T [rows, K] fp64; row r uses bits_per_row[r % len]."""
     T = np.ascontiguousarray(T, dtype=np.float64)

@@ -1,7 +1,11 @@
 """Pins for the CPU oracle: it is checked against what the paper and the mathematics fix,
 never against itself.  Every test names the passage it pins.  CPU only."""
+import importlib.util
 import math
 import os
+import subprocess
+import tempfile
+from fractions import Fraction
 
 import numpy as np
 import pytest
@@ -309,10 +313,23 @@ def _python_loop_layer(X, W, bias, n, levels, k_hi):
                 T[b0 + t][j] = v[t]
 
     def quant(row, qmax):
+        """Nearest of the 2 qmax + 1 levels s * k by brute force in exact rational arithmetic; a value closer
+        than 2^-20 (relative) to the midpoint of two levels is a tie at fp32 resolution and is reported in
+        `ties` instead of being decided here."""
         amax = max(abs(x) for x in row)
         s = float(np.float32(amax) / np.float32(qmax)) if amax > 0 else 1.0
-        # the rounding decision is taken in fp32 (np.rint: half to even)
-        return [max(-qmax, min(qmax, int(np.rint(np.float32(x) / np.float32(s))))) for x in row], s
+        sf = Fraction(s)
+        codes = []
+        for x in row:
+            xf = Fraction(x)
+            dist = sorted((abs(xf - sf * k), k) for k in range(-qmax, qmax + 1))
+            (d0, k0), (d1, _) = dist[0], dist[1]
+            if d1 - d0 <= sf * Fraction(1, 1 << 20) * max(1, abs(k0)):
+                ties.append((x, s))
+            codes.append(k0)
+        return codes, s
+
+    ties = []
 
     qs = [quant(T[i], 127 if (i % n) < k_hi else 7) for i in range(L)]
     ws = [quant(W[c], 7) for c in range(N)]
@@ -332,7 +349,7 @@ def _python_loop_layer(X, W, bias, n, levels, k_hi):
                 length *= 2
             for t in range(n):
                 Y[b0 + t][c] = v[t] + bias[c]
-    return np.array(Y), np.array([x[0] for x in qs]), np.array([x[1] for x in qs])
+    return np.array(Y), np.array([x[0] for x in qs]), np.array([x[1] for x in qs]), ties
 
 
 def test_layer_vs_python_loops(oracle):
@@ -345,8 +362,9 @@ def test_layer_vs_python_loops(oracle):
     W = (rng.standard_normal((N, K)) * 0.1).astype(np.float32)
     bias = rng.standard_normal(N).astype(np.float32)
     out = oracle.stamp_linear(X[None], W, bias, transform=T_HAAR, block=n, levels=levels, k_hi=k_hi)
-    Y, q, s = _python_loop_layer(X.astype(float).tolist(), W.astype(float).tolist(), bias.astype(float).tolist(),
-                                 n, levels, k_hi)
+    Y, q, s, ties = _python_loop_layer(X.astype(float).tolist(), W.astype(float).tolist(), bias.astype(float).tolist(),
+                                       n, levels, k_hi)
+    assert not ties          # no value of this input sits on a rounding boundary: the nearest level is unique
     assert np.array_equal(out["q"], q)
     assert np.allclose(out["x_scale"], s, rtol=1e-7)
     assert np.max(np.abs(out["Y"] - Y)) <= 1e-12 * np.max(np.abs(Y))
@@ -603,3 +621,145 @@ def test_asym_layer_composes_and_is_closer_than_symmetric_on_shifted_activations
     ea = np.linalg.norm(out["Y"] - ref) / np.linalg.norm(ref)
     es = np.linalg.norm(sym["Y"] - ref) / np.linalg.norm(ref)
     assert ea < es and ea < 0.2
+
+
+# --------------------------------------------------------------------------------------
+# The precision of the rounding decision (Sec. 2.1 fixes none): how often the two readings differ
+# --------------------------------------------------------------------------------------
+
+def _transformed(oracle, cfg):
+    X = gen.make_activation(cfg)
+    n = cfg.block_len
+    if cfg.transform == T_HAAR and n > 4096:
+        T = oracle.apply_csr(oracle.haar_matrix_csr(n, cfg.levels), n, X)
+    else:
+        T = oracle.apply_dense(oracle.transform_matrix(cfg.transform, n, cfg.levels, grid_w=cfg.grid), X)
+    return T.reshape(-1, cfg.K)
+
+
+ROUNDING_CASES = {
+    "tiny": gen.config_tiny(),
+    "llm_mlp_up": gen.config_llm_up(),
+    "dit_attn_proj": gen.config_dit_proj(),
+    "llm_down_proj_reduced": gen.scaled(gen.config_llm_down(), B=1, L=1024, K=2048),
+    "sweep_L2048_D2048": gen.config_sweep(2048, 2048),
+}
+
+
+@pytest.mark.parametrize("name", list(ROUNDING_CASES))
+def test_fp32_and_fp64_rounding_decisions_differ_only_at_fp32_ties(oracle, name):
+    """The quantizer's quotient t / s can be rounded to an integer from its fp32 or from its fp64 value.  The two
+    readings give different codes only where the fp32 quotient IS a half-integer (bf16 inputs make absmax / qmax land
+    there exactly) while the fp64 quotient of the same fp32 scale sits a hair beside it; the disagreement is one code
+    step.  The counts printed here are recorded with the reading taken (fp32, the precision of the scale)."""
+    cfg = ROUNDING_CASES[name]
+    T = _transformed(oracle, cfg)
+    bits = oracle.bit_map(cfg.L, cfg.block_len, cfg.k_hi)
+    assert oracle.set_rounding_decision(False) is False
+    q32, s32 = oracle.quantize_rows(T, bits)
+    oracle.set_rounding_decision(True)
+    try:
+        q64, s64 = oracle.quantize_rows(T, bits)
+    finally:
+        oracle.set_rounding_decision(False)
+    assert np.array_equal(s32, s64)
+    r, c = np.nonzero(q32 != q64)
+    print(f"[{name}] codes on which the fp32 and fp64 rounding decisions differ: {len(r)} of {q32.size} "
+          f"({len(r) / q32.size:.2e})")
+    if len(r):
+        assert np.abs(q32[r, c].astype(int) - q64[r, c].astype(int)).max() == 1
+        quo32 = T[r, c].astype(np.float32) / s32[r]
+        assert np.all(np.abs(quo32 - np.trunc(quo32)) == 0.5)          # an exact tie in fp32 ...
+        quo64 = T[r, c] / s32[r].astype(np.float64)
+        frac = np.abs(quo64 - np.trunc(quo64))
+        assert np.all(np.abs(frac - 0.5) <= 2.0 ** -21 * np.maximum(1.0, np.abs(quo64)))   # ... a near-tie in fp64
+        assert np.all(frac != 0.5)
+
+
+# --------------------------------------------------------------------------------------
+# Planted mistakes: each plausible slip in the oracle's source fails a pin above
+# --------------------------------------------------------------------------------------
+
+_ORACLE_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle")
+
+MUTANTS = {
+    # name: (text in stamp_oracle.c, replacement, [pins that must fail])
+    "haar_detail_sign": ("tmp[half + i] = (v[2 * i] - v[2 * i + 1]) * r;", "tmp[half + i] = (v[2 * i + 1] - v[2 * i]) * r;",
+                         ["test_haar_n2_hand_case", "closed_form"]),
+    "haar_step_not_normalised": ("const double r = 1.0 / sqrt(2.0);\n  int half", "const double r = 0.5;\n  int half",
+                                 ["orthonormal_haar"]),
+    "inverse_uses_untransposed_matrix": ("double l = transpose ? Lmat[(size_t)t * n + i] : Lmat[(size_t)i * n + t];",
+                                         "double l = Lmat[(size_t)i * n + t];", ["reconstruction", "plain_matmul"]),
+    "dct_dc_row_not_rescaled": ("double cu = (u == 0) ? 1.0 / sqrt(2.0) : 1.0;", "double cu = 1.0;",
+                                ["orthonormal_dct", "dct_scipy"]),
+    "bias_dropped": ("Y[(size_t)m * N + j] += (double)bias[j];", "Y[(size_t)m * N + j] += 0.0;",
+                     ["exact_codes", "python_loops"]),
+    "qmax_is_two_to_b_minus_1": ("float qmaxf = (float)((1 << (bits - 1)) - 1);\n    double amax = 0.0;\n    for (int j = 0; j < K; ++j) {\n      double a = fabs(t[j]);",
+                                 "float qmaxf = (float)((1 << (bits - 1)));\n    double amax = 0.0;\n    for (int j = 0; j < K; ++j) {\n      double a = fabs(t[j]);",
+                                 ["quantizer_hand_rows", "quantizer_properties"]),
+    "round_toward_zero": ("float q = g_decide_fp64 ? (float)nearbyint(t[j] / (double)s) : rintf((float)t[j] / s);",
+                          "float q = truncf((float)t[j] / s);", ["quantizer_hand_rows", "quantizer_properties"]),
+    "gemm_weight_operand_transposed": ("const int8_t* b = wq + (size_t)n * K;\n      for (int k = 0; k < K; ++k) s += (int64_t)a[k] * (int64_t)b[k];",
+                                       "const int8_t* b = wq + n;\n      for (int k = 0; k < K; ++k) s += (int64_t)a[k] * (int64_t)b[(size_t)(k % N) * K + (k / N)];",
+                                       ["gemm_brute_force"]),
+    "dequant_forgets_weight_scale": ("(double)acc[(size_t)m * N + n] * (double)sx[m] * (double)sw[n];",
+                                     "(double)acc[(size_t)m * N + n] * (double)sx[m];", ["exact_codes", "python_loops"]),
+    "high_precision_rows_off_by_one": ("bits[i] = ((i % n) < k_hi) ? bits_hi : bits_lo;", "bits[i] = ((i % n) <= k_hi) ? bits_hi : bits_lo;",
+                                       ["printed_bits"]),
+    "wht_natural_order": ("Lmat[(size_t)changes * n + j] = par ? -r : r;", "Lmat[(size_t)i * n + j] = par ? -r : r;",
+                          ["wht_sequency"]),
+    "haar2d_lh_hl_swapped_sign": ("tmp[3 * q + i] = (a - b - c + d) * 0.5;", "tmp[3 * q + i] = (a - b - c - d) * 0.5;",
+                                  ["haar2d_orthonormal"]),
+}
+
+_PINS = {
+    "test_haar_n2_hand_case": lambda o: test_haar_n2_hand_case(o),
+    "closed_form": lambda o: test_haar_closed_form_rows(o, 16, 3),
+    "orthonormal_haar": lambda o: test_orthonormal(o, T_HAAR, 64, 3),
+    "orthonormal_dct": lambda o: test_orthonormal(o, T_DCT, 8, 0),
+    "dct_scipy": lambda o: test_dct_matches_scipy_ortho_dct2(o, 16),
+    "reconstruction": lambda o: test_energy_and_reconstruction(o, T_HAAR, 128, 3),
+    "plain_matmul": lambda o: test_unquantized_pipeline_is_plain_matmul(o),
+    "exact_codes": lambda o: test_layer_exact_when_codes_are_exact(o),
+    "python_loops": lambda o: test_layer_vs_python_loops(o),
+    "quantizer_hand_rows": lambda o: test_quantizer_round_half_to_even_and_zero_row(o),
+    "quantizer_properties": lambda o: test_quantizer_properties(o),
+    "gemm_brute_force": lambda o: test_gemm_brute_force(o),
+    "printed_bits": lambda o: test_bit_map_reproduces_printed_effective_bits(o),
+    "wht_sequency": lambda o: test_wht_is_the_sequency_ordered_hadamard_matrix(o, 8),
+    "haar2d_orthonormal": lambda o: test_haar2d_orthonormal_and_lowpass_closed_form(o, 8, 8, 3),
+}
+
+
+def _load_mutant(tmpdir, name, old, new):
+    """A second copy of the oracle's ctypes wrapper bound to a library compiled from the mutated source."""
+    src = open(os.path.join(_ORACLE_DIR, "stamp_oracle.c")).read()
+    assert src.count(old) == 1, f"mutation site of {name!r} not found exactly once in the oracle source"
+    c_path = os.path.join(tmpdir, f"mutant_{name}.c")
+    so_path = os.path.join(tmpdir, f"libmutant_{name}.so")
+    with open(c_path, "w") as f:
+        f.write(src.replace(old, new))
+    subprocess.check_call(["gcc", "-O1", "-fopenmp", "-shared", "-fPIC", "-o", so_path, c_path, "-lm"])
+    spec = importlib.util.spec_from_file_location(f"mutant_oracle_{name}", os.path.join(_ORACLE_DIR, "stamp_oracle.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod._SRC, mod._LIB = c_path, so_path
+    return mod
+
+
+@pytest.mark.parametrize("name", list(MUTANTS))
+def test_planted_mistake_fails_its_pins(name):
+    """Mutate a COPY of the oracle's source (the committed oracle is untouched), build it, and run the named pins
+    on the mutant: every one of them must fail.  The mutations are the slips a plausible rewrite would make --
+    a flipped sign, a missing normalisation, a transposed operand, a dropped term, a wrong code range."""
+    old, new, pins = MUTANTS[name]
+    with tempfile.TemporaryDirectory() as tmpdir:
+        mutant = _load_mutant(tmpdir, name, old, new)
+        for pin in pins:
+            with pytest.raises(AssertionError):
+                _PINS[pin](mutant)
+
+
+def test_unmutated_oracle_passes_the_pins_the_mutants_fail(oracle):
+    for pin in _PINS.values():
+        pin(oracle)
