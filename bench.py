@@ -30,12 +30,15 @@ from paper_2510_26771_b200 import inputs as gen  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_I8_OVER_BF16 = 2.0      # dense tensor peaks: 4.5 POPS int8 vs 2.25 PFLOPS bf16
+NOMINAL_I8_TOPS = 4500.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
+DEFAULT_WORKLOAD = "sweep_L32768_D8192"   # the largest single-GPU shape of the throughput sweep
+SECONDARY_WORKLOAD = "llm_mlp_up"         # read as well (extra.secondary): the LLM layer of the named configurations
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None until
-# a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {"llm_mlp_up": 54400000 + 14459392}   # profiles/k_gemm_i8_haar_epilogue_llm_mlp_up.txt
+# DRAM bytes per launch of the dominant kernel from an ncu capture of the kernel as it stands (see profiles/);
+# a workload is listed only while that capture is current.
+NCU_TRAFFIC_BYTES = {}
 
 
 def workloads():
@@ -110,6 +113,59 @@ class ClockSampler:
         return out
 
 
+def time_loop(fn, iters, warm=3):
+    """Mean milliseconds per call of fn(i) over `iters` back-to-back calls (CUDA events on the current stream)."""
+    import torch
+    for i in range(warm):
+        fn(i)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(iters):
+        fn(i)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / iters
+
+
+def measure_i8_ceilings(st, local_rank):
+    """The int8 tensor ceilings of THIS GPU, taken in this run:
+    * the issue-only tcgen05.mma kind::i8 loop on tiles resident in shared memory (stamp_measure_i8_mma_issue):
+      burst = best of 5 launches of about 4 ms, sustained = mean over about a second of back-to-back launches,
+      with the SM clock sampled meanwhile;
+    * torch._int_mm 8192^3 (the vendor library's int8 GEMM), burst and mean."""
+    import torch
+    out = {}
+    nbatch = 1000
+    ops = st.stamp_measure_i8_mma_issue(nbatch)   # warm-up, sets the function attribute
+    torch.cuda.synchronize()
+    best = min(time_loop(lambda i: st.stamp_measure_i8_mma_issue(nbatch), 1, warm=0) for _ in range(5))
+    out["issue_only_burst_tops"] = ops / (best * 1e-3) / 1e12
+    sampler = ClockSampler(local_rank)
+    n = max(10, int(1000.0 / best))
+    mean = time_loop(lambda i: st.stamp_measure_i8_mma_issue(nbatch), n, warm=0)
+    clk = sampler.stop()
+    out["issue_only_sustained_tops"] = ops / (mean * 1e-3) / 1e12
+    out["issue_only_sustained_sm_mhz"] = clk["sm_mhz"]
+    out["issue_only_reasons"] = clk["reasons"]
+    out["issue_only_shape"] = "M128 x N256 x K32, cta_group::1, one CTA per SM, 64000 instructions per CTA and launch"
+    try:
+        a = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda")
+        b = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda").t()
+        torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        t_best = min(time_loop(lambda i: torch._int_mm(a, b), 1, warm=0) for _ in range(10))
+        t_mean = time_loop(lambda i: torch._int_mm(a, b), 20, warm=0)
+        out["torch_int_mm_8192_burst_tops"] = 2.0 * 8192 ** 3 / (t_best * 1e-3) / 1e12
+        out["torch_int_mm_8192_tops"] = 2.0 * 8192 ** 3 / (t_mean * 1e-3) / 1e12
+        del a, b
+    except Exception:
+        out["torch_int_mm_8192_burst_tops"] = out["torch_int_mm_8192_tops"] = None
+    if st.stamp_last_device_status() != 0:
+        raise RuntimeError("device status word raised by the issue-only loop")
+    return out
+
+
 def max_over_ranks_ms(local_ms: float, device="cpu") -> float:
     """Timed-region duration of the whole job: the slowest rank's (all-reduce MAX; identity for one rank)."""
     import torch
@@ -170,7 +226,7 @@ def run_reference(args, cfg):
                          want=("Y",))
     for _ in range(min(args.warmup, 1)):
         step()
-    steps = max(1, min(args.steps, 5))
+    steps = max(1, min(args.steps, 3))
     t0 = time.perf_counter()
     for _ in range(steps):
         step()
@@ -188,18 +244,61 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def quick_reading(st, cfg, y_t, steps):
+    """ms per step, layer TOPS and GEMM share of another workload through the same call (no side measurements)."""
+    import torch
+    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid, zero_point=cfg.zero_point)
+    x_t = torch.bfloat16 if cfg.dtype == gen.BF16 else torch.float32
+    X_host = torch.from_numpy(gen.make_activation(cfg)).to(x_t)
+    W_dev = torch.from_numpy(gen.make_weight(cfg)).cuda().to(x_t)
+    bias = torch.from_numpy(gen.make_bias(cfg)).cuda()
+    wq, w_scale = st.stamp_quantize_weights(c, W_dev)
+    w_op, w_fmt, _ = weight_operand(st, c, wq)
+    n_x = max(2, -(-2 * L2_BYTES // (X_host.numel() * X_host.element_size())))
+    n_w = max(2, -(-2 * L2_BYTES // (w_op.numel() * w_op.element_size())))
+    Xs = [X_host.cuda() for _ in range(n_x)]
+    Ws = [w_op.clone() for _ in range(n_w)]
+    Y = torch.empty((cfg.B, cfg.L, cfg.N), dtype=y_t, device="cuda")
+    ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def step(i):
+        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], w_fmt, w_scale, bias, ws, out=Y)
+    ms = time_loop(step, steps, warm=20)
+    launches = st.stamp_last_launch_count()
+    st.stamp_profile_gemm_events(g0, g1)
+    gms = []
+    for i in range(20):
+        step(i)
+        torch.cuda.synchronize()
+        gms.append(g0.elapsed_time(g1))
+    st.stamp_profile_gemm_events(None, None)
+    ops = 2.0 * cfg.M * cfg.N * cfg.K
+    gemm_ms = statistics.mean(gms)
+    return {"workload": cfg.name, "steps": steps, "ms_per_step": ms, "tops": ops / (ms * 1e-3) / 1e12,
+            "gemm_ms": gemm_ms, "gemm_tops": ops / (gemm_ms * 1e-3) / 1e12, "launches_per_step": launches,
+            "device_status": st.stamp_last_device_status()}
+
+
+def weight_operand(st, c, wq):
+    """The weight operand the benchmark hands to the layer: prepared once, offline (weights are static)."""
+    w8 = st.stamp_prepare_weights(c, wq)
+    return w8, st.W_INT8, "int4 codes, one per int8, prepared offline"
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="native", choices=("native", "reference"))
-    ap.add_argument("--workload", default="llm_mlp_up")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--out-dtype", default="bf16", choices=("bf16", "f32"))
     ap.add_argument("--levels", type=int, default=None,
                     help="override the workload's Haar level count (0 = full depth) and, with --k-hi, its 8-bit rows")
     ap.add_argument("--k-hi", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the second reading on the LLM layer")
     ap.add_argument("--quick", action="store_true",
                     help="timed region only (no side measurements, no CPU baseline): for profiler captures")
     ap.add_argument("--stage", default="fused", choices=("fused", "quantize", "inverse"),
@@ -239,20 +338,20 @@ def main():
     W_dev = torch.from_numpy(gen.make_weight(cfg)).cuda().to(x_t)
     bias = torch.from_numpy(gen.make_bias(cfg)).cuda()
     wq, w_scale = st.stamp_quantize_weights(c, W_dev)       # offline: weights are static
-    w8 = st.stamp_prepare_weights(c, wq)
+    w8, w_fmt, weights_note = weight_operand(st, c, wq)
     del W_dev
     x_bytes = X_host.numel() * X_host.element_size()
     y_bytes = M * N * (2 if y_t == torch.bfloat16 else 4)
     # rotate over enough distinct copies that consecutive steps never find their inputs in L2
     n_x = max(2, -(-2 * L2_BYTES // x_bytes))
-    n_w = max(2, -(-2 * L2_BYTES // w8.numel()))
+    n_w = max(2, -(-2 * L2_BYTES // (w8.numel() * w8.element_size())))
     Xs = [X_host.cuda() for _ in range(n_x)]
     Ws = [w8.clone() for _ in range(n_w)]
     Y = torch.empty((B, L, N), dtype=y_t, device="cuda")
     ws = st.alloc_workspace(c, B, L, K, N)
 
     def step(i):
-        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], st.W_INT8, w_scale, bias, ws, out=Y)
+        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], w_fmt, w_scale, bias, ws, out=Y)
 
     if args.quick and args.stage == "quantize":
         def step(i):  # noqa: F811
@@ -272,7 +371,9 @@ def main():
 
     # ---- timed region: exactly `steps` steps, CUDA events, GEMM bracketed by its own events ----
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    n_ev = min(steps, 200)
+    # the GEMM of every `ev_stride`-th step is bracketed by its own events: up to 200 samples spread over the whole region
+    ev_stride = max(1, -(-steps // 200))
+    n_ev = -(-steps // ev_stride)
     g0 = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev)]
     g1 = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev)]
     for e in g0 + g1:
@@ -283,9 +384,9 @@ def main():
     torch.cuda.synchronize()
     ev0.record()
     for i in range(steps):
-        if i < n_ev:
-            st.stamp_profile_gemm_events(g0[i], g1[i])
-        elif i == n_ev:
+        if i % ev_stride == 0:
+            st.stamp_profile_gemm_events(g0[i // ev_stride], g1[i // ev_stride])
+        elif i % ev_stride == 1:
             st.stamp_profile_gemm_events(None, None)
         step(i)
     ev1.record()
@@ -329,19 +430,7 @@ def main():
                           "gpu_launches": launches_per_step * steps, "clocks": clocks}), flush=True)
         return
 
-    # ---- the bandwidth-bound passes, timed alone (L2 defeated by the same rotation) ----
-    def time_loop(fn, iters):
-        for i in range(3):
-            fn(i)
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for i in range(iters):
-            fn(i)
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / iters
-
+    # ---- the bandwidth-bound passes, timed alone on this same workload (L2 defeated by the same rotation) ----
     iters = max(10, min(steps, 200))
     nh = st.n_hi_rows(c, B, L)
     quant_bytes = x_bytes + nh * K + (M - nh) * K // 2 + 4 * M
@@ -352,25 +441,15 @@ def main():
     i_ms = time_loop(lambda i: st.stamp_inverse(c, Yts[i % n_yt], bias, ws, out=Y), iters)
     del Yts
 
-    # ---- int8 GEMM throughput of the vendor library on this machine, for context ----
-    int_mm_tops = None
-    try:
-        a = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda")
-        b = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda").t()
-        mm_ms = time_loop(lambda i: torch._int_mm(a, b), 20)
-        int_mm_tops = 2.0 * 8192 ** 3 / (mm_ms * 1e-3) / 1e12
-        del a, b
-    except Exception:
-        pass
-
     # ---- end to end: host buffers, copies inside the timed region, through the C ABI ----
     # Two calls are kept in flight, on two streams with a workspace and a pinned result buffer each, so that
     # one step's result copy (device to host) overlaps the next step's input copy (host to device): the link is
     # full duplex.  Every step still copies its X in and its Y out inside the timed region.
     ws_bytes_h = st.stamp_workspace_bytes_host(c, B, L, K, N, st._dtype_code(X_host), 1 if y_t == torch.bfloat16 else 0)
+    del ws
     lanes = [(torch.cuda.Stream(), torch.empty(ws_bytes_h, dtype=torch.uint8, device="cuda"),
               torch.empty((B, L, N), dtype=y_t).pin_memory()) for _ in range(2)]
-    e2e_steps = max(6, min(steps, 100))
+    e2e_steps = max(6, min(steps, 100, int(2000.0 / max(ms_per_step * 8, 1e-3))))
 
     def e2e_loop(iters):
         main = torch.cuda.current_stream()
@@ -381,7 +460,7 @@ def main():
         for i in range(iters):
             stream, ws_h, Y_host = lanes[i % 2]
             with torch.cuda.stream(stream):
-                st.stamp_linear_fused_host(c, X_host, Ws[i % n_w], st.W_INT8, w_scale, bias, Y_host, ws_h)
+                st.stamp_linear_fused_host(c, X_host, Ws[i % n_w], w_fmt, w_scale, bias, Y_host, ws_h)
         for lane in lanes:
             done = torch.cuda.Event()
             done.record(lane[0])
@@ -392,38 +471,62 @@ def main():
 
     e2e_loop(4)
     e2e_ms = e2e_loop(e2e_steps)
-    e2e = {"value": ops / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": x_bytes,
-           "d2h_bytes_per_step": y_bytes, "ms_per_step": e2e_ms, "in_flight": 2}
-    del lanes
+    e2e = {"value": world * ops / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS", "h2d_bytes_per_step": x_bytes,
+           "d2h_bytes_per_step": y_bytes, "ms_per_step": e2e_ms, "in_flight": 2, "steps": e2e_steps}
+    del lanes, Xs, Ws, Y
 
-    i8_peak = peaks["bf16_sustained"] * NOMINAL_I8_OVER_BF16
+    # ---- a second reading on the LLM layer of the named configurations (same code path, smaller shape) ----
+    secondary = None
+    if cfg.name != SECONDARY_WORKLOAD and not args.no_secondary:
+        secondary = quick_reading(st, workloads()[SECONDARY_WORKLOAD], y_t, min(steps, 1000))
+
+    # ---- int8 ceilings of this GPU, measured now ----
+    ceil = measure_i8_ceilings(st, local_rank)
+
+    # The GEMM's denominator.  A timed region shorter than about a second runs at boost clocks (burst regime);
+    # a longer one settles under the power cap (sustained regime): the measured ceilings of the same regime apply.
+    burst = total_ms < 1000.0
+    regime = "burst" if burst else "sustained"
+    bf16x2 = (peaks["bf16_burst"] if burst else peaks["bf16_sustained"]) * NOMINAL_I8_OVER_BF16
+    candidates = {
+        f"issue-only tcgen05.mma kind::i8 loop, {regime}": ceil["issue_only_burst_tops" if burst else "issue_only_sustained_tops"],
+        f"torch._int_mm 8192^3, {regime}": ceil["torch_int_mm_8192_burst_tops" if burst else "torch_int_mm_8192_tops"],
+        f"2 x {peaks['source']} bf16 {regime} ({peaks['bf16_burst' if burst else 'bf16_sustained']} TFLOP/s)": bf16x2,
+    }
+    peak_name, i8_peak = max(((k, v) for k, v in candidates.items() if v), key=lambda kv: kv[1])
     gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "k_gemm_i8", "achieved": gemm_tops, "peak": i8_peak, "unit": "TFLOP/s",
-                "frac": gemm_tops / i8_peak, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
-                "note": f"int8 ops; peak = {peaks['source']} sustained bf16 {peaks['bf16_sustained']} TFLOP/s x 2 "
-                        "(nominal int8:bf16 ratio); kernel timed inside the long step loop"}
+                "frac": gemm_tops / i8_peak, "frac_of_nominal": gemm_tops / NOMINAL_I8_TOPS,
+                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                "note": f"int8 ops; timed region {total_ms:.0f} ms => {regime} regime; peak = the highest of the int8 "
+                        f"ceilings measured in this run for that regime: {peak_name}; all candidates (TOPS): "
+                        + ", ".join(f"{k} = {v:.0f}" for k, v in candidates.items() if v)
+                        + f"; nominal dense int8 {NOMINAL_I8_TOPS:.0f}"}
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         cpu_baseline, _ = cpu_oracle_sample(cfg)
 
+    sm_mhz = clocks["sm_mhz"] if clocks else None
     line = {
         "metric": "stamp_linear_tops", "value": value, "unit": "TOPS", "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": cfg.name, "B": B, "L": L, "K": K, "N": N, "transform": int(cfg.transform),
                    "block": cfg.block, "levels": cfg.levels, "k_hi": cfg.k_hi, "x_dtype": str(x_t).split(".")[-1],
-                   "y_dtype": str(y_t).split(".")[-1], "weights": "int4 codes, one per int8, prepared offline",
+                   "y_dtype": str(y_t).split(".")[-1], "weights": weights_note,
                    "l2": f"inputs rotate over {n_x} activation and {n_w} weight copies (> 2x L2)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * steps, "roofline": roofline,
         "cpu_baseline": cpu_baseline,
-        "extra": {"gemm_ms": gemm_ms, "gemm_tops": gemm_tops, "frac_of_nominal_4500": gemm_tops / 4500.0,
+        "extra": {"gemm_ms": gemm_ms, "gemm_tops": gemm_tops, "timed_region_ms": total_ms,
+                  "ms_per_step_x_sm_mhz": ms_per_step * sm_mhz if sm_mhz else None,
                   "layer_frac_of_i8_peak": value / world / i8_peak,
-                  "quant_ms": q_ms, "quant_gbs": quant_bytes / (q_ms * 1e-3) / 1e9,
+                  "layer_frac_of_nominal": value / world / NOMINAL_I8_TOPS,
+                  "quant_ms": q_ms, "quant_gbs": quant_bytes / (q_ms * 1e-3) / 1e9, "quant_bytes": quant_bytes,
                   "quant_frac_hbm": quant_bytes / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                  "inverse_ms": i_ms, "inverse_gbs": inv_bytes / (i_ms * 1e-3) / 1e9,
+                  "inverse_ms": i_ms, "inverse_gbs": inv_bytes / (i_ms * 1e-3) / 1e9, "inverse_bytes": inv_bytes,
                   "inverse_frac_hbm": inv_bytes / (i_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                  "torch_int_mm_8192_tops": int_mm_tops, "launches_per_step": launches_per_step,
+                  "i8_ceilings": ceil, "secondary": secondary, "launches_per_step": launches_per_step,
                   "device_status": status, "peaks": peaks},
     }
     print(json.dumps(line), flush=True)

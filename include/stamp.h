@@ -36,8 +36,8 @@
  *         LL = (a+b+c+d)/2, LH = (a-b+c-d)/2, HL = (a+b-c-d)/2, HH = (a-b-c+d)/2 and LL recurses;
  *         order [LL_l | LH_l | HL_l | HH_l | LH_(l-1) | ... | HH_1], bands in raster order;
  *         levels = 1..3, 2^levels divides both grid sides.
- *     The 8-bit tokens are the rows {i : i mod n < k_hi} ("the first 64 tokens are kept at
- *     8 bits", Sec. "Optimal bit allocation").
+ *     The 8-bit tokens are the rows {i : i mod n < k_hi}: the two-level allocation at the end of
+ *     Sec. "Optimal bit allocation" (k_hi leading transformed tokens at bits_hi, the rest at bits_lo).
  *   - Quantizer (Sec. 2.1, first equation, symmetric form): scale = absmax / qmax,
  *     code = clamp(round_half_even(t / scale), -qmax, +qmax), qmax = 2^(bits-1) - 1; a zero
  *     row gets scale 1.  Nothing clips (min-max range setting of Sec. 2.1).
@@ -225,6 +225,27 @@ int stamp_debug_gemm_i32(const stamp_config* cfg, const void* q_hi, const void* 
                          int w_format, int B, int L, int K, int N, int32_t* acc, void* ws, size_t ws_bytes,
                          void* stream);
 
+/*
+ * The token operand of the GEMM as the one-call layer (stamp_linear_fused) produces it, mapped back to logical
+ * order.  For a Haar transform of at least 5 levels over blocks that are multiples of 256 tokens, and for the
+ * three-level 2-D Haar transform, that call's transform+quantize kernels store their codes in the order the GEMM's
+ * fused inverse consumes (not through the stamp_quantize format).  This export runs those same kernels on X and
+ * gathers, for every logical transformed token (the order of stamp_quantize's outputs):
+ *   codes   [B, L, K] int8   its codes as stored (zero-point mode: offset by 2^(b-1), as in stamp_quantize)      out
+ *   factor  [B, L]    float  what the fused inverse multiplies the row's accumulators with: scale * 2^(-j/2) for
+ *                            a 1-D Haar row of level j <= 8, the plain scale for rows of levels above 8 (they go
+ *                            through a separate small product), scale * 2^(-l) for a 2-D Haar row of level l    out
+ *   level   [B, L]    int32  that level j (or l)                                                                  out
+ *   zero    [B, L]    int32  zero points of the stored codes (zero-point mode; zeros otherwise); may be NULL in
+ *                            symmetric mode                                                                       out
+ * Other configurations keep their operand in logical order (what stamp_quantize returns): STAMP_ERR_UNSUPPORTED.
+ * No counterpart in the paper: the row order of the operand is a layout choice of this implementation, and parity
+ * is judged on logical order.
+ */
+int stamp_debug_fused_operand(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, int N,
+                              int8_t* codes, float* factor, int32_t* level, int32_t* zero, void* ws, size_t ws_bytes,
+                              void* stream);
+
 /* Synchronizes `stream`, then reads and clears the device status word of the current device.
  * *status is STAMP_OK or STAMP_ERR_TIMEOUT (a bounded wait inside a kernel expired; outputs of
  * the calls since the last read are then invalid). */
@@ -234,6 +255,14 @@ int stamp_last_device_status(void* stream, int* status);
  * calling thread is bracketed by cudaEventRecord(start) / cudaEventRecord(stop) on its stream
  * (each launch re-records the pair).  Pass NULLs to switch it off.  Events are cudaEvent_t. */
 int stamp_profile_gemm_events(void* start_event, void* stop_event);
+
+/* Measurement: the rate of the tensor cores' int8 instruction alone.  Launches one CTA per SM; each issues
+ * nbatch * 64 tcgen05.mma kind::i8 instructions (M128 x N256 x K32, int32 accumulators in tensor memory) on
+ * operand tiles that stay in shared memory -- no loads in the loop, waits bounded -- and *ops_out receives the
+ * integer operations of the whole launch (2 * M * N * K per instruction).  The caller times the launch with
+ * events on `stream`; ops / time is the ceiling the layer's GEMM is reported against.  No counterpart in the
+ * paper: it measures the machine.  1 <= nbatch <= 2^20. */
+int stamp_measure_i8_mma_issue(int nbatch, long long* ops_out, void* stream);
 
 /* How many kernels of this library the calling thread's last API call launched. */
 int stamp_last_launch_count(void);

@@ -70,7 +70,8 @@ static void haar_step(double* v, int len, double* tmp) {
 }
 
 /* Multi-level Haar DWT of a length-n vector: each level re-applies the step to the low-pass
- * half, "pushing the energy in the first half" level by level; after `levels` levels the order
+ * half, so that the energy moves into the leading entries level by level (Sec. "Efficient Energy
+ * Concentration"); after `levels` levels the order
  * is [a_levels | d_levels | d_{levels-1} | ... | d_1]. */
 static void haar_forward(double* v, int n, int levels, double* tmp) {
   int len = n;

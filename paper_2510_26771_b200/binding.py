@@ -23,7 +23,8 @@ EXPORTS = (
     "stamp_linear", "stamp_inverse", "stamp_linear_fused", "stamp_workspace_bytes_host",
     "stamp_linear_fused_host", "stamp_profile_gemm_events", "stamp_debug_transform",
     "stamp_debug_unpack_codes", "stamp_debug_gemm_i32", "stamp_last_device_status",
-    "stamp_last_launch_count", "stamp_status_string", "stamp_inverse_noalloc",
+    "stamp_last_launch_count", "stamp_status_string", "stamp_inverse_noalloc", "stamp_debug_fused_operand",
+    "stamp_measure_i8_mma_issue",
 )
 
 
@@ -246,10 +247,31 @@ def stamp_debug_gemm_i32(cfg: StampConfig, q_hi, q_lo, w, w_format: int, B: int,
     return acc
 
 
+def stamp_debug_fused_operand(cfg: StampConfig, X: torch.Tensor, N: int, ws: torch.Tensor):
+    """Codes, per-row factors, levels and zero points of the one-call layer's GEMM operand, in logical order."""
+    B, L, K = X.shape
+    codes = torch.empty((B, L, K), dtype=torch.int8, device=X.device)
+    factor = torch.empty((B, L), dtype=torch.float32, device=X.device)
+    level = torch.empty((B, L), dtype=torch.int32, device=X.device)
+    zero = torch.empty((B, L), dtype=torch.int32, device=X.device)
+    wp, wb = _ws_args(ws)
+    _check(lib().stamp_debug_fused_operand(ctypes.byref(cfg), _ptr(X), _dtype_code(X), B, L, K, N, _ptr(codes),
+                                           _ptr(factor), _ptr(level), _ptr(zero), wp, wb, _stream()),
+           "stamp_debug_fused_operand")
+    return codes, factor, level, zero
+
+
 def stamp_last_device_status() -> int:
     st = ctypes.c_int(0)
     _check(lib().stamp_last_device_status(_stream(), ctypes.byref(st)), "stamp_last_device_status")
     return int(st.value)
+
+
+def stamp_measure_i8_mma_issue(nbatch: int) -> int:
+    """Enqueue the issue-only int8 tensor-core loop on the current stream; returns the integer operations it performs."""
+    ops = ctypes.c_longlong(0)
+    _check(lib().stamp_measure_i8_mma_issue(int(nbatch), ctypes.byref(ops), _stream()), "stamp_measure_i8_mma_issue")
+    return int(ops.value)
 
 
 def stamp_last_launch_count() -> int:

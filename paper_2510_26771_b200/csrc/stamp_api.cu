@@ -9,10 +9,13 @@
 #include "common.cuh"
 #include "k_dct.cuh"
 #include "k_dct_tc.cuh"
+#include "k_debug.cuh"
 #include "k_gemm.cuh"
 #include "k_haar2d.cuh"
 #include "k_generic.cuh"
 #include "k_haar_cq.cuh"
+#include "k_haar_tc.cuh"
+#include "k_peak.cuh"
 #include "k_top_gemv.cuh"
 #include "stamp.h"
 
@@ -115,7 +118,7 @@ static PassPlan make_plan(int levels) {
 // Workspace layout (one layout for all calls of a problem size).
 // ------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t rowmax, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, dctsplit, xzero, wsum, total;
+  size_t rowmax, htc_cnt, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, dctsplit, xzero, wsum, total;
 };
 static Workspace layout(const Problem& pb) {
   Workspace w{};
@@ -126,6 +129,8 @@ static Workspace layout(const Problem& pb) {
   const size_t pong_rows = pl.npass > 2 ? (M >> (pl.p[0] + pl.p[1])) : 0;
   size_t off = 0;
   w.rowmax = off; off += align256(M * 4);
+  // (directly behind the row maxima: one memset clears both before the tensor-core transform+quantize launch)
+  w.htc_cnt = off; off += align256((M >> 7) * 4 + 4);
   w.xscale = off; off += align256(M * 4);
   w.T = off;      off += align256(M * (size_t)pb.K * 4);
   w.ping = off;   off += align256(ping_rows * KN * 4);
@@ -194,14 +199,14 @@ static int make_tmap_i8(const void* base, long rows, int K, int box_rows, CUtens
   return r == CUDA_SUCCESS ? STAMP_OK : STAMP_ERR_CUDA;
 }
 
-// bf16 matrix [rows, cols] row-major; box = 64 columns (128 bytes) x 256 rows, 128-byte swizzle.
-static int make_tmap_bf16(const void* base, long rows, long cols, CUtensorMap* out) {
+// bf16 matrix [rows, cols] row-major; box = 64 columns (128 bytes) x box_rows rows, 128-byte swizzle.
+static int make_tmap_bf16(const void* base, long rows, long cols, CUtensorMap* out, int box_rows = 256) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return STAMP_ERR_CUDA;
   if ((reinterpret_cast<uintptr_t>(base) & 15) != 0) return STAMP_ERR_INVALID_ARG;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {64u, 256u};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1u, 1u};
   CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -226,15 +231,47 @@ static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
   return cudaLaunchKernelEx(&lc, kern, KArgs(args)...);
 }
 
+// Per-device facts and settings.  A process may use the library on several GPUs: the SM count, the
+// opt-in to more than 48 KB of dynamic shared memory (a per-device function attribute) and the number of
+// resident clusters are therefore cached per device, under one mutex (host threads may call concurrently).
+constexpr int MAX_DEVICES = 64;
+static std::mutex g_dev_mu;
+
+static int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -1;
+  return dev;
+}
+
 static int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
+  static int n_of[MAX_DEVICES] = {};
+  const int dev = current_device();
+  if (dev < 0) return 148;
+  std::lock_guard<std::mutex> lock(g_dev_mu);
+  if (n_of[dev] == 0) {
+    int n = 0;
     cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
+    n_of[dev] = n > 0 ? n : 148;
   }
-  return n;
+  return n_of[dev];
+}
+
+// Make sure `func` may be launched with `bytes` of dynamic shared memory on the current device.
+static int ensure_dyn_smem(const void* func, size_t bytes) {
+  static std::unordered_map<unsigned long long, size_t> granted;   // (device, function) -> bytes already allowed
+  const int dev = current_device();
+  if (dev < 0) return STAMP_ERR_CUDA;
+  const unsigned long long key = (static_cast<unsigned long long>(dev) << 56) ^ reinterpret_cast<uintptr_t>(func);
+  std::lock_guard<std::mutex> lock(g_dev_mu);
+  size_t& have = granted[key];
+  if (bytes > have) {
+    if (cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+      cudaGetLastError();
+      return STAMP_ERR_CUDA;
+    }
+    have = bytes;
+  }
+  return STAMP_OK;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -245,12 +282,7 @@ static int launch_dct_tc(const CUtensorMap& ta, const CUtensorMap& tb0, const CU
                          cudaStream_t st) {
   using SM = DctSmem<NATOM, NPLANE>;
   auto kern = k_dct_tc<MODE, NATOM, NPLANE>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::DYN_BYTES) != cudaSuccess)
-      return STAMP_ERR_CUDA;
-    attr_set = true;
-  }
+  if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), SM::DYN_BYTES)) return rc;
   const int tiles = dp.nblk * (dp.cols / (NATOM * 64));
   const int grid = tiles < sm_count() ? tiles : sm_count();
   if (launch_pdl(kern, dim3((unsigned)grid), dim3(DCT_THREADS), SM::DYN_BYTES, st, ta, tb0, tb1, dp) != cudaSuccess) {
@@ -265,12 +297,7 @@ template <int BN, int STAGES, int EPI>
 static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const GemmParams& gp, cudaStream_t st) {
   using SM = GemmSmem<BN, STAGES>;
   auto kern = k_gemm_i8<BN, STAGES, EPI>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::DYN_BYTES) != cudaSuccess)
-      return STAMP_ERR_CUDA;
-    attr_set = true;
-  }
+  if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), SM::DYN_BYTES)) return rc;
   const int ch_tiles = (gp.n_out + GEMM_BM - 1) / GEMM_BM;
   const int tok_tiles = (gp.m_tok + BN - 1) / BN;
   const int tiles = ch_tiles * tok_tiles;
@@ -406,12 +433,7 @@ static int launch_haar2d_fwd(const Problem& pb, const TIn* X, float* T, unsigned
 template <typename TIn, int THREADS, bool ZP>
 static int launch_haar2d_patch(const Haar2dPatchParams& pp, long npatch, size_t smem, cudaStream_t st) {
   auto kern = k_haar2d_patch_quant<TIn, THREADS, ZP>;
-  static size_t attr_smem = 0;
-  if (smem > attr_smem) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return STAMP_ERR_CUDA;
-    attr_smem = smem;
-  }
+  if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return rc;
   kern<<<(unsigned)npatch, THREADS, smem, st>>>(pp);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
@@ -426,8 +448,13 @@ static int run_quantize_haar2d_patch(const Problem& pb, const TIn* X, unsigned* 
   const size_t smem = (size_t)64 * pb.K * sizeof(TIn);
   if (smem <= 224 * 1024) {
     Haar2dPatchParams pp{X, pb.n, pb.grid_w, pb.K, pb.k_hi, (float)pb.qmax_hi, (float)pb.qmax_lo, a8, sx_epi, x_scale,
-                         zp_epi, pb.act_zp ? w8 : nullptr, pb.act_zp ? pb.N : 0, w_sum, nullptr, 0};
-    if ((size_t)pb.N * pb.K <= (size_t)24 << 20) {   // small weight matrix: have it in L2 when the GEMM starts
+                         zp_epi, nullptr, 0, nullptr, nullptr, 0};
+    if (pb.act_zp && w8 && w_sum) {   // the weight row sums of the zero-point term, taken by the same launch
+      pp.rs_w8 = w8;
+      pp.rs_rows = pb.N;
+      pp.rs_out = w_sum;
+    }
+    if (w8 && (size_t)pb.N * pb.K <= (size_t)24 << 20) {   // small weight matrix: have it in L2 when the GEMM starts
       pp.pf_base = reinterpret_cast<const uint8_t*>(w8);
       pp.pf_bytes = (long)pb.N * pb.K;
     }
@@ -644,12 +671,7 @@ static int launch_cq_t(CqParams cp, const CqChoice& c, cudaStream_t st) {
     cp.nstages = (int)ns;
     smem += slab * ns;
   }
-  static size_t attr_smem = 0;
-  if (smem > attr_smem) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return STAMP_ERR_CUDA;
-    attr_smem = smem;
-  }
+  if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return rc;
   cudaLaunchConfig_t lc{};
   lc.blockDim = dim3((unsigned)c.NT);
   lc.dynamicSmemBytes = smem;
@@ -666,7 +688,8 @@ static int launch_cq_t(CqParams cp, const CqChoice& c, cudaStream_t st) {
   // persistent clusters: as many as can be resident at once (cached per launch shape)
   static std::mutex mu;
   static std::unordered_map<unsigned long long, int> resident;
-  const unsigned long long key = ((unsigned long long)smem << 24) | ((unsigned long long)c.NT << 8) | (unsigned)c.C;
+  const unsigned long long key = ((unsigned long long)(current_device() & 0xFF) << 56) | ((unsigned long long)smem << 24) |
+                                 ((unsigned long long)c.NT << 8) | (unsigned)c.C;
   int ncl = 0;
   {
     std::lock_guard<std::mutex> lock(mu);
@@ -721,10 +744,12 @@ struct CqTiled {
   const uint8_t* pf_base = nullptr;   // weight codes to pull towards L2 during the first launch (optional)
   long pf_bytes = 0;
 };
+// start_lvl > 0: the first start_lvl levels have been applied already and X holds the un-normalised fp32 sums
+// over 2^start_lvl tokens, [nseq, n >> start_lvl, K], in the workspace's first hand-over buffer.
 static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, int x_dtype, int8_t* a8, void* q_hi,
                            void* q_lo, float* x_scale, float* T_out, uint8_t* base, const Workspace& wl,
-                           cudaStream_t st, const CqTiled* tiled = nullptr) {
-  const PassPlan pl = make_plan_max(pb.levels, c.pmax);
+                           cudaStream_t st, const CqTiled* tiled = nullptr, int start_lvl = 0) {
+  const PassPlan pl = make_plan_max(pb.levels - start_lvl, c.pmax);
   float* bufs[3] = {reinterpret_cast<float*>(base + wl.atop), reinterpret_cast<float*>(base + wl.top_ping),
                     reinterpret_cast<float*>(base + wl.top_pong)};
   CqParams cp{};
@@ -745,12 +770,13 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
     cp.sx_epi = tiled->sx_epi;
   }
   const void* in = X;
-  int Lin = pb.n, lvl0 = 0;
+  int Lin = pb.n >> start_lvl, lvl0 = start_lvl;
   for (int i = 0; i < pl.npass; ++i) {
     const int P = pl.p[i];
     const bool last = (i == pl.npass - 1);
     // launch i writes into buffer min(i, 1 + (i - 1) % 2): atop, then ping / pong alternately
-    float* aout = last ? nullptr : bufs[i == 0 ? 0 : 1 + ((i - 1) & 1)];
+    // (a continuation reads atop, so its launches alternate between ping and pong from the start)
+    float* aout = last ? nullptr : start_lvl ? bufs[1 + (i & 1)] : bufs[i == 0 ? 0 : 1 + ((i - 1) & 1)];
     cp.in = in;
     cp.aout = aout;
     cp.pf_base = (tiled && i == 0) ? tiled->pf_base : nullptr;
@@ -758,7 +784,7 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
     cp.Lin = Lin;
     cp.lvl0 = lvl0;
     cp.ngroups = (long)pb.nseq * (Lin >> P);
-    const bool bf16_in = (i == 0 && x_dtype == STAMP_BF16);
+    const bool bf16_in = (i == 0 && start_lvl == 0 && x_dtype == STAMP_BF16);
     const int rc = tiled ? launch_cq_o<CQ_OUT_TILED>(P, bf16_in, cp, c, st)
                    : a8  ? launch_cq_o<CQ_OUT_A8>(P, bf16_in, cp, c, st)
                       : T_out ? launch_cq_o<CQ_OUT_T>(P, bf16_in, cp, c, st)
@@ -769,6 +795,80 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
     lvl0 += P;
   }
   return STAMP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Haar transform + quantizer for bf16 activations: up to seven levels on the tensor cores with the
+// coefficients resident in tensor memory (k_haar_tc), deeper levels by the butterfly kernel on the
+// 128-token sums.
+// ------------------------------------------------------------------------------------------
+static bool htc_ok(const Problem& pb, int x_dtype) {
+  return pb.transform == STAMP_T_HAAR && x_dtype == STAMP_BF16 && pb.levels >= 1 && pb.n % 128 == 0 && !pb.act_zp &&
+         pb.K / 128 <= sm_count();
+}
+
+template <int OUT>
+static int launch_htc(const CUtensorMap& tx, const HtcParams& hp, cudaStream_t st) {
+  auto kern = k_haar_tc<OUT>;
+  if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), HTC_DYN_BYTES)) return rc;
+  const long items = hp.ntiles * hp.nchunks;
+  const int grid = items < sm_count() ? (int)items : sm_count();
+  if (launch_pdl(kern, dim3((unsigned)grid), dim3(HTC_THREADS), HTC_DYN_BYTES, st, tx, hp) != cudaSuccess) {
+    cudaGetLastError();
+    return STAMP_ERR_CUDA;
+  }
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+// Exactly one kind of output besides the scales, as for run_quantize_cq: a8 (tile order when `tiled`), or
+// (q_hi, q_lo), or T_out.
+static int run_quantize_haar(const Problem& pb, const CqChoice& c, const void* X, int x_dtype, int8_t* a8, void* q_hi,
+                             void* q_lo, float* x_scale, float* T_out, uint8_t* base, const Workspace& wl,
+                             cudaStream_t st, const CqTiled* tiled = nullptr) {
+  if (!htc_ok(pb, x_dtype)) return run_quantize_cq(pb, c, X, x_dtype, a8, q_hi, q_lo, x_scale, T_out, base, wl, st, tiled);
+  const int lv = pb.levels < 7 ? pb.levels : 7;
+  HtcParams hp{};
+  hp.K = pb.K;
+  hp.n = pb.n;
+  hp.lv = lv;
+  hp.last = (lv == pb.levels) ? 1 : 0;
+  hp.k_hi = pb.k_hi;
+  hp.qmax_hi = (float)pb.qmax_hi;
+  hp.qmax_lo = (float)pb.qmax_lo;
+  hp.ntiles = pb.M >> 7;
+  hp.nchunks = pb.K / 128;
+  hp.rowmax = reinterpret_cast<unsigned*>(base + wl.rowmax);
+  hp.cnt = reinterpret_cast<unsigned*>(base + wl.htc_cnt);
+  hp.aout = reinterpret_cast<float*>(base + wl.atop);
+  hp.a8 = a8;
+  hp.q_hi = static_cast<int8_t*>(q_hi);
+  hp.q_lo = static_cast<uint8_t*>(q_lo);
+  hp.x_scale = x_scale;
+  hp.T_out = T_out;
+  if (tiled) {
+    hp.sx_epi = tiled->sx_epi;
+    hp.pf_base = tiled->pf_base;
+    hp.pf_bytes = tiled->pf_bytes;
+  }
+  // row maxima and tile counts start from zero (the two regions are adjacent)
+  if (cudaMemsetAsync(base + wl.rowmax, 0, (wl.htc_cnt - wl.rowmax) + (size_t)(pb.M >> 7) * 4, st) != cudaSuccess)
+    return STAMP_ERR_CUDA;
+  CUtensorMap tx;
+  int rc = make_tmap_bf16(X, pb.M, pb.K, &tx, 128);
+  if (rc) return rc;
+  rc = tiled ? launch_htc<HTC_OUT_TILED>(tx, hp, st)
+       : a8  ? launch_htc<HTC_OUT_A8>(tx, hp, st)
+        : T_out ? launch_htc<HTC_OUT_T>(tx, hp, st)
+                : launch_htc<HTC_OUT_PUBLIC>(tx, hp, st);
+  if (rc || hp.last) return rc;
+  CqTiled rest;
+  if (tiled) {
+    rest = *tiled;
+    rest.pf_base = nullptr;   // the hints went out with the first launch
+    rest.pf_bytes = 0;
+  }
+  return run_quantize_cq(pb, c, hp.aout, STAMP_F32, a8, q_hi, q_lo, x_scale, T_out, base, wl, st, tiled ? &rest : nullptr, lv);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -834,12 +934,7 @@ static int launch_top_gemv(const int8_t* codes, const float* sx, const int8_t* w
                            float* a8v, cudaStream_t st) {
   auto kern = k_top_gemv<R>;
   const size_t smem = (size_t)R * K;
-  static size_t attr_smem = 0;
-  if (smem > attr_smem) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return STAMP_ERR_CUDA;
-    attr_smem = smem;
-  }
+  if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return rc;
   const int per_cta = (TOPG_THREADS / 32) * TOPG_CH_PER_WARP;
   if (launch_pdl(kern, dim3((unsigned)((N + per_cta - 1) / per_cta)), dim3(TOPG_THREADS), smem, st, codes, sx, w8, K, N,
                  top_levels, a8v) != cudaSuccess) {
@@ -893,7 +988,6 @@ static int weights_as_int8(const Problem& pb, const void* w, int w_format, int8_
 static __device__ __align__(256) unsigned char g_noalloc_scratch[STAMP_NOALLOC_SCRATCH_BYTES];
 
 static int noalloc_scratch_base(uint8_t** out) {
-  constexpr int MAX_DEVICES = 64;
   static std::mutex mu;
   static uint8_t* base_of[MAX_DEVICES] = {};
   int dev = -1;
@@ -909,6 +1003,69 @@ static int noalloc_scratch_base(uint8_t** out) {
   }
   *out = base_of[dev];
   return STAMP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Routes of the one-call layer and their transform+quantize stages (shared with the debug export of
+// the fused operand, so that the export runs the very kernels the layer runs).
+// ------------------------------------------------------------------------------------------
+enum FusedRoute { ROUTE_PATCH2D = 0, ROUTE_ZP_GENERAL = 1, ROUTE_TILED = 2, ROUTE_DCT_TC = 3, ROUTE_GENERAL = 4 };
+
+static FusedRoute fused_route(const Problem& pb, int x_dtype, CqChoice* cc, bool* have_cq) {
+  const bool patch_fits = (size_t)64 * pb.K * (x_dtype == STAMP_BF16 ? 2 : 4) <= 224 * 1024;
+  *have_cq = (pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, cc);
+  if (pb.transform == STAMP_T_HAAR2D && pb.levels == 3 && pb.M % 256 == 0 && (!pb.act_zp || patch_fits)) return ROUTE_PATCH2D;
+  if (pb.act_zp) return ROUTE_ZP_GENERAL;
+  if (*have_cq && pb.transform == STAMP_T_HAAR && pb.levels >= 5 && pb.n % 256 == 0) return ROUTE_TILED;
+  if (dct_tc_ok(pb, x_dtype)) return ROUTE_DCT_TC;
+  return ROUTE_GENERAL;
+}
+
+// Where the patch-order route keeps its per-row tables (the fp32 T of the general route is not materialised
+// there, so its space is reused).
+struct PatchTables {
+  float* x_inv;
+  float* sx_epi;
+  int* zp_epi;
+};
+static PatchTables patch_tables(const Problem& pb, uint8_t* base, const Workspace& wl) {
+  float* T = reinterpret_cast<float*>(base + wl.T);
+  return PatchTables{T, T + pb.M, reinterpret_cast<int*>(T + 2 * pb.M)};
+}
+
+// Patch-order route: one CTA per 8 x 8 patch finds the row maxima (or minima and maxima, for zero-point
+// codes) and writes codes in patch order.  w8 / w_sum: weight codes and the buffer of their row sums for the
+// zero-point term (w8 may be null: no sums are taken).
+static int fused_quantize_patch2d(const Problem& pb, const void* X, int x_dtype, uint8_t* base, const Workspace& wl,
+                                  const int8_t* w8, int* w_sum, cudaStream_t st) {
+  const PatchTables pt = patch_tables(pb, base, wl);
+  unsigned* rowmax = reinterpret_cast<unsigned*>(base + wl.rowmax);
+  float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
+  int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
+  if (x_dtype == STAMP_BF16)
+    return run_quantize_haar2d_patch(pb, static_cast<const __nv_bfloat16*>(X), rowmax, x_scale, pt.x_inv, a8, pt.sx_epi,
+                                     pt.zp_epi, w8, w_sum, st);
+  return run_quantize_haar2d_patch(pb, static_cast<const float*>(X), rowmax, x_scale, pt.x_inv, a8, pt.sx_epi, pt.zp_epi,
+                                   w8, w_sum, st);
+}
+
+// Tile-order route: the transform+quantize chain writes the token operand in tile order (rows of levels above
+// 8 into the table behind it).  w8: weight codes to pull towards L2 during the first launch, or null.
+static int fused_quantize_tiled(const Problem& pb, const CqChoice& cc, const void* X, int x_dtype, uint8_t* base,
+                                const Workspace& wl, const int8_t* w8, CqTiled* tl_out, cudaStream_t st) {
+  int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
+  float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
+  CqTiled tl{reinterpret_cast<int8_t*>(base + wl.a8top), reinterpret_cast<float*>(base + wl.sxtop), x_scale};
+  // The first launch of the transform chain also pulls a small weight matrix towards L2: the chain's later
+  // launches are small and leave HBM idle, and the GEMM (and the skinny top-row product before it) then
+  // start on weights that are already there.  Measured: 8 to 20 % per step up to 16 MB of codes; nothing
+  // to gain, or a loss, at 45 MB and above, whether the whole matrix or its first 16 MB are asked for.
+  if (w8 && (size_t)pb.N * pb.K <= (size_t)24 << 20) {
+    tl.pf_base = reinterpret_cast<const uint8_t*>(w8);
+    tl.pf_bytes = (long)pb.N * pb.K;
+  }
+  *tl_out = tl;
+  return run_quantize_haar(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st, &tl);
 }
 
 }  // namespace stamp
@@ -976,7 +1133,7 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   }
   CqChoice cc;
   if ((pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc))
-    return run_quantize_cq(pb, cc, X, x_dtype, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
+    return run_quantize_haar(pb, cc, X, x_dtype, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
   if (dct_tc_ok(pb, x_dtype)) {
     int8_t* a8 = reinterpret_cast<int8_t*>(base + w.a8);
     if ((rc = run_quantize_dct_tc(pb, X, a8, x_scale, base, w, st))) return rc;
@@ -1073,29 +1230,23 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
   int8_t* a8 = reinterpret_cast<int8_t*>(base + wl.a8);
   float* x_scale = reinterpret_cast<float*>(base + wl.xscale);
   float* yt = reinterpret_cast<float*>(base + wl.yt);
-  const bool patch_fits = (size_t)64 * K * (x_dtype == STAMP_BF16 ? 2 : 4) <= 224 * 1024;
-  if (pb.transform == STAMP_T_HAAR2D && pb.levels == 3 && pb.M % 256 == 0 && (!pb.act_zp || patch_fits)) {
+  CqChoice cc;
+  bool have_cq = false;
+  const FusedRoute route = fused_route(pb, x_dtype, &cc, &have_cq);
+  if (route == ROUTE_PATCH2D) {
     // Fused route of the paper's LVM transform: one CTA per 8 x 8 patch finds the row maxima (or minima and maxima,
     // for zero-point codes) and writes codes in patch order; the GEMM's epilogue inverts the four patches of its
     // 256-token tile.
-    float* x_inv = T;               // the fp32 T of the general route is not materialised here: reuse its space
-    float* sx_epi = T + pb.M;
-    int* zp_epi = reinterpret_cast<int*>(T + 2 * pb.M);
+    const PatchTables pt = patch_tables(pb, base, wl);
     const int8_t* w8p = nullptr;
     if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8p, st))) return rc;
     // (zero-point codes: the patch kernel also takes the weight row sums of the correction term)
     int* w_sum = pb.act_zp ? reinterpret_cast<int*>(base + wl.wsum) : nullptr;
-    if (x_dtype == STAMP_BF16)
-      rc = run_quantize_haar2d_patch(pb, static_cast<const __nv_bfloat16*>(X), rowmax, x_scale, x_inv, a8, sx_epi, zp_epi,
-                                     w8p, w_sum, st);
-    else
-      rc = run_quantize_haar2d_patch(pb, static_cast<const float*>(X), rowmax, x_scale, x_inv, a8, sx_epi, zp_epi, w8p,
-                                     w_sum, st);
-    if (rc) return rc;
-    return launch_gemm(a8, w8p, pb.M, N, K, sx_epi, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR2D_BF16 : EPI_HAAR2D_F32,
-                       st, bias, nullptr, 0, pb.act_zp ? zp_epi : nullptr, w_sum, pb.grid_w, pb.n);
+    if ((rc = fused_quantize_patch2d(pb, X, x_dtype, base, wl, w8p, w_sum, st))) return rc;
+    return launch_gemm(a8, w8p, pb.M, N, K, pt.sx_epi, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR2D_BF16 : EPI_HAAR2D_F32,
+                       st, bias, nullptr, 0, pb.act_zp ? pt.zp_epi : nullptr, w_sum, pb.grid_w, pb.n);
   }
-  if (pb.act_zp) {
+  if (route == ROUTE_ZP_GENERAL) {
     // zero-point codes: transform, min-max quantizer, GEMM with the zero-point term in its epilogue, inverse
     int* x_zero = reinterpret_cast<int*>(base + wl.xzero);
     int* w_sum = reinterpret_cast<int*>(base + wl.wsum);
@@ -1109,25 +1260,15 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
       return rc;
     return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
   }
-  CqChoice cc;
-  const bool have_cq = (pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc);
-  if (have_cq && pb.transform == STAMP_T_HAAR && pb.levels >= 5 && pb.n % 256 == 0) {
+  if (route == ROUTE_TILED) {
     // Fused route: the transform+quantize kernel writes the token operand in tile order, the GEMM's
     // epilogue de-quantizes and inverts the (up to) 8 levels that close inside its 256-token tile.
     // Levels above 8 live in M / 256 extra rows: a small GEMM and the general inverse turn them into
     // the level-8 approximation of every tile first.
-    CqTiled tl{reinterpret_cast<int8_t*>(base + wl.a8top), reinterpret_cast<float*>(base + wl.sxtop), x_scale};
     const int8_t* w8f = nullptr;
     if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8f, st))) return rc;
-    // The first launch of the transform chain also pulls a small weight matrix towards L2: the chain's later
-    // launches are small and leave HBM idle, and the GEMM (and the skinny top-row product before it) then
-    // start on weights that are already there.  Measured: 8 to 20 % per step up to 16 MB of codes; nothing
-    // to gain, or a loss, at 45 MB and above, whether the whole matrix or its first 16 MB are asked for.
-    if ((size_t)N * K <= (size_t)24 << 20) {
-      tl.pf_base = reinterpret_cast<const uint8_t*>(w8f);
-      tl.pf_bytes = (long)N * K;
-    }
-    if ((rc = run_quantize_cq(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st, &tl))) return rc;
+    CqTiled tl{};
+    if ((rc = fused_quantize_tiled(pb, cc, X, x_dtype, base, wl, w8f, &tl, st))) return rc;
     const float* a8v = nullptr;
     if (pb.levels > 8) {
       float* yttop = reinterpret_cast<float*>(base + wl.yttop);
@@ -1154,7 +1295,7 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     return launch_gemm(a8, w8f, pb.M, N, K, x_scale, w_scale, Y, y_dtype == STAMP_BF16 ? EPI_HAAR_BF16 : EPI_HAAR_F32, st,
                        bias, a8v, pb.levels < 8 ? pb.levels : 8);
   }
-  if (dct_tc_ok(pb, x_dtype)) {
+  if (route == ROUTE_DCT_TC) {
     if ((rc = run_quantize_dct_tc(pb, X, a8, x_scale, base, wl, st))) return rc;
     const int8_t* w8d = nullptr;
     if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8d, st))) return rc;
@@ -1166,7 +1307,7 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
   }
   if (have_cq) {
-    if ((rc = run_quantize_cq(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
+    if ((rc = run_quantize_haar(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
   } else {
     if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
       return rc;
@@ -1226,8 +1367,8 @@ int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, i
   uint8_t* base = static_cast<uint8_t*>(ws);
   CqChoice cc;
   if ((pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc))  // the product path's kernel with the fp32 export on
-    return run_quantize_cq(pb, cc, X, x_dtype, nullptr, nullptr, nullptr, reinterpret_cast<float*>(base + wl.xscale), T,
-                           base, wl, static_cast<cudaStream_t>(stream));
+    return run_quantize_haar(pb, cc, X, x_dtype, nullptr, nullptr, nullptr, reinterpret_cast<float*>(base + wl.xscale), T,
+                             base, wl, static_cast<cudaStream_t>(stream));
   return run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + wl.ping),
                                reinterpret_cast<float*>(base + wl.pong), reinterpret_cast<float*>(base + wl.dctmat),
                                static_cast<cudaStream_t>(stream));
@@ -1263,6 +1404,43 @@ int stamp_debug_gemm_i32(const stamp_config* cfg, const void* q_hi, const void* 
   return launch_gemm(a8, w8, pb.M, N, K, nullptr, nullptr, acc, EPI_RAW_I32, st);
 }
 
+int stamp_debug_fused_operand(const stamp_config* cfg, const void* X, int x_dtype, int B, int L, int K, int N,
+                              int8_t* codes, float* factor, int32_t* level, int32_t* zero, void* ws, size_t ws_bytes,
+                              void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, N, true, &pb);
+  if (rc) return rc;
+  if (!X || !codes || !factor || !level || !dtype_ok(x_dtype)) return STAMP_ERR_INVALID_ARG;
+  const Workspace wl = layout(pb);
+  if ((rc = check_ws(wl, ws, ws_bytes))) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  const int8_t* a8 = reinterpret_cast<const int8_t*>(base + wl.a8);
+  CqChoice cc;
+  bool have_cq = false;
+  const FusedRoute route = fused_route(pb, x_dtype, &cc, &have_cq);
+  if (route == ROUTE_TILED) {
+    CqTiled tl{};
+    if ((rc = fused_quantize_tiled(pb, cc, X, x_dtype, base, wl, nullptr, &tl, st))) return rc;
+    k_debug_gather_tiled<<<(unsigned)pb.M, 256, 0, st>>>(a8, tl.sx_epi, tl.sx_top, pb.M, pb.n, pb.levels, K, codes, factor,
+                                                         level);
+    STAMP_CHECK_LAUNCH();
+    if (zero && cudaMemsetAsync(zero, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+    return STAMP_OK;
+  }
+  if (route == ROUTE_PATCH2D) {
+    if (pb.act_zp && !zero) return STAMP_ERR_INVALID_ARG;
+    if ((rc = fused_quantize_patch2d(pb, X, x_dtype, base, wl, nullptr, nullptr, st))) return rc;
+    const PatchTables pt = patch_tables(pb, base, wl);
+    k_debug_gather_patch<<<(unsigned)pb.M, 256, 0, st>>>(a8, pt.sx_epi, pb.act_zp ? pt.zp_epi : nullptr, pb.M, pb.n,
+                                                         pb.grid_w, K, codes, factor, level, zero);
+    STAMP_CHECK_LAUNCH();
+    return STAMP_OK;
+  }
+  return STAMP_ERR_UNSUPPORTED;   // the other routes keep their operand in logical order: stamp_quantize shows it
+}
+
 int stamp_last_device_status(void* stream, int* status) {
   if (!status) return STAMP_ERR_INVALID_ARG;
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return STAMP_ERR_CUDA;
@@ -1280,6 +1458,17 @@ int stamp_profile_gemm_events(void* start_event, void* stop_event) {
   if ((start_event == nullptr) != (stop_event == nullptr)) return STAMP_ERR_INVALID_ARG;
   t_gemm_ev_start = static_cast<cudaEvent_t>(start_event);
   t_gemm_ev_stop = static_cast<cudaEvent_t>(stop_event);
+  return STAMP_OK;
+}
+
+int stamp_measure_i8_mma_issue(int nbatch, long long* ops_out, void* stream) {
+  t_launches = 0;
+  if (nbatch <= 0 || nbatch > (1 << 20) || !ops_out) return STAMP_ERR_INVALID_ARG;
+  if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(k_peak_mma_i8), PEAK_SMEM)) return rc;
+  const int grid = sm_count();
+  k_peak_mma_i8<<<grid, PEAK_THREADS, PEAK_SMEM, static_cast<cudaStream_t>(stream)>>>(nbatch);
+  STAMP_CHECK_LAUNCH();
+  *ops_out = (long long)grid * nbatch * PEAK_BATCH * (2LL * 128 * 256 * 32);
   return STAMP_OK;
 }
 
