@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
       for (long item = blockIdx.x; item < nitems; item += gridDim.x) {
         const long rb = item / p.nchunks;
         const int c = static_cast<int>(item - rb * p.nchunks);
-        if (!ptx::mbar_wait_bounded(&sempty[stage], phase ^ 1u, abort_word, HTC_WAIT_LIMIT)) {
+        if (!ptx::mbar_wait_bounded_sleepy(&sempty[stage], phase ^ 1u, abort_word, HTC_WAIT_LIMIT)) {
           ok = false;
           break;
         }
@@ -262,7 +262,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
       // also hands the stage back to the producer
       auto product = [&](int stage, bool release_stage) -> bool {
         const int buf = static_cast<int>(job & (HTC_NBUF - 1));
-        if (!ptx::mbar_wait_bounded(&tempty[buf], static_cast<uint32_t>(((job / HTC_NBUF) & 1) ^ 1), abort_word, HTC_WAIT_LIMIT))
+        if (!ptx::mbar_wait_bounded_sleepy(&tempty[buf], static_cast<uint32_t>(((job / HTC_NBUF) & 1) ^ 1), abort_word, HTC_WAIT_LIMIT))
           return false;
         ptx::tc_fence_after();
         const uint32_t bbase = ptx::smem_u32(b_sm + stage * HTC_TILE_BYTES);
@@ -281,7 +281,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
       for (long t = 0; t < n_local + HTC_LAG && ok; ++t) {
         if (t < n_local) {   // P1 of item t
           const int stage = static_cast<int>(t % HTC_STAGES);
-          if (!ptx::mbar_wait_bounded(&sfull[stage], static_cast<uint32_t>((t / HTC_STAGES) & 1), abort_word, HTC_WAIT_LIMIT) ||
+          if (!ptx::mbar_wait_bounded_sleepy(&sfull[stage], static_cast<uint32_t>((t / HTC_STAGES) & 1), abort_word, HTC_WAIT_LIMIT) ||
               !product(stage, false)) {
             ok = false;
             break;
@@ -320,7 +320,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     long k = 0;
     for (long i = set; i < n_local; i += 2, ++k) {
       const long rb = (blockIdx.x + i * gridDim.x) / p.nchunks;
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&pfull[set], static_cast<uint32_t>(k & 1), abort_word, HTC_WAIT_LIMIT))) {
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&pfull[set], static_cast<uint32_t>(k & 1), abort_word, HTC_WAIT_LIMIT))) {
         ok = false;
         break;
       }
@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     auto job_p2 = [&](long i) -> long { return i + HTC_LAG < n_local ? 2 * i + HTC_LAG + 1 : n_local + i; };
     auto wait_acc = [&](long jb) -> bool {
       const int buf = static_cast<int>(jb & (HTC_NBUF - 1));
-      const bool got = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(&tfull[buf], static_cast<uint32_t>((jb / HTC_NBUF) & 1),
+      const bool got = __all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&tfull[buf], static_cast<uint32_t>((jb / HTC_NBUF) & 1),
                                                                       abort_word, HTC_WAIT_LIMIT));
       ptx::tc_fence_after();
       return got;
@@ -515,7 +515,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
           m1 = fmaxf(m1, fabsf(__uint_as_float(v[1][q4])));
         }
         // hand the maxima to the set's publisher warp (its slot is clear once it has taken the previous tile's)
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&pempty[set], static_cast<uint32_t>(((i >> 1) & 1) ^ 1), abort_word,
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&pempty[set], static_cast<uint32_t>(((i >> 1) & 1) ^ 1), abort_word,
                                                             HTC_WAIT_LIMIT))) {
           ok = false;
           break;

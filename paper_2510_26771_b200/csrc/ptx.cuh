@@ -89,6 +89,31 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   }
 }
 
+// The same bounded wait for threads that expect to wait long: try_wait is given a suspend-time hint, so the
+// thread sleeps in hardware until the phase completes (or the hint runs out) instead of spinning through the
+// issue slots of the warps that are working.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded_sleepy(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_word,
+                                                         long long limit_cycles) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (mbar_try_wait_hint(bar, parity, 20000u)) return true;
+    if (*abort_word != 0u) return false;
+    if (clock64() - t0 > limit_cycles) return false;
+  }
+}
+
 // The same bounded wait for a barrier completed by other CTAs of the cluster (acquire at cluster scope).
 __device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_word,
                                                           long long limit_cycles) {
