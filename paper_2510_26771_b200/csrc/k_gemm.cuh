@@ -21,6 +21,15 @@
 //              half of the accumulator's columns
 // Every mbarrier wait is bounded; when one expires the CTA raises the device status word,
 // drains its outstanding copies, frees TMEM and returns.
+//
+// PAIR = true: the same kernel on CTA pairs (tcgen05 cta_group::2, clusters of two).  A pair owns a tile of 256
+// channels x 256 tokens: either CTA stages ITS 128 channels and ITS 128 tokens of every K block (32 KB per
+// stage instead of 48), the even-ranked CTA issues one M256 x N256 x K32 instruction for both, and either
+// CTA's epilogue drains the 128 accumulator lanes that land in its own tensor memory.  With half of the token
+// operand coming from the neighbour, a CTA moves 16 KB through its shared memory per instruction instead of
+// 24 KB, which is what kept the single-CTA main loop below the tensor rate.  The odd-ranked CTA's copies are
+// counted on the even-ranked CTA's barrier; stage and accumulator hand-backs reach both CTAs with one
+// multicast commit; the epilogue threads of both CTAs release an accumulator on the issuing CTA's barrier.
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
@@ -65,10 +74,10 @@ constexpr int GEMM_EPI_THREADS = 256;   // two epilogue warps per TMEM lane quar
 constexpr int GEMM_THREADS = 64 + GEMM_EPI_THREADS;
 constexpr long long GEMM_WAIT_LIMIT = 4000000000LL;  // SM clocks (~2 s) before a wait gives up
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, bool PAIR = false>
 struct GemmSmem {
   static constexpr int W_BYTES = GEMM_BM * GEMM_BK;
-  static constexpr int X_BYTES = BN * GEMM_BK;
+  static constexpr int X_BYTES = (PAIR ? BN / 2 : BN) * GEMM_BK;   // a CTA of a pair stages half of the token tile
   static constexpr int STAGE_BYTES = W_BYTES + X_BYTES;
   static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
   // full[STAGES], empty[STAGES], tfull[2], tempty[2], then tmem base + abort word
@@ -91,10 +100,11 @@ __device__ __forceinline__ void tile_coords(int tile, int ch_tiles, int tok_tile
   ch_t = first + (rem - tok_t * height);
 }
 
-template <int BN, int STAGES, int EPI>
+template <int BN, int STAGES, int EPI, bool PAIR = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
     k_gemm_i8(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, GemmParams p) {
-  using SM = GemmSmem<BN, STAGES>;
+  using SM = GemmSmem<BN, STAGES, PAIR>;
+  static_assert(!PAIR || BN == 256, "a pair works on 256-token tiles");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + SM::BAR_OFFSET);
@@ -108,10 +118,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int ch_tiles = (p.n_out + GEMM_BM - 1) / GEMM_BM;
+  // PAIR: a work item is a pair tile of 2 x 128 channels; this CTA takes channel tile 2 ch_t + rank of it
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  constexpr int CH_PER_TILE = PAIR ? 2 * GEMM_BM : GEMM_BM;
+  const int ch_tiles = (p.n_out + CH_PER_TILE - 1) / CH_PER_TILE;
   const int tok_tiles = (p.m_tok + BN - 1) / BN;
   const int num_tiles = ch_tiles * tok_tiles;
   const int num_kb = p.k / GEMM_BK;
+  const int tile0 = PAIR ? blockIdx.x >> 1 : blockIdx.x;
+  const int tile_step = PAIR ? gridDim.x >> 1 : gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -120,7 +135,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&tfull[a], 1);
-      ptx::mbar_init(&tempty[a], GEMM_EPI_THREADS);
+      ptx::mbar_init(&tempty[a], PAIR ? 2 * GEMM_EPI_THREADS : GEMM_EPI_THREADS);
     }
     *abort_word = 0;
     ptx::fence_mbar_init();
@@ -128,11 +143,18 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     ptx::prefetch_tensormap(&tmap_x);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, 2 * BN);
-    ptx::tmem_relinquish();
+    if constexpr (PAIR) {
+      ptx::tmem_alloc_pair(tmem_slot, 2 * BN);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(tmem_slot, 2 * BN);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  // both CTAs of a pair have initialised their barriers before either signals the other's
+  if constexpr (PAIR) ptx::cluster_sync();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   ptx::grid_dependency_wait();   // operands and scales come from the kernels launched before
@@ -144,7 +166,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       uint32_t phase = 0;
       uint32_t armed = 0, armed_parity = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int tile = tile0; tile < num_tiles && ok; tile += tile_step) {
         int ch_t, tok_t;
         tile_coords(tile, ch_tiles, tok_tiles, p.group, ch_t, tok_t);
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -153,9 +175,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
             break;
           }
           uint8_t* ws = smem + stage * SM::STAGE_BYTES;
+          if constexpr (PAIR) {
+            // this CTA's 128 channels and 128 tokens; all four copies of the pair are counted on the even CTA's barrier
+            const uint32_t bar0 = ptx::mapa(ptx::smem_u32(&full[stage]), 0u);
+            if (rank == 0) ptx::mbar_arrive_expect_tx(&full[stage], 2 * SM::STAGE_BYTES);
+            ptx::tma_load_2d_pair(ws, &tmap_w, bar0, kb * GEMM_BK, (2 * ch_t + static_cast<int>(rank)) * GEMM_BM);
+            ptx::tma_load_2d_pair(ws + SM::W_BYTES, &tmap_x, bar0, kb * GEMM_BK, tok_t * BN + static_cast<int>(rank) * (BN / 2));
+          } else {
           ptx::mbar_arrive_expect_tx(&full[stage], SM::STAGE_BYTES);
           ptx::tma_load_2d(ws, &tmap_w, &full[stage], kb * GEMM_BK, ch_t * GEMM_BM);
           ptx::tma_load_2d(ws + SM::W_BYTES, &tmap_x, &full[stage], kb * GEMM_BK, tok_t * BN);
+          }
           armed |= 1u << stage;
           armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == STAGES) {
@@ -171,20 +201,21 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
         for (int s = 0; s < STAGES; ++s)
           if (armed & (1u << s)) {
             const long long t0 = clock64();
-            while (!ptx::mbar_try_wait(&full[s], (armed_parity >> s) & 1u) && clock64() - t0 < 2000000LL) {
+            // (the odd CTA of a pair has no barrier of its own to watch: it just gives its copies the time)
+            while ((rank != 0 || !ptx::mbar_try_wait(&full[s], (armed_parity >> s) & 1u)) && clock64() - t0 < 2000000LL) {
             }
           }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::make_i8_idesc(GEMM_BM, BN);
+    // ------------------------------------------------------------------ MMA issuer (PAIR: the even-ranked CTA's, for both)
+    if (rank == 0 && ptx::elect_one()) {
+      constexpr uint32_t idesc = ptx::make_i8_idesc(PAIR ? 2 * GEMM_BM : GEMM_BM, BN);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++it) {
         const int a = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1u;
         if (!ptx::mbar_wait_bounded(&tempty[a], acc_phase ^ 1u, abort_word, GEMM_WAIT_LIMIT)) {
@@ -205,15 +236,21 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
           for (int k = 0; k < GEMM_BK / 32; ++k) {
             const uint64_t adesc = ptx::make_kmajor_sw128_desc(wa + k * 32);
             const uint64_t bdesc = ptx::make_kmajor_sw128_desc(xa + k * 32);
-            ptx::mma_i8_ss(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            if constexpr (PAIR)
+              ptx::mma_i8_ss_pair(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            else
+              ptx::mma_i8_ss(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          ptx::tc_commit(&empty[stage]);  // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if constexpr (PAIR) ptx::tc_commit_pair(&empty[stage], 3); else ptx::tc_commit(&empty[stage]);
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1u;
           }
         }
-        if (ok) ptx::tc_commit(&tfull[a]);  // accumulator complete
+        if (ok) {                           // accumulator complete (in both CTAs of a pair)
+          if constexpr (PAIR) ptx::tc_commit_pair(&tfull[a], 3); else ptx::tc_commit(&tfull[a]);
+        }
       }
       if (!ok) {
         *abort_word = 1;
@@ -228,9 +265,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
     const int ep_tid = threadIdx.x - 64;  // 0..255
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+    const uint32_t tempty_bar0 = PAIR ? ptx::mapa(ptx::smem_u32(&tempty[0]), 0u) : 0u;   // the issuing CTA's barriers
+    for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++it) {
       int ch_t, tok_t;
       tile_coords(tile, ch_tiles, tok_tiles, p.group, ch_t, tok_t);
+      if constexpr (PAIR) ch_t = 2 * ch_t + static_cast<int>(rank);
       const int a = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1u;
       const int ch = ch_t * GEMM_BM + row;
@@ -463,7 +502,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
       }
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&tempty[a]);
+      if constexpr (PAIR) ptx::mbar_arrive_cluster(tempty_bar0 + static_cast<uint32_t>(a) * 8u); else ptx::mbar_arrive(&tempty[a]);
     }
     if (!ok) {
       *abort_word = 1;
@@ -473,9 +512,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 
   ptx::tc_fence_before();
   __syncthreads();
+  // neither CTA of a pair lets go of its shared and tensor memory while the other may still signal into it
+  if constexpr (PAIR) ptx::cluster_sync();
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, 2 * BN);
+    if constexpr (PAIR) ptx::tmem_dealloc_pair(tmem_base, 2 * BN); else ptx::tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 

@@ -293,18 +293,37 @@ static int launch_dct_tc(const CUtensorMap& ta, const CUtensorMap& tb0, const CU
   return STAMP_OK;
 }
 
-template <int BN, int STAGES, int EPI>
+template <int BN, int STAGES, int EPI, bool PAIR = false>
 static int launch_gemm_t(const CUtensorMap& tw, const CUtensorMap& tx, const GemmParams& gp, cudaStream_t st) {
-  using SM = GemmSmem<BN, STAGES>;
-  auto kern = k_gemm_i8<BN, STAGES, EPI>;
+  using SM = GemmSmem<BN, STAGES, PAIR>;
+  auto kern = k_gemm_i8<BN, STAGES, EPI, PAIR>;
   if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), SM::DYN_BYTES)) return rc;
-  const int ch_tiles = (gp.n_out + GEMM_BM - 1) / GEMM_BM;
+  const int ch_tiles = (gp.n_out + (PAIR ? 2 : 1) * GEMM_BM - 1) / ((PAIR ? 2 : 1) * GEMM_BM);
   const int tok_tiles = (gp.m_tok + BN - 1) / BN;
   const int tiles = ch_tiles * tok_tiles;
-  const int grid = tiles < sm_count() ? tiles : sm_count();
+  const int slots = PAIR ? sm_count() / 2 : sm_count();
+  const int grid = (tiles < slots ? tiles : slots) * (PAIR ? 2 : 1);
   const bool timed = t_gemm_ev_start && t_gemm_ev_stop;
   if (timed) cudaEventRecord(t_gemm_ev_start, st);
-  launch_pdl(kern, dim3((unsigned)grid), dim3(GEMM_THREADS), SM::DYN_BYTES, st, tw, tx, gp);
+  if (PAIR) {
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)grid);
+    lc.blockDim = dim3(GEMM_THREADS);
+    lc.dynamicSmemBytes = SM::DYN_BYTES;
+    lc.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at;
+    lc.numAttrs = 2;
+    cudaLaunchKernelEx(&lc, kern, tw, tx, gp);
+  } else {
+    launch_pdl(kern, dim3((unsigned)grid), dim3(GEMM_THREADS), SM::DYN_BYTES, st, tw, tx, gp);
+  }
   if (timed) cudaEventRecord(t_gemm_ev_stop, st);
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
@@ -333,30 +352,31 @@ static int launch_gemm(const int8_t* a8, const int8_t* w8, long M, int N, int K,
   CUtensorMap tw, tx;
   int rc = make_tmap_i8(w8, N, K, GEMM_BM, &tw);
   if (rc) return rc;
+  // 256 tokens and more: CTA pairs, each CTA staging 128 tokens of the pair's 256-token tile
   const bool wide = M >= 256;
-  rc = make_tmap_i8(a8, M, K, wide ? 256 : 128, &tx);
+  rc = make_tmap_i8(a8, M, K, 128, &tx);
   if (rc) return rc;
   if (epi == EPI_HAAR_F32 || epi == EPI_HAAR_BF16) {
     if (!wide || M % 256 != 0 || depth < 5 || depth > 8) return STAMP_ERR_UNSUPPORTED;
-    if (epi == EPI_HAAR_F32) return launch_gemm_t<256, 4, EPI_HAAR_F32>(tw, tx, gp, st);
-    return launch_gemm_t<256, 4, EPI_HAAR_BF16>(tw, tx, gp, st);
+    if (epi == EPI_HAAR_F32) return launch_gemm_t<256, 6, EPI_HAAR_F32, true>(tw, tx, gp, st);
+    return launch_gemm_t<256, 6, EPI_HAAR_BF16, true>(tw, tx, gp, st);
   }
   if (epi == EPI_DEQUANT_BF16X2)
-    return wide ? launch_gemm_t<256, 4, EPI_DEQUANT_BF16X2>(tw, tx, gp, st)
+    return wide ? launch_gemm_t<256, 6, EPI_DEQUANT_BF16X2, true>(tw, tx, gp, st)
                 : launch_gemm_t<128, 6, EPI_DEQUANT_BF16X2>(tw, tx, gp, st);
   if (epi == EPI_HAAR2D_F32 || epi == EPI_HAAR2D_BF16) {
     if (!wide || M % 256 != 0 || grid_w < 8 || grid_w % 8 != 0 || n_block % (8 * grid_w) != 0) return STAMP_ERR_UNSUPPORTED;
-    if (epi == EPI_HAAR2D_F32) return launch_gemm_t<256, 4, EPI_HAAR2D_F32>(tw, tx, gp, st);
-    return launch_gemm_t<256, 4, EPI_HAAR2D_BF16>(tw, tx, gp, st);
+    if (epi == EPI_HAAR2D_F32) return launch_gemm_t<256, 6, EPI_HAAR2D_F32, true>(tw, tx, gp, st);
+    return launch_gemm_t<256, 6, EPI_HAAR2D_BF16, true>(tw, tx, gp, st);
   }
   if (epi == EPI_DEQUANT_ZP_F32) {
     if (!x_zero || !w_sum) return STAMP_ERR_INVALID_ARG;
-    return wide ? launch_gemm_t<256, 4, EPI_DEQUANT_ZP_F32>(tw, tx, gp, st)
+    return wide ? launch_gemm_t<256, 6, EPI_DEQUANT_ZP_F32, true>(tw, tx, gp, st)
                 : launch_gemm_t<128, 6, EPI_DEQUANT_ZP_F32>(tw, tx, gp, st);
   }
   if (wide) {
-    if (epi == EPI_DEQUANT_F32) return launch_gemm_t<256, 4, EPI_DEQUANT_F32>(tw, tx, gp, st);
-    return launch_gemm_t<256, 4, EPI_RAW_I32>(tw, tx, gp, st);
+    if (epi == EPI_DEQUANT_F32) return launch_gemm_t<256, 6, EPI_DEQUANT_F32, true>(tw, tx, gp, st);
+    return launch_gemm_t<256, 6, EPI_RAW_I32, true>(tw, tx, gp, st);
   }
   if (epi == EPI_DEQUANT_F32) return launch_gemm_t<128, 6, EPI_DEQUANT_F32>(tw, tx, gp, st);
   return launch_gemm_t<128, 6, EPI_RAW_I32>(tw, tx, gp, st);
