@@ -261,6 +261,8 @@ def quick_reading(st, cfg, y_t, steps):
     Y = torch.empty((cfg.B, cfg.L, cfg.N), dtype=y_t, device="cuda")
     ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
     g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()      # (an event has no handle to pass to the library before its first record)
+    g1.record()
 
     def step(i):
         st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], w_fmt, w_scale, bias, ws, out=Y)

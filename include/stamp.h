@@ -256,6 +256,12 @@ int stamp_last_device_status(void* stream, int* status);
  * (each launch re-records the pair).  Pass NULLs to switch it off.  Events are cudaEvent_t. */
 int stamp_profile_gemm_events(void* start_event, void* stop_event);
 
+/* Test hook for the failure path: launches one thread that waits, with the same bounded wait the product
+ * kernels use, on a barrier nobody completes.  After limit_cycles SM clocks (1 .. 2e9) the wait gives up, the
+ * kernel records STAMP_ERR_TIMEOUT in the device status word and returns normally; the next
+ * stamp_last_device_status() reports it once.  Nothing faults or hangs.  No counterpart in the paper. */
+int stamp_debug_expire_wait(long long limit_cycles, void* stream);
+
 /* Measurement: the rate of the tensor cores' int8 instruction alone.  Launches one CTA per SM; each issues
  * nbatch * 64 tcgen05.mma kind::i8 instructions (M128 x N256 x K32, int32 accumulators in tensor memory) on
  * operand tiles that stay in shared memory -- no loads in the loop, waits bounded -- and *ops_out receives the

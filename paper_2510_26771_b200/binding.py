@@ -24,7 +24,7 @@ EXPORTS = (
     "stamp_linear_fused_host", "stamp_profile_gemm_events", "stamp_debug_transform",
     "stamp_debug_unpack_codes", "stamp_debug_gemm_i32", "stamp_last_device_status",
     "stamp_last_launch_count", "stamp_status_string", "stamp_inverse_noalloc", "stamp_debug_fused_operand",
-    "stamp_measure_i8_mma_issue",
+    "stamp_measure_i8_mma_issue", "stamp_debug_expire_wait",
 )
 
 
@@ -272,6 +272,11 @@ def stamp_measure_i8_mma_issue(nbatch: int) -> int:
     ops = ctypes.c_longlong(0)
     _check(lib().stamp_measure_i8_mma_issue(int(nbatch), ctypes.byref(ops), _stream()), "stamp_measure_i8_mma_issue")
     return int(ops.value)
+
+
+def stamp_debug_expire_wait(limit_cycles: int) -> None:
+    """Launch the test kernel whose bounded wait runs out after limit_cycles SM clocks (device status: time-out)."""
+    _check(lib().stamp_debug_expire_wait(ctypes.c_longlong(int(limit_cycles)), _stream()), "stamp_debug_expire_wait")
 
 
 def stamp_last_launch_count() -> int:

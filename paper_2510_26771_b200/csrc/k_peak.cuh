@@ -70,4 +70,23 @@ __global__ void __launch_bounds__(PEAK_THREADS, 1) k_peak_mma_i8(int nbatch) {
   }
 }
 
+// Test kernel for the failure path every kernel of the library shares: one thread waits, with the bounded wait
+// the product kernels use, on an mbarrier that nobody will ever complete.  After `limit_cycles` SM clocks the
+// wait gives up, the thread records STAMP_ERR_TIMEOUT in the device status word and the kernel returns normally:
+// nothing faults, traps or hangs, and the context stays usable.
+__global__ void __launch_bounds__(32, 1) k_expire_wait(long long limit_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_word;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    abort_word = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncwarp();
+  if (threadIdx.x == 0 && !ptx::mbar_wait_bounded(&bar, 0u, &abort_word, limit_cycles)) {
+    abort_word = 1;
+    raise_device_status(STAMP_ERR_TIMEOUT);
+  }
+}
+
 }  // namespace stamp

@@ -1492,6 +1492,14 @@ int stamp_measure_i8_mma_issue(int nbatch, long long* ops_out, void* stream) {
   return STAMP_OK;
 }
 
+int stamp_debug_expire_wait(long long limit_cycles, void* stream) {
+  t_launches = 0;
+  if (limit_cycles <= 0 || limit_cycles > 2000000000LL) return STAMP_ERR_INVALID_ARG;
+  k_expire_wait<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(limit_cycles);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
 int stamp_last_launch_count(void) { return t_launches; }
 
 const char* stamp_status_string(int status) {

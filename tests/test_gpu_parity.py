@@ -434,3 +434,57 @@ def test_fused_call_can_be_captured_in_a_cuda_graph(st):
             assert torch.equal(out, want)
         assert st.stamp_last_device_status() == 0
 
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_context_usable(st):
+    """Failure detection without a fault: a kernel waits on a barrier nobody completes; its bounded wait gives up
+    after about a millisecond, the status word reads time-out exactly once, and the library keeps working."""
+    import torch
+    assert st.stamp_last_device_status() == 0
+    st.stamp_debug_expire_wait(2_000_000)
+    assert st.stamp_last_device_status() == 5          # STAMP_ERR_TIMEOUT ...
+    assert "wait" in st.status_string(5)
+    assert st.stamp_last_device_status() == 0          # ... reported once, then cleared
+    # the context is intact: a layer call still gives the right answer
+    cfg = gen.scaled(gen.config_llm_up(), B=1, L=512, K=256, N=136)
+    c = _cfg_struct(st, cfg)
+    W, bias = gen.make_weight(cfg), gen.make_bias(cfg)
+    wq, wsc = st.stamp_quantize_weights(c, H.to_device(W, cfg.dtype))
+    bd = torch.from_numpy(bias).cuda()
+    ws = st.alloc_workspace(c, cfg.B, cfg.L, cfg.K, cfg.N)
+    Xz = torch.zeros((cfg.B, cfg.L, cfg.K), dtype=torch.bfloat16, device="cuda")
+    Y = st.stamp_linear_fused(c, Xz, wq, st.W_PACKED4, wsc, bd, ws)
+    assert torch.equal(Y.reshape(-1, cfg.N), bd.expand(cfg.M, cfg.N))
+    assert st.stamp_last_device_status() == 0
+
+
+@pytest.mark.parametrize("name", ["tiny", "ragged", "blocked", "dct_blocks", "haar2d_oblong", "wide_k8192"])
+def test_guard_bands_around_workspace_and_output_stay_intact(st, name):
+    """Canaries: the workspace and the output are carved out of larger allocations whose margins hold a pattern.  After
+    the public calls have run on ragged shapes (tiles that hang over the edge in every direction) the margins must
+    be untouched -- no kernel writes outside the buffers it was given."""
+    import torch
+    cfg = CASES[name]
+    c = _cfg_struct(st, cfg)
+    B, L, K, N = cfg.B, cfg.L, cfg.K, cfg.N
+    X, W, bias = gen.make_activation(cfg), gen.make_weight(cfg), gen.make_bias(cfg)
+    Xd, Wd, bd = H.to_device(X, cfg.dtype), H.to_device(W, cfg.dtype), torch.from_numpy(bias).cuda()
+    guard = 1 << 16
+    need = st.stamp_workspace_bytes(c, B, L, K, N)
+    raw = torch.full((need + 2 * guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    ws = raw[guard:guard + need]
+    assert ws.data_ptr() % 256 == 0
+    for out_dtype, esz in ((torch.float32, 4), (torch.bfloat16, 2)):
+        ybytes = B * L * N * esz
+        yraw = torch.full((ybytes + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+        Y = yraw[guard:guard + ybytes].view(out_dtype).reshape(B, L, N)
+        wq, wsc = st.stamp_quantize_weights(c, Wd)
+        q_hi, q_lo, xs = st.stamp_quantize(c, Xd, ws)
+        Yt = st.stamp_linear(c, q_hi, q_lo, xs, wq, st.W_PACKED4, wsc, B, L, K, N, ws)
+        st.stamp_inverse(c, Yt, bd, ws, out=Y)
+        st.stamp_linear_fused(c, Xd, wq, st.W_PACKED4, wsc, bd, ws, out=Y)
+        st.stamp_debug_transform(c, Xd, ws)
+        torch.cuda.synchronize()
+        assert bool((raw[:guard] == 0xA5).all()) and bool((raw[guard + need:] == 0xA5).all()), "workspace overrun"
+        assert bool((yraw[:guard] == 0x5A).all()) and bool((yraw[guard + ybytes:] == 0x5A).all()), "output overrun"
+    assert st.stamp_last_device_status() == 0
