@@ -41,7 +41,8 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_T_IDENTITY = 0, ORACLE_T_HAAR = 1, ORACLE_T_DCT2 = 2, ORACLE_T_HAAR2D = 3, ORACLE_T_WHT = 4 };
+enum { ORACLE_T_IDENTITY = 0, ORACLE_T_HAAR = 1, ORACLE_T_DCT2 = 2, ORACLE_T_HAAR2D = 3, ORACLE_T_WHT = 4,
+       ORACLE_T_HAAR_SKIP1 = 5 };
 
 int oracle_num_threads(void) {
 #ifdef _OPENMP
@@ -81,6 +82,32 @@ static void haar_forward(double* v, int n, int levels, double* tmp) {
   }
 }
 
+/* Haar analysis of a block whose FIRST token is left alone (App. "Experimental details / LLMs", STaMP paragraph:
+ * the first token of an LLM sequence carries massive outliers, stays at 8 bits, and the sequence transform is
+ * not applied to it).  The paper gives no rule for the odd number of tokens that remain; the reading taken here:
+ * the step pairs neighbours as usual and an element without a partner is CARRIED into the low-pass half
+ * unchanged (so a step on m entries yields ceil(m/2) averages-or-carried and floor(m/2) differences, and is
+ * still orthonormal: 2 x 2 rotations plus a 1 x 1 identity).  v[0] is the excluded token; the transform acts on
+ * v[1..n-1].  Output order: [token 0 | a_levels | d_levels | ... | d_1]. */
+static void haar_step_carry(double* v, int len, double* tmp) {
+  const double r = 1.0 / sqrt(2.0);
+  int pairs = len / 2, lows = len - pairs;   /* lows = ceil(len / 2) */
+  for (int i = 0; i < pairs; ++i) {
+    tmp[i] = (v[2 * i] + v[2 * i + 1]) * r;
+    tmp[lows + i] = (v[2 * i] - v[2 * i + 1]) * r;
+  }
+  if (len & 1) tmp[pairs] = v[len - 1];      /* no partner: carried, unscaled */
+  memcpy(v, tmp, sizeof(double) * (size_t)len);
+}
+
+static void haar_forward_skip_first(double* v, int n, int levels, double* tmp) {
+  int len = n - 1;
+  for (int l = 0; l < levels && len > 1; ++l) {
+    haar_step_carry(v + 1, len, tmp);
+    len = len - len / 2;
+  }
+}
+
 static int ilog2_exact(int n) {
   int l = 0;
   while ((1 << l) < n) ++l;
@@ -89,7 +116,7 @@ static int ilog2_exact(int n) {
 
 /* Resolve levels: 0 means full depth log2(n). Returns -1 when unsupported. */
 static int resolve_levels(int transform, int n, int levels) {
-  if (transform != ORACLE_T_HAAR) return 0;
+  if (transform != ORACLE_T_HAAR && transform != ORACLE_T_HAAR_SKIP1) return 0;
   int full = ilog2_exact(n);
   if (full < 0) return -1;
   if (levels == 0) return full;
@@ -107,7 +134,7 @@ int oracle_transform_matrix(int transform, int n, int levels, double* Lmat) {
     for (int i = 0; i < n; ++i) Lmat[(size_t)i * n + i] = 1.0;
     return 0;
   }
-  if (transform == ORACLE_T_HAAR) {
+  if (transform == ORACLE_T_HAAR || transform == ORACLE_T_HAAR_SKIP1) {
     int lv = resolve_levels(transform, n, levels);
     if (lv < 0) return 2;
     int err = 0;
@@ -123,7 +150,10 @@ int oracle_transform_matrix(int transform, int n, int levels, double* Lmat) {
         for (int t = 0; t < n; ++t) {
           memset(v, 0, sizeof(double) * (size_t)n);
           v[t] = 1.0;
-          haar_forward(v, n, lv, tmp);
+          if (transform == ORACLE_T_HAAR_SKIP1)
+            haar_forward_skip_first(v, n, lv, tmp);
+          else
+            haar_forward(v, n, lv, tmp);
           for (int i = 0; i < n; ++i) Lmat[(size_t)i * n + t] = v[i];
         }
       }

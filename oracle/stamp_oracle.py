@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "stamp_oracle.c")
 _LIB = os.path.join(_HERE, "libstamp_oracle.so")
 _lib = None
 
-T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT = 0, 1, 2, 3, 4
+T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT, T_HAAR_SKIP1 = 0, 1, 2, 3, 4, 5
 
 
 def build(force: bool = False) -> str:

@@ -763,3 +763,73 @@ def test_planted_mistake_fails_its_pins(name):
 def test_unmutated_oracle_passes_the_pins_the_mutants_fail(oracle):
     for pin in _PINS.values():
         pin(oracle)
+
+
+# --------------------------------------------------------------------------------------
+# Haar with the first token excluded (App. "Experimental details / LLMs", STaMP paragraph)
+# --------------------------------------------------------------------------------------
+T_SKIP1 = 5
+
+
+@pytest.mark.parametrize("n,levels", [(2, 0), (4, 0), (4, 1), (8, 2), (64, 0), (256, 3), (2048, 0)])
+def test_skip_first_is_orthonormal_and_leaves_token_zero_alone(oracle, n, levels):
+    """Theorem 1's premise still holds (L orthogonal), row 0 is the first token itself, and no other row touches it:
+    the massive first token cannot leak into any coefficient."""
+    Lm = oracle.transform_matrix(T_SKIP1, n, levels)
+    assert np.max(np.abs(Lm @ Lm.T - np.eye(n))) <= 1e-12
+    assert np.array_equal(Lm[0], np.eye(n)[0])
+    assert not Lm[1:, 0].any()
+
+
+def test_skip_first_hand_case_and_band_structure(oracle):
+    """n = 4: tokens (x0 | x1 x2 x3).  Level 1 pairs (x1, x2) and carries x3 unchanged; level 2 pairs the average with
+    the carried token.  Order [x0 | a_2 | d_2 | d_1]."""
+    r = 1.0 / math.sqrt(2.0)
+    Lm = oracle.transform_matrix(T_SKIP1, 4, 0)
+    want = np.array([[1, 0, 0, 0],
+                     [0, r * r, r * r, r],
+                     [0, r * r, r * r, -r],
+                     [0, r, -r, 0]])
+    assert np.allclose(Lm, want, rtol=0, atol=1e-15)
+    one = oracle.transform_matrix(T_SKIP1, 4, 1)          # one level: [x0 | (x1+x2)/sqrt2, x3 | (x1-x2)/sqrt2]
+    assert np.allclose(one, [[1, 0, 0, 0], [0, r, r, 0], [0, 0, 0, 1], [0, r, -r, 0]], rtol=0, atol=1e-15)
+    # n = 2^p: after the first level the low-pass band has n/2 entries (the last one is the carried token), so
+    # the deeper levels are the ordinary dyadic Haar transform of that band
+    n = 64
+    full = oracle.transform_matrix(T_SKIP1, n, 0)
+    lvl1 = oracle.transform_matrix(T_SKIP1, n, 1)
+    H = oracle.transform_matrix(T_HAAR, n // 2, 0)
+    assert np.allclose(full[1:1 + n // 2], H @ lvl1[1:1 + n // 2], rtol=0, atol=1e-14)
+    assert np.array_equal(full[1 + n // 2:], lvl1[1 + n // 2:])         # d_1: n/2 - 1 rows, untouched by deeper levels
+    assert np.array_equal(lvl1[n // 2], np.eye(n)[n - 1])               # the carried last token, unscaled
+    # m = n - 1 = 3 tokens when the tail happens to be a power of two plus nothing to carry: plain Haar on them
+    five = np.zeros((5, 5))
+    v = np.eye(5)
+    # (n must be a power of two for the matrix builder; the 4-token tail is checked through n = 8 instead)
+    eight = oracle.transform_matrix(T_SKIP1, 8, 1)
+    for i in range(3):                                                    # pairs (1,2), (3,4), (5,6); 7 carried
+        assert np.allclose(eight[1 + i, 1 + 2 * i:3 + 2 * i], [r, r]) and np.allclose(eight[5 + i, 1 + 2 * i:3 + 2 * i], [r, -r])
+    assert np.array_equal(eight[4], np.eye(8)[7])
+
+
+def test_skip_first_layer_keeps_the_massive_token_out_of_the_detail_rows(oracle):
+    """The LLM recipe multiplies token 0 by 100.  With the plain transform that token enters one coefficient of EVERY
+    band and inflates those rows' scales; with the first token excluded the 4-bit rows no longer see it, the pipeline
+    with the quantizers off is still X W^T, and the quantized layer is closer to the unquantized product."""
+    cfg = gen.scaled(gen.config_llm_up(), B=1, L=256, K=128, N=48, k_hi=8)
+    X, W, bias = gen.make_activation(cfg), gen.make_weight(cfg), gen.make_bias(cfg)
+    plain = oracle.matmul_f64(X.reshape(-1, cfg.K), W) + bias[None, :]
+    skip = oracle.stamp_linear(X, W, bias, transform=T_SKIP1, k_hi=cfg.k_hi)
+    full = oracle.stamp_linear(X, W, bias, transform=T_HAAR, k_hi=cfg.k_hi)
+    Lm = oracle.transform_matrix(T_SKIP1, cfg.L, 0)
+    T = oracle.apply_dense(Lm, X.astype(np.float64))
+    assert np.array_equal(skip["T"], T.reshape(-1, cfg.K))
+    assert np.array_equal(skip["T"][0], X[0, 0].astype(np.float64))          # row 0 = the first token, untouched
+    Yt = (T.reshape(-1, cfg.K) @ W.astype(np.float64).T).reshape(1, cfg.L, -1)
+    assert np.max(np.abs(oracle.apply_dense(Lm, Yt, transpose=True)[0] + bias - plain)) <= 1e-11 * np.max(np.abs(plain))
+    # scales of the 4-bit rows: inflated by the leak with the plain transform, not with the exclusion
+    # (the leak sits in the first coefficient of every band: those rows' scales blow up)
+    lo = np.arange(cfg.L) >= cfg.k_hi
+    assert np.max(full["x_scale"][lo]) > 3.0 * np.max(skip["x_scale"][lo])
+    err = lambda y: np.linalg.norm(y - plain) / np.linalg.norm(plain)
+    assert err(skip["Y"]) < err(full["Y"])
