@@ -36,6 +36,13 @@
  *         LL = (a+b+c+d)/2, LH = (a-b+c-d)/2, HL = (a+b-c-d)/2, HH = (a-b-c+d)/2 and LL recurses;
  *         order [LL_l | LH_l | HL_l | HH_l | LH_(l-1) | ... | HH_1], bands in raster order;
  *         levels = 1..3, 2^levels divides both grid sides.
+ *       Haar with the first token excluded (STAMP_T_HAAR_SKIP1; App. "Experimental details / LLMs", STaMP paragraph:
+ *         the first token of an LLM sequence carries massive outliers, stays at 8 bits and is not transformed):
+ *         row 0 of a block is its token 0 itself; the other n - 1 tokens go through a Haar transform whose first level
+ *         pairs (x1, x2), (x3, x4), ... and carries the last token, which has no partner, into the low-pass band
+ *         unchanged (that band has n / 2 entries, so all deeper levels are ordinary dyadic steps; the paper gives no
+ *         rule for the odd length, this is the reading taken).  Order [x0 | a_l | d_l | ... | d_2 | d_1 (n/2 - 1 rows)],
+ *         levels = 1..log2(n) (0 => log2 n).  Runs as separate transform, quantize, GEMM and inverse kernels.
  *     The 8-bit tokens are the rows {i : i mod n < k_hi}: the two-level allocation at the end of
  *     Sec. "Optimal bit allocation" (k_hi leading transformed tokens at bits_hi, the rest at bits_lo).
  *   - Quantizer (Sec. 2.1, first equation, symmetric form): scale = absmax / qmax,
@@ -64,7 +71,8 @@ typedef enum {
 
 typedef enum { STAMP_F32 = 0, STAMP_BF16 = 1 } stamp_dtype;
 
-typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2, STAMP_T_HAAR2D = 3, STAMP_T_WHT = 4 } stamp_transform;
+typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2, STAMP_T_HAAR2D = 3, STAMP_T_WHT = 4,
+               STAMP_T_HAAR_SKIP1 = 5 } stamp_transform;
 
 typedef enum { STAMP_G_PER_TOKEN = 0, STAMP_G_PER_CHANNEL = 1 } stamp_granularity;
 

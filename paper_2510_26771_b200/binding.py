@@ -14,7 +14,7 @@ from .build import LIB_PATH
 
 STAMP_OK = 0
 F32, BF16 = 0, 1
-T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT = 0, 1, 2, 3, 4
+T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT, T_HAAR_SKIP1 = 0, 1, 2, 3, 4, 5
 G_PER_TOKEN, G_PER_CHANNEL = 0, 1
 W_PACKED4, W_INT8 = 0, 1
 

@@ -90,11 +90,14 @@ __global__ void __launch_bounds__(128) k_haar_fwd_pass(const TIn* __restrict__ i
 //                                  first pass (the approximation rows of Yt are read instead)
 //   out   jlo > 0 : [nseq, n >> jlo, N] float partial sums for the next pass
 //         jlo == 0: Y [nseq * n, N] TOut, bias added
+// norm_off: a level-j coefficient carries 2^(-(j + norm_off)/2) (-1 when the rows belong to a transform that sits one
+// level above the table's row order: the dyadic part of the first-token-excluded Haar transform).
 // ------------------------------------------------------------------------------------------
 template <int P, typename TOut>
 __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__ Yt, const float* __restrict__ ain,
                                                        int n, int jlo, long ngroups, int N,
-                                                       const float* __restrict__ bias, void* __restrict__ out_) {
+                                                       const float* __restrict__ bias, void* __restrict__ out_,
+                                                       int norm_off) {
   constexpr int G = 1 << P;
   ptx::grid_dependency_wait();
   const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
@@ -118,7 +121,7 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
       v0[0] = a.x;
       v1[0] = a.y;
     } else {
-      const HaarNorm nrm = haar_norm(jlo + P);
+      const HaarNorm nrm = haar_norm(jlo + P + norm_off);
       const float2 a = load2(Yseq + (long)g * N);
       v0[0] = mul_norm(a.x, nrm);
       v1[0] = mul_norm(a.y, nrm);
@@ -127,7 +130,7 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
     for (int l = P; l >= 1; --l) {
       const int span = 1 << l;               // tokens covered by one level-l coefficient
       const int j = jlo + l;
-      const HaarNorm nrm = haar_norm(j);
+      const HaarNorm nrm = haar_norm(j + norm_off);
       const int row0 = (n >> j) + g * (G >> l);
 #pragma unroll
       for (int i = 0; i < G; i += span) {
@@ -148,6 +151,85 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
       float* dst = static_cast<float*>(out_) + ((s * (long)(n >> jlo) + (long)g * G) * N + c);
 #pragma unroll
       for (int t = 0; t < G; ++t) store2(dst + (long)t * N, v0[t], v1[t]);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Haar transform that leaves the first token of every block alone (App. "Experimental details / LLMs": the first
+// token of an LLM sequence holds massive outliers, stays at 8 bits and is not transformed).  The n - 1 tokens that
+// remain are an odd number: the first level pairs (x1, x2), (x3, x4), ... and carries the last token, which has no
+// partner, into the low-pass band unchanged; that band then has n / 2 entries and every deeper level is an ordinary
+// dyadic step.  Row order of a block: [x0 | a_l | d_l | ... | d_2 | d_1 (n/2 - 1 rows)].
+// First level, forward: writes x0 and the d_1 rows to T (with their maxima), the low-pass band to a1 [nseq, n/2, K]
+// (or, when the transform has one level only, to its rows of T).  One thread per channel pair and token pair.
+// ------------------------------------------------------------------------------------------
+template <typename TIn>
+__global__ void __launch_bounds__(128) k_skip1_fwd_level1(const TIn* __restrict__ X, int n, long npairs, int K,
+                                                          float* __restrict__ T, float* __restrict__ a1, int one_level,
+                                                          unsigned* __restrict__ rowmax) {
+  const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
+  if (c >= K) return;
+  const int half = n >> 1;
+  const HaarNorm nrm = haar_norm(1);
+  for (long pr = blockIdx.y; pr < npairs; pr += gridDim.y) {
+    const long s = pr / half;
+    const int i = static_cast<int>(pr - s * half);
+    const TIn* xb = X + (s * n) * (long)K + c;
+    float* Tb = T + (s * n) * (long)K + c;
+    unsigned* rm = rowmax ? rowmax + s * n : nullptr;
+    auto put = [&](int row, float v0, float v1) {
+      store2(Tb + (long)row * K, v0, v1);
+      if (rm) {
+        const unsigned m = __reduce_max_sync(0xffffffffu, max(absbits(v0), absbits(v1)));
+        if ((threadIdx.x & 31) == 0) atomicMax(rm + row, m);
+      }
+    };
+    float lo0, lo1;
+    if (i < half - 1) {
+      const float2 p = load2(xb + (long)(1 + 2 * i) * K), q = load2(xb + (long)(2 + 2 * i) * K);
+      lo0 = mul_norm(p.x + q.x, nrm);
+      lo1 = mul_norm(p.y + q.y, nrm);
+      put(1 + half + i, mul_norm(p.x - q.x, nrm), mul_norm(p.y - q.y, nrm));
+    } else {
+      const float2 p = load2(xb + (long)(n - 1) * K);   // no partner: carried as it is
+      lo0 = p.x;
+      lo1 = p.y;
+      const float2 z = load2(xb);                        // and the excluded first token
+      put(0, z.x, z.y);
+    }
+    if (one_level)
+      put(1 + i, lo0, lo1);
+    else
+      store2(a1 + (s * half + i) * (long)K + c, lo0, lo1);
+  }
+}
+
+// First level, inverse: Y[x0] = Yt row 0; (x_{2i+1}, x_{2i+2}) = (a1[i] +- d_1[i]) / sqrt 2; x_{n-1} = a1[n/2 - 1]; bias added.
+// a1 [nseq, n/2, N] is the low-pass band rebuilt by the dyadic passes (or, for a one-level transform, rows 1.. of Yt).
+template <typename TOut>
+__global__ void __launch_bounds__(128) k_skip1_inv_level1(const float* __restrict__ Yt, const float* __restrict__ a1, int n,
+                                                          long npairs, int N, const float* __restrict__ bias,
+                                                          TOut* __restrict__ Y) {
+  const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
+  if (c >= N) return;
+  const int half = n >> 1;
+  const HaarNorm nrm = haar_norm(1);
+  const float b0 = bias ? bias[c] : 0.f, b1 = bias ? bias[c + 1] : 0.f;
+  for (long pr = blockIdx.y; pr < npairs; pr += gridDim.y) {
+    const long s = pr / half;
+    const int i = static_cast<int>(pr - s * half);
+    const float* yb = Yt + (s * n) * (long)N + c;
+    TOut* ob = Y + (s * n) * (long)N + c;
+    const float2 a = a1 ? load2(a1 + (s * half + i) * (long)N + c) : load2(yb + (long)(1 + i) * N);
+    if (i < half - 1) {
+      const float2 d = load2(yb + (long)(1 + half + i) * N);
+      store2(ob + (long)(1 + 2 * i) * N, mul_norm(a.x + d.x, nrm) + b0, mul_norm(a.y + d.y, nrm) + b1);
+      store2(ob + (long)(2 + 2 * i) * N, mul_norm(a.x - d.x, nrm) + b0, mul_norm(a.y - d.y, nrm) + b1);
+    } else {
+      store2(ob + (long)(n - 1) * N, a.x + b0, a.y + b1);
+      const float2 z = load2(yb);
+      store2(ob, z.x + b0, z.y + b1);
     }
   }
 }

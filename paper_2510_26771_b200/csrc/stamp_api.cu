@@ -44,7 +44,7 @@ static inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool need_n, Problem* out) {
   if (!cfg || !out) return STAMP_ERR_INVALID_ARG;
   if (B <= 0 || L <= 0 || K <= 0 || (need_n && N <= 0)) return STAMP_ERR_INVALID_ARG;
-  if (cfg->transform < STAMP_T_IDENTITY || cfg->transform > STAMP_T_WHT) return STAMP_ERR_INVALID_ARG;
+  if (cfg->transform < STAMP_T_IDENTITY || cfg->transform > STAMP_T_HAAR_SKIP1) return STAMP_ERR_INVALID_ARG;
   if (cfg->block < 0 || cfg->levels < 0 || cfg->k_hi < 0 || cfg->grid_w < 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->transform != STAMP_T_HAAR2D && cfg->grid_w != 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->bits_hi != 8 || cfg->bits_lo != 4 || cfg->bits_w != 4) return STAMP_ERR_UNSUPPORTED;
@@ -57,7 +57,8 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
   if (need_n && N % 8 != 0) return STAMP_ERR_UNSUPPORTED;
   if ((long)B * L > (1L << 30)) return STAMP_ERR_UNSUPPORTED;
   int levels = 0;
-  if (cfg->transform == STAMP_T_HAAR) {
+  if (cfg->transform == STAMP_T_HAAR || cfg->transform == STAMP_T_HAAR_SKIP1) {
+    if (cfg->transform == STAMP_T_HAAR_SKIP1 && n < 2) return STAMP_ERR_UNSUPPORTED;
     const int full = ilog2(n);
     levels = cfg->levels ? cfg->levels : full;
     if (levels > full) return STAMP_ERR_UNSUPPORTED;
@@ -118,7 +119,7 @@ static PassPlan make_plan(int levels) {
 // Workspace layout (one layout for all calls of a problem size).
 // ------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t rowmax, htc_cnt, xscale, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, dctsplit, xzero, wsum, total;
+  size_t rowmax, htc_cnt, xscale, skipa, T, ping, pong, atop, top_ping, top_pong, dctmat, a8, w8, yt, a8top, sxtop, yttop, a8v, dctsplit, xzero, wsum, total;
 };
 static Workspace layout(const Problem& pb) {
   Workspace w{};
@@ -132,6 +133,8 @@ static Workspace layout(const Problem& pb) {
   // (directly behind the row maxima: one memset clears both before the tensor-core transform+quantize launch)
   w.htc_cnt = off; off += align256((M >> 7) * 4 + 4);
   w.xscale = off; off += align256(M * 4);
+  // low-pass band after the first level of the first-token-excluded Haar transform (forward: K wide, inverse: N wide)
+  w.skipa = off;  off += align256(pb.transform == STAMP_T_HAAR_SKIP1 ? (M / 2) * KN * 4 : 0);
   w.T = off;      off += align256(M * (size_t)pb.K * 4);
   w.ping = off;   off += align256(ping_rows * KN * 4);
   w.pong = off;   off += align256(pong_rows * KN * 4);
@@ -505,7 +508,25 @@ static int launch_haar2d_inv(const Problem& pb, const float* Yt, const float* bi
 }
 
 static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, float* T, unsigned* rowmax,
-                                 float* ping, float* pong, float* mat, cudaStream_t st) {
+                                 float* ping, float* pong, float* mat, cudaStream_t st, float* skipa = nullptr) {
+  if (pb.transform == STAMP_T_HAAR_SKIP1) {
+    // first level (pairs from token 1 on, last token carried, token 0 copied), then the dyadic levels on the
+    // low-pass band, whose rows sit one below their place in a plain Haar block
+    if (!skipa) return STAMP_ERR_INVALID_ARG;
+    if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
+    const long npairs = pb.M / 2;
+    dim3 grid((pb.K / 2 + 127) / 128, (unsigned)(npairs < 32768 ? npairs : 32768));
+    const int one = pb.levels == 1;
+    if (x_dtype == STAMP_BF16)
+      k_skip1_fwd_level1<__nv_bfloat16><<<grid, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(X), pb.n, npairs, pb.K, T, skipa,
+                                                              one, rowmax);
+    else
+      k_skip1_fwd_level1<float><<<grid, 128, 0, st>>>(static_cast<const float*>(X), pb.n, npairs, pb.K, T, skipa, one, rowmax);
+    STAMP_CHECK_LAUNCH();
+    if (one) return STAMP_OK;
+    return run_haar_passes(skipa, false, pb.nseq, pb.n / 2, pb.K, pb.levels - 1, T + pb.K, pb.n, 1, -1,
+                           rowmax ? rowmax + 1 : nullptr, 0, ping, pong, st);
+  }
   if (pb.transform == STAMP_T_HAAR2D) {
     if (rowmax && cudaMemsetAsync(rowmax, 0, (size_t)pb.M * 4, st) != cudaSuccess) return STAMP_ERR_CUDA;
     const bool bf = x_dtype == STAMP_BF16;
@@ -536,15 +557,15 @@ static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, 
 
 template <typename TOut>
 static int launch_inv_pass(int P, const float* Yt, const float* ain, int n, int jlo, long ngroups, int N,
-                           const float* bias, void* out, cudaStream_t st) {
+                           const float* bias, void* out, cudaStream_t st, int norm_off = 0) {
   dim3 grid((N / 2 + 127) / 128, (unsigned)(ngroups < 32768 ? ngroups : 32768));
   switch (P) {
-    case 0: launch_pdl(k_haar_inv_pass<0, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 1: launch_pdl(k_haar_inv_pass<1, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 2: launch_pdl(k_haar_inv_pass<2, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 3: launch_pdl(k_haar_inv_pass<3, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    case 4: launch_pdl(k_haar_inv_pass<4, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
-    default: launch_pdl(k_haar_inv_pass<5, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out); break;
+    case 0: launch_pdl(k_haar_inv_pass<0, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out, norm_off); break;
+    case 1: launch_pdl(k_haar_inv_pass<1, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out, norm_off); break;
+    case 2: launch_pdl(k_haar_inv_pass<2, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out, norm_off); break;
+    case 3: launch_pdl(k_haar_inv_pass<3, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out, norm_off); break;
+    case 4: launch_pdl(k_haar_inv_pass<4, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out, norm_off); break;
+    default: launch_pdl(k_haar_inv_pass<5, TOut>, grid, dim3(128), 0, st, Yt, ain, n, jlo, ngroups, N, bias, out, norm_off); break;
   }
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
@@ -552,7 +573,38 @@ static int launch_inv_pass(int P, const float* Yt, const float* ain, int n, int 
 
 // Y = L^T Yt + bias (Haar or identity), coarse passes first.
 static int run_inverse_generic(const Problem& pb, const float* Yt, const float* bias, void* Y, int y_dtype,
-                               float* ping, float* pong, float* mat, cudaStream_t st) {
+                               float* ping, float* pong, float* mat, cudaStream_t st, float* skipa = nullptr) {
+  if (pb.transform == STAMP_T_HAAR_SKIP1) {
+    if (!skipa) return STAMP_ERR_INVALID_ARG;
+    const float* a1 = nullptr;
+    if (pb.levels > 1) {   // dyadic levels l..2, coarse to fine, down to the low-pass band of level 1
+      const PassPlan pl = make_plan(pb.levels - 1);
+      int jlo_of[8];
+      int acc = 1;
+      for (int i = 0; i < pl.npass; ++i) {
+        jlo_of[i] = acc;
+        acc += pl.p[i];
+      }
+      const float* ain = nullptr;
+      float* bufs[2] = {ping, pong};
+      for (int i = pl.npass - 1; i >= 0; --i) {
+        const int P = pl.p[i], jlo = jlo_of[i];
+        const long ngroups = (long)pb.nseq * (pb.n >> (jlo + P));
+        float* aout = i == 0 ? skipa : bufs[(i - 1) & 1];
+        if (int rc = launch_inv_pass<float>(P, Yt + pb.N, ain, pb.n, jlo, ngroups, pb.N, nullptr, aout, st, -1)) return rc;
+        ain = aout;
+      }
+      a1 = skipa;
+    }
+    const long npairs = pb.M / 2;
+    dim3 grid((pb.N / 2 + 127) / 128, (unsigned)(npairs < 32768 ? npairs : 32768));
+    if (y_dtype == STAMP_BF16)
+      k_skip1_inv_level1<__nv_bfloat16><<<grid, 128, 0, st>>>(Yt, a1, pb.n, npairs, pb.N, bias, static_cast<__nv_bfloat16*>(Y));
+    else
+      k_skip1_inv_level1<float><<<grid, 128, 0, st>>>(Yt, a1, pb.n, npairs, pb.N, bias, static_cast<float*>(Y));
+    STAMP_CHECK_LAUNCH();
+    return STAMP_OK;
+  }
   if (pb.transform == STAMP_T_HAAR2D) {
     const bool bf = y_dtype == STAMP_BF16;
     __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(Y);
@@ -1147,7 +1199,7 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
   unsigned* rowmax = reinterpret_cast<unsigned*>(base + w.rowmax);
   if (pb.act_zp) {
     rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
-                               reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st);
+                               reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st, reinterpret_cast<float*>(base + w.skipa));
     if (rc) return rc;
     return run_quant_rows_zp(pb, T, nullptr, q_hi, q_lo, x_scale, reinterpret_cast<int*>(x_scale + pb.M), st);
   }
@@ -1163,7 +1215,7 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
     return STAMP_OK;
   }
   rc = run_transform_generic(pb, X, x_dtype, T, rowmax, reinterpret_cast<float*>(base + w.ping),
-                             reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st);
+                             reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st, reinterpret_cast<float*>(base + w.skipa));
   if (rc) return rc;
   return run_quant_rows(pb, T, rowmax, pb.n, nullptr, q_hi, q_lo, x_scale, st);
 }
@@ -1207,7 +1259,7 @@ int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, i
   uint8_t* base = static_cast<uint8_t*>(ws);
   return run_inverse_generic(pb, Yt, bias, Y, y_dtype, reinterpret_cast<float*>(base + wl.ping),
                              reinterpret_cast<float*>(base + wl.pong), reinterpret_cast<float*>(base + wl.dctmat),
-                             static_cast<cudaStream_t>(stream));
+                             static_cast<cudaStream_t>(stream), reinterpret_cast<float*>(base + wl.skipa));
 }
 
 int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
@@ -1217,6 +1269,7 @@ int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float*
   int rc = resolve(cfg, B, L, 128, N, true, &pb);
   if (rc) return rc;
   if (!Yt || !Y || !dtype_ok(y_dtype)) return STAMP_ERR_INVALID_ARG;
+  if (pb.transform == STAMP_T_HAAR_SKIP1) return STAMP_ERR_UNSUPPORTED;   // (its low-pass band would need half of Yt again)
   // partial sums between the coarse-to-fine passes: the only scratch the inverse needs
   const PassPlan pl = make_plan(pb.levels);
   const size_t ping_bytes = pl.npass > 1 ? align256(((size_t)pb.M >> pl.p[0]) * pb.N * 4) : 0;
@@ -1270,7 +1323,7 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     // zero-point codes: transform, min-max quantizer, GEMM with the zero-point term in its epilogue, inverse
     int* x_zero = reinterpret_cast<int*>(base + wl.xzero);
     int* w_sum = reinterpret_cast<int*>(base + wl.wsum);
-    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
+    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st, reinterpret_cast<float*>(base + wl.skipa))))
       return rc;
     const int8_t* w8z = nullptr;
     if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8z, st))) return rc;
@@ -1278,7 +1331,7 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     if ((rc = launch_gemm(a8, w8z, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_ZP_F32, st, nullptr, nullptr, 0, x_zero,
                           w_sum)))
       return rc;
-    return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
+    return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st, reinterpret_cast<float*>(base + wl.skipa));
   }
   if (route == ROUTE_TILED) {
     // Fused route: the transform+quantize kernel writes the token operand in tile order, the GEMM's
@@ -1324,19 +1377,19 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
       return run_inverse_dct_tc(pb, reinterpret_cast<const __nv_bfloat16*>(yt), bias, Y, y_dtype, base, wl, st);
     }
     if ((rc = launch_gemm(a8, w8d, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_F32, st))) return rc;
-    return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
+    return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st, reinterpret_cast<float*>(base + wl.skipa));
   }
   if (have_cq) {
     if ((rc = run_quantize_haar(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;
   } else {
-    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st)))
+    if ((rc = run_transform_generic(pb, X, x_dtype, T, rowmax, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st, reinterpret_cast<float*>(base + wl.skipa))))
       return rc;
     if ((rc = run_quant_rows(pb, T, rowmax, pb.n, a8, nullptr, nullptr, x_scale, st))) return rc;
   }
   const int8_t* w8 = nullptr;
   if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
   if ((rc = launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_F32, st))) return rc;
-  return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st);
+  return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st, reinterpret_cast<float*>(base + wl.skipa));
 }
 
 static size_t dtype_size(int d) { return d == STAMP_BF16 ? 2 : 4; }
@@ -1391,7 +1444,7 @@ int stamp_debug_transform(const stamp_config* cfg, const void* X, int x_dtype, i
                              base, wl, static_cast<cudaStream_t>(stream));
   return run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + wl.ping),
                                reinterpret_cast<float*>(base + wl.pong), reinterpret_cast<float*>(base + wl.dctmat),
-                               static_cast<cudaStream_t>(stream));
+                               static_cast<cudaStream_t>(stream), reinterpret_cast<float*>(base + wl.skipa));
 }
 
 int stamp_debug_unpack_codes(const stamp_config* cfg, const void* q_hi, const void* q_lo, int B, int L, int K,

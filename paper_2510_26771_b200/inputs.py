@@ -21,7 +21,7 @@ import numpy as np
 from scipy.signal import lfilter
 
 # transform identifiers (values match the public C header's stamp_transform)
-T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT = 0, 1, 2, 3, 4
+T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT, T_HAAR_SKIP1 = 0, 1, 2, 3, 4, 5
 # storage dtypes (values match stamp_dtype)
 F32, BF16 = 0, 1
 
@@ -200,6 +200,12 @@ def config_llm_up_zp() -> LayerConfig:
     return dataclasses.replace(config_llm_up(), name="llm_mlp_up_zp", zero_point=True)
 
 
+def config_llm_up_skip1() -> LayerConfig:
+    """The MLP up-projection workload as the paper runs LLMs: the massive first token is left out of the sequence
+    transform (and is one of the 8-bit rows)."""
+    return dataclasses.replace(config_llm_up(), name="llm_mlp_up_skip1", transform=T_HAAR_SKIP1)
+
+
 def config_dit_proj_2d() -> LayerConfig:
     """The DiT projection with the paper's own LVM transform: 3-level 2-D Haar over the 64 x 64 patch grid,
     whose 64 low-pass tokens are the 8-bit ones."""
@@ -231,7 +237,7 @@ def config_sweep(L: int, D: int, levels: int = 0) -> LayerConfig:
 
 def named_configs() -> dict:
     return {c.name: c for c in (config_tiny(), config_llm_up(), config_dit_proj(), config_llm_down(), config_dit_proj_2d(), config_llm_down_wht(),
-                                config_llm_up_zp(), config_dit_proj_2d_zp())}
+                                config_llm_up_zp(), config_dit_proj_2d_zp(), config_llm_up_skip1())}
 
 
 def scaled(cfg: LayerConfig, **kw) -> LayerConfig:

@@ -39,6 +39,7 @@ FULL = {
     "dit_attn_proj_2d": gen.config_dit_proj_2d(),
     "llm_down_proj_wht": gen.config_llm_down_wht(),
     "llm_mlp_up_zp": gen.config_llm_up_zp(),
+    "llm_mlp_up_skip1": gen.config_llm_up_skip1(),
     "dit_attn_proj_2d_zp": gen.config_dit_proj_2d_zp(),
 }
 # the throughput sweep: all twelve shapes
@@ -121,7 +122,9 @@ def test_full_size_parity(oracle, name):
     del Y
     err = H.rel_fro(Y_s, ref["Y"])
     print(f"[{name}] output relative Frobenius error {err:.2e} on {ncols} sampled channels")
-    assert err <= _fused_y_tol(cfg)
+    # (the tight bound presumes the oracle's codes; a code that sat on a rounding boundary and fell the other way --
+    #  allowed up to 1e-5 of them -- moves the output by a code step of its row, far more than fp32 rounding)
+    assert err <= (_fused_y_tol(cfg) if bad == 0 else Y_TOL)
     Yb = st.stamp_linear_fused(c, Xd, w8, st.W_INT8, w_scale, bd, ws, out_dtype=torch.bfloat16)
     Yb_s = Yb.reshape(M, N)[:, cols_d].float().cpu().numpy()
     # bf16 output: the fp32 result rounded once (2^-9 relative) on top of the fp32 path's own error

@@ -130,6 +130,11 @@ CASES = {
                                   dtype=gen.F32, recipe="ar1"),
     # a patch (64 tokens x 2048 channels) that does not fit in shared memory: row maxima and codes in separate launches
     "haar2d_wide_k": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=2048, N=64, grid=16, levels=3, k_hi=4),
+    # Haar with the first token excluded (the LLM setting): full depth with ragged tiles, one level, fp32 blocks
+    "skip_first": gen.scaled(gen.config_llm_up_skip1(), B=2, L=512, K=384, N=392, k_hi=16),
+    "skip_first_one_level": gen.scaled(gen.config_llm_up_skip1(), B=1, L=256, K=128, N=64, levels=1, k_hi=130),
+    "skip_first_fp32_blocks": gen.scaled(gen.config_tiny(), B=2, L=256, K=128, N=72, block=64, levels=3, k_hi=8,
+                                         transform=gen.T_HAAR_SKIP1),
     # two levels only: no cluster tree, approximation rows quantized by the same kernel
     "two_levels": gen.scaled(gen.config_dit_proj(), B=2, L=256, K=1152, N=128, grid=16, levels=2, k_hi=64),
 }
@@ -165,6 +170,7 @@ def test_stagewise_parity(st, oracle, name):
     bad, worst = H.code_mismatch(codes, ref["q"])
     print(f"[{name}] activation code mismatches: {bad} of {codes.size} (max |diff| {worst})")
     assert worst <= 1 and bad <= _allowed(codes.size), (bad, worst, codes.size)
+    act_bad = bad
 
     # a4: weights
     wq, wsc = st.stamp_quantize_weights(c, Wd)
@@ -208,7 +214,9 @@ def test_stagewise_parity(st, oracle, name):
         Y3 = st.stamp_linear_fused(c, Xd, wbuf, wfmt, wsc, bd, ws).cpu().numpy().reshape(-1, N)
         err = H.rel_fro(Y3, ref["Y"])
         print(f"[{name}] one-call layer, output relative Frobenius error {err:.2e}")
-        assert err <= _fused_y_tol(cfg)
+        # (the tight bound presumes the oracle's codes; a code on a rounding boundary that fell the other way moves
+        #  the output by a whole code step of its row)
+        assert err <= (_fused_y_tol(cfg) if act_bad == 0 else Y_TOL)
     assert st.stamp_last_launch_count() > 0
     # the operand of the one-call layer's GEMM, code by code (routes that reorder it)
     mapped = check_fused_operand(st, c, cfg, Xd, ws, ref["q"], ref["x_scale"], label=name)
@@ -223,6 +231,7 @@ ZP_CASES = {
     "zp_dct": gen.scaled(gen.config_llm_down(), B=1, L=512, K=256, N=136),
     "zp_wht": gen.scaled(gen.config_llm_down_wht(), B=1, L=256, K=128, N=64, block=64, k_hi=4),
     "zp_haar2d": gen.scaled(gen.config_dit_proj_2d(), B=1, L=1024, K=256, N=128, grid=32, levels=3, k_hi=16),
+    "zp_skip_first": gen.scaled(gen.config_llm_up_skip1(), B=1, L=256, K=128, N=72, k_hi=8),
     "zp_identity": gen.scaled(gen.config_sweep(512, 2048), L=256, K=256, N=128, transform=gen.T_IDENTITY, k_hi=8),
 }
 
