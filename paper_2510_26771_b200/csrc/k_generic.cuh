@@ -163,6 +163,8 @@ __global__ void __launch_bounds__(128) k_haar_inv_pass(const float* __restrict__
 // dyadic step.  Row order of a block: [x0 | a_l | d_l | ... | d_2 | d_1 (n/2 - 1 rows)].
 // First level, forward: writes x0 and the d_1 rows to T (with their maxima), the low-pass band to a1 [nseq, n/2, K]
 // (or, when the transform has one level only, to its rows of T).  One thread per channel pair and token pair.
+// a1 holds UN-NORMALISED sums x_{2i+1} + x_{2i+2}, as the deeper passes expect of their input (every coefficient
+// is then rounded once, when it is written); the carried token enters that band as x * sqrt 2.
 // ------------------------------------------------------------------------------------------
 template <typename TIn>
 __global__ void __launch_bounds__(128) k_skip1_fwd_level1(const TIn* __restrict__ X, int n, long npairs, int K,
@@ -185,16 +187,21 @@ __global__ void __launch_bounds__(128) k_skip1_fwd_level1(const TIn* __restrict_
         if ((threadIdx.x & 31) == 0) atomicMax(rm + row, m);
       }
     };
-    float lo0, lo1;
+    constexpr float SQRT2_HI = 1.41421354f, SQRT2_LO = 2.4203235e-8f;   // fp32(sqrt 2) and what it leaves out
+    float lo0, lo1;       // low-pass entry: un-normalised (times sqrt 2) unless this is the only level
     if (i < half - 1) {
       const float2 p = load2(xb + (long)(1 + 2 * i) * K), q = load2(xb + (long)(2 + 2 * i) * K);
-      lo0 = mul_norm(p.x + q.x, nrm);
-      lo1 = mul_norm(p.y + q.y, nrm);
+      lo0 = p.x + q.x;
+      lo1 = p.y + q.y;
+      if (one_level) {
+        lo0 = mul_norm(lo0, nrm);
+        lo1 = mul_norm(lo1, nrm);
+      }
       put(1 + half + i, mul_norm(p.x - q.x, nrm), mul_norm(p.y - q.y, nrm));
     } else {
       const float2 p = load2(xb + (long)(n - 1) * K);   // no partner: carried as it is
-      lo0 = p.x;
-      lo1 = p.y;
+      lo0 = one_level ? p.x : fmaf(p.x, SQRT2_HI, p.x * SQRT2_LO);
+      lo1 = one_level ? p.y : fmaf(p.y, SQRT2_HI, p.y * SQRT2_LO);
       const float2 z = load2(xb);                        // and the excluded first token
       put(0, z.x, z.y);
     }
@@ -206,7 +213,8 @@ __global__ void __launch_bounds__(128) k_skip1_fwd_level1(const TIn* __restrict_
 }
 
 // First level, inverse: Y[x0] = Yt row 0; (x_{2i+1}, x_{2i+2}) = (a1[i] +- d_1[i]) / sqrt 2; x_{n-1} = a1[n/2 - 1]; bias added.
-// a1 [nseq, n/2, N] is the low-pass band rebuilt by the dyadic passes (or, for a one-level transform, rows 1.. of Yt).
+// a1 [nseq, n/2, N] is the low-pass band rebuilt by the dyadic passes, as they leave it: a_1 / sqrt 2 (for a one-level
+// transform a1 is null and a_1 itself is read from rows 1.. of Yt).
 template <typename TOut>
 __global__ void __launch_bounds__(128) k_skip1_inv_level1(const float* __restrict__ Yt, const float* __restrict__ a1, int n,
                                                           long npairs, int N, const float* __restrict__ bias,
@@ -221,12 +229,22 @@ __global__ void __launch_bounds__(128) k_skip1_inv_level1(const float* __restric
     const int i = static_cast<int>(pr - s * half);
     const float* yb = Yt + (s * n) * (long)N + c;
     TOut* ob = Y + (s * n) * (long)N + c;
-    const float2 a = a1 ? load2(a1 + (s * half + i) * (long)N + c) : load2(yb + (long)(1 + i) * N);
+    constexpr float SQRT2_HI = 1.41421354f, SQRT2_LO = 2.4203235e-8f;
+    float2 a = a1 ? load2(a1 + (s * half + i) * (long)N + c) : load2(yb + (long)(1 + i) * N);
     if (i < half - 1) {
       const float2 d = load2(yb + (long)(1 + half + i) * N);
-      store2(ob + (long)(1 + 2 * i) * N, mul_norm(a.x + d.x, nrm) + b0, mul_norm(a.y + d.y, nrm) + b1);
-      store2(ob + (long)(2 + 2 * i) * N, mul_norm(a.x - d.x, nrm) + b0, mul_norm(a.y - d.y, nrm) + b1);
+      const float d0 = mul_norm(d.x, nrm), d1 = mul_norm(d.y, nrm);
+      if (!a1) {
+        a.x = mul_norm(a.x, nrm);
+        a.y = mul_norm(a.y, nrm);
+      }
+      store2(ob + (long)(1 + 2 * i) * N, a.x + d0 + b0, a.y + d1 + b1);
+      store2(ob + (long)(2 + 2 * i) * N, a.x - d0 + b0, a.y - d1 + b1);
     } else {
+      if (a1) {   // a_1 / sqrt 2 -> the carried token
+        a.x = fmaf(a.x, SQRT2_HI, a.x * SQRT2_LO);
+        a.y = fmaf(a.y, SQRT2_HI, a.y * SQRT2_LO);
+      }
       store2(ob + (long)(n - 1) * N, a.x + b0, a.y + b1);
       const float2 z = load2(yb);
       store2(ob, z.x + b0, z.y + b1);

@@ -524,7 +524,7 @@ static int run_transform_generic(const Problem& pb, const void* X, int x_dtype, 
       k_skip1_fwd_level1<float><<<grid, 128, 0, st>>>(static_cast<const float*>(X), pb.n, npairs, pb.K, T, skipa, one, rowmax);
     STAMP_CHECK_LAUNCH();
     if (one) return STAMP_OK;
-    return run_haar_passes(skipa, false, pb.nseq, pb.n / 2, pb.K, pb.levels - 1, T + pb.K, pb.n, 1, -1,
+    return run_haar_passes(skipa, false, pb.nseq, pb.n / 2, pb.K, pb.levels - 1, T + pb.K, pb.n, 1, 0,
                            rowmax ? rowmax + 1 : nullptr, 0, ping, pong, st);
   }
   if (pb.transform == STAMP_T_HAAR2D) {
@@ -591,7 +591,7 @@ static int run_inverse_generic(const Problem& pb, const float* Yt, const float* 
         const int P = pl.p[i], jlo = jlo_of[i];
         const long ngroups = (long)pb.nseq * (pb.n >> (jlo + P));
         float* aout = i == 0 ? skipa : bufs[(i - 1) & 1];
-        if (int rc = launch_inv_pass<float>(P, Yt + pb.N, ain, pb.n, jlo, ngroups, pb.N, nullptr, aout, st, -1)) return rc;
+        if (int rc = launch_inv_pass<float>(P, Yt + pb.N, ain, pb.n, jlo, ngroups, pb.N, nullptr, aout, st)) return rc;
         ain = aout;
       }
       a1 = skipa;
