@@ -562,6 +562,80 @@ int oracle_quantize_rows_f32in(const float* W, long rows, int K, int bits, float
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Per-block ("group") scales along the feature axis (the LVM table's setting: W4A4 per-block quantization with
+ * block size 64; App. "Experimental details / LVMs": per-block weight and activation quantization as in SVDQuant).
+ * Every run of `group` consecutive features of a row has a scale of its own,
+ *   s[r][g] = (float)max_{k in g}|t[r][k]| / (float)qmax   (1 for an all-zero group),
+ *   q[r][k] = clamp(rne((float)t[r][k] / s[r][k / group]), -qmax, qmax),
+ * the symmetric quantizer of oracle_quantize_rows applied group by group (same fp32 rounding decision).  The
+ * paper names the scheme and the block size, not its formulas: symmetric codes and absmax range are the
+ * reading shared with the per-token quantizer.  K must be a multiple of group.  scale is [rows][K / group].
+ * ------------------------------------------------------------------------------------------ */
+int oracle_quantize_rows_grouped(const double* T, long rows, int K, const int32_t* bits_per_row, int period, int group,
+                                 float* scale, int8_t* codes) {
+  if (period <= 0 || group <= 0 || K % group) return 1;
+  int ng = K / group;
+#pragma omp parallel for schedule(static)
+  for (long r = 0; r < rows; ++r) {
+    const double* t = T + (size_t)r * K;
+    int bits = bits_per_row[r % period];
+    float qmaxf = (float)((1 << (bits - 1)) - 1);
+    for (int g = 0; g < ng; ++g) {
+      double amax = 0.0;
+      for (int j = g * group; j < (g + 1) * group; ++j) {
+        double a = fabs(t[j]);
+        if (a > amax) amax = a;
+      }
+      float s = (amax > 0.0) ? ((float)amax / qmaxf) : 1.0f;
+      if (!(s > 0.0f)) s = 1.0f;
+      scale[(size_t)r * ng + g] = s;
+      for (int j = g * group; j < (g + 1) * group; ++j) {
+        float q = rintf((float)t[j] / s);
+        if (q > qmaxf) q = qmaxf;
+        if (q < -qmaxf) q = -qmaxf;
+        codes[(size_t)r * K + j] = (int8_t)q;
+      }
+    }
+  }
+  return 0;
+}
+
+int oracle_quantize_rows_grouped_f32in(const float* W, long rows, int K, int bits, int group, float* scale, int8_t* codes) {
+  if (group <= 0 || K % group) return 1;
+  double* t = (double*)malloc(sizeof(double) * (size_t)rows * K);
+  if (!t) return 3;
+  for (size_t i = 0; i < (size_t)rows * K; ++i) t[i] = (double)W[i];
+  int32_t b = bits;
+  int rc = oracle_quantize_rows_grouped(t, rows, K, &b, 1, group, scale, codes);
+  free(t);
+  return rc;
+}
+
+/* Product of two group-scaled operands, de-quantized (Sec. 2.1: (x_int - z) s with z = 0, once per group):
+ *   Yt[m][n] = sum_g ( sum_{k in g} q[m][k] wq[n][k] ) * sx[m][g] * sw[n][g]
+ * The inner sums are exact integers (int64, far from overflow for a group); the outer sum runs over the groups
+ * in increasing order in fp64. */
+int oracle_gemm_grouped(const int8_t* q, const float* sx, const int8_t* wq, const float* sw, long M, int N, int K,
+                        int group, double* Yt) {
+  if (group <= 0 || K % group) return 1;
+  int ng = K / group;
+#pragma omp parallel for schedule(static)
+  for (long m = 0; m < M; ++m)
+    for (int n = 0; n < N; ++n) {
+      const int8_t* a = q + (size_t)m * K;
+      const int8_t* b = wq + (size_t)n * K;
+      double y = 0.0;
+      for (int g = 0; g < ng; ++g) {
+        int64_t acc = 0;
+        for (int k = g * group; k < (g + 1) * group; ++k) acc += (int64_t)a[k] * (int64_t)b[k];
+        y += (double)acc * (double)sx[(size_t)m * ng + g] * (double)sw[(size_t)n * ng + g];
+      }
+      Yt[(size_t)m * N + n] = y;
+    }
+  return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Integer matmul (Algorithm line "Y <- X W^T" on the integer codes): naive triple loop,
  * acc[m][n] = sum_k q[m][k] * wq[n][k], accumulated in int64 and checked to fit int32.
  * Returns 5 if any accumulator would overflow int32.
@@ -623,12 +697,15 @@ int oracle_matmul_f64(const float* X, const float* W, long M, int N, int K, doub
  *   Y        [B*L, N]  fp64   final output
  * act_asym != 0 selects the zero-point activation quantizer: q then holds UNSIGNED bytes, x_zero
  * [B*L] receives the zero points (it may be null otherwise) and acc is the sum over (q - z) * wq.
+ * group > 0 selects per-block scales of `group` features for activations AND weights (symmetric codes only):
+ * x_scale is then [B*L][K/group], w_scale [N][K/group], and acc is not produced (the integer partial sums are
+ * scaled group by group).
  * Returns 0 on success.
  * ------------------------------------------------------------------------------------------ */
 int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B, int L, int K, int N,
                         int transform, int block, int levels, int k_hi, int bits_hi, int bits_lo,
                         int bits_w, double* T, float* x_scale, int8_t* q, float* w_scale, int8_t* wq,
-                        int32_t* acc, double* Yt, double* Y, int grid_w, int act_asym, int32_t* x_zero) {
+                        int32_t* acc, double* Yt, double* Y, int grid_w, int act_asym, int32_t* x_zero, int group) {
   int n = block ? block : L;
   if (n <= 0 || L % n) return 1;
   long M = (long)B * L;
@@ -642,10 +719,12 @@ int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B
 #define OWN(ptr, flag, type, count)                                   \
   if (!(ptr)) { ptr = (type*)malloc(sizeof(type) * (size_t)(count)); flag = 1; if (!(ptr)) { rc = 3; goto done; } }
   OWN(T, own_T, double, (size_t)M * K)
-  OWN(x_scale, own_xs, float, M)
+  if (group > 0 && (act_asym || K % group)) return 1;
+  int ng = group > 0 ? K / group : 1;
+  OWN(x_scale, own_xs, float, (size_t)M * ng)
   OWN(q, own_q, int8_t, (size_t)M * K)
   if (act_asym) { OWN(x_zero, own_xz, int32_t, M) }
-  OWN(w_scale, own_ws, float, N)
+  OWN(w_scale, own_ws, float, (size_t)N * ng)
   OWN(wq, own_wq, int8_t, (size_t)N * K)
   OWN(acc, own_acc, int32_t, (size_t)M * N)
   OWN(Yt, own_Yt, double, (size_t)M * N)
@@ -678,20 +757,27 @@ int oracle_stamp_linear(const float* X, const float* W, const float* bias, int B
   if (!bits) { rc = 3; goto done; }
   rc = oracle_bit_map(L, n, k_hi, bits_hi, bits_lo, bits);
   if (rc) goto done;
-  rc = act_asym ? oracle_quantize_rows_asym(T, M, K, bits, L, x_scale, x_zero, (uint8_t*)q)
-                : oracle_quantize_rows(T, M, K, bits, L, x_scale, q);
+  rc = group > 0 ? oracle_quantize_rows_grouped(T, M, K, bits, L, group, x_scale, q)
+       : act_asym ? oracle_quantize_rows_asym(T, M, K, bits, L, x_scale, x_zero, (uint8_t*)q)
+                  : oracle_quantize_rows(T, M, K, bits, L, x_scale, q);
   if (rc) goto done;
 
   /* quantized weights (static; untouched by the sequence transform) */
-  rc = oracle_quantize_rows_f32in(W, N, K, bits_w, w_scale, wq);
+  rc = group > 0 ? oracle_quantize_rows_grouped_f32in(W, N, K, bits_w, group, w_scale, wq)
+                 : oracle_quantize_rows_f32in(W, N, K, bits_w, w_scale, wq);
   if (rc) goto done;
 
   /* Y <- X W^T on the integer codes, then de-quantize */
-  rc = act_asym ? oracle_gemm_zp_i32((const uint8_t*)q, x_zero, wq, M, N, K, acc)
-                : oracle_gemm_i32(q, wq, M, N, K, acc);
-  if (rc) goto done;
-  rc = oracle_dequant(acc, x_scale, w_scale, M, N, Yt);
-  if (rc) goto done;
+  if (group > 0) {
+    rc = oracle_gemm_grouped(q, x_scale, wq, w_scale, M, N, K, group, Yt);
+    if (rc) goto done;
+  } else {
+    rc = act_asym ? oracle_gemm_zp_i32((const uint8_t*)q, x_zero, wq, M, N, K, acc)
+                  : oracle_gemm_i32(q, wq, M, N, K, acc);
+    if (rc) goto done;
+    rc = oracle_dequant(acc, x_scale, w_scale, M, N, Yt);
+    if (rc) goto done;
+  }
 
   /* Y <- L^{-1} Y  (= L^T Y), then Y <- Y + bias */
   if (Y) {

@@ -158,6 +158,42 @@ def quantize_weights(W: np.ndarray, bits: int = 4):
     return codes, scale
 
 
+def quantize_rows_grouped(T: np.ndarray, bits_per_row: np.ndarray, group: int):
+    """Symmetric RTN quantizer with one scale per `group` consecutive features.  Returns codes [rows, K] int8 and
+    scales [rows, K / group] float32."""
+    T = np.ascontiguousarray(T, dtype=np.float64)
+    rows, K = T.shape
+    bits_per_row = np.ascontiguousarray(bits_per_row, dtype=np.int32)
+    scale = np.empty((rows, K // group), dtype=np.float32)
+    codes = np.empty((rows, K), dtype=np.int8)
+    _check(lib().oracle_quantize_rows_grouped(_p(T), ctypes.c_long(rows), K, _p(bits_per_row), len(bits_per_row),
+                                              int(group), _p(scale), _p(codes)), "quantize_rows_grouped")
+    return codes, scale
+
+
+def quantize_weights_grouped(W: np.ndarray, group: int, bits: int = 4):
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, K = W.shape
+    scale = np.empty((N, K // group), dtype=np.float32)
+    codes = np.empty((N, K), dtype=np.int8)
+    _check(lib().oracle_quantize_rows_grouped_f32in(_p(W), ctypes.c_long(N), K, bits, int(group), _p(scale), _p(codes)),
+           "quantize_weights_grouped")
+    return codes, scale
+
+
+def gemm_grouped(q: np.ndarray, sx: np.ndarray, wq: np.ndarray, sw: np.ndarray, group: int) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.int8)
+    wq = np.ascontiguousarray(wq, dtype=np.int8)
+    sx = np.ascontiguousarray(sx, dtype=np.float32)
+    sw = np.ascontiguousarray(sw, dtype=np.float32)
+    M, K = q.shape
+    N = wq.shape[0]
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().oracle_gemm_grouped(_p(q), _p(sx), _p(wq), _p(sw), ctypes.c_long(M), N, K, int(group), _p(out)),
+           "gemm_grouped")
+    return out
+
+
 def gemm_i32(q: np.ndarray, wq: np.ndarray) -> np.ndarray:
     q = np.ascontiguousarray(q, dtype=np.int8)
     wq = np.ascontiguousarray(wq, dtype=np.int8)
@@ -190,12 +226,15 @@ def matmul_f64(X: np.ndarray, W: np.ndarray) -> np.ndarray:
 
 def stamp_linear(X: np.ndarray, W: np.ndarray, bias: Optional[np.ndarray] = None, *, transform: int,
                  block: int = 0, levels: int = 0, k_hi: int = 64, bits_hi: int = 8, bits_lo: int = 4,
-                 bits_w: int = 4, grid_w: int = 0, asym: bool = False,
+                 bits_w: int = 4, grid_w: int = 0, asym: bool = False, group: int = 0,
                  want=("T", "x_scale", "q", "w_scale", "wq", "acc", "Yt", "Y")) -> Dict[str, np.ndarray]:
     """Run the whole layer; returns the stages named in `want`.
 
     asym=True selects the zero-point activation quantizer: "q" is then uint8 and "x_zero" (int32 per
     transformed token) is returned as well.
+
+    group > 0 selects per-block scales of `group` features for activations and weights: "x_scale" is then
+    [B*L, K/group], "w_scale" [N, K/group], and "acc" is not available.
 
     X [B, L, K] float32 (values already rounded to the storage dtype), W [N, K] float32."""
     X = np.ascontiguousarray(X, dtype=np.float32)
@@ -207,15 +246,18 @@ def stamp_linear(X: np.ndarray, W: np.ndarray, bias: Optional[np.ndarray] = None
         bias = np.ascontiguousarray(bias, dtype=np.float32)
     if asym and "x_scale" in want:
         want = tuple(want) + ("x_zero",)
-    shapes = {"T": ((M, K), np.float64), "x_scale": ((M,), np.float32),
+    ng = K // group if group else 1
+    if group:
+        want = tuple(w for w in want if w != "acc")
+    shapes = {"T": ((M, K), np.float64), "x_scale": ((M, ng) if group else (M,), np.float32),
               "q": ((M, K), np.uint8 if asym else np.int8), "x_zero": ((M,), np.int32),
-              "w_scale": ((N,), np.float32), "wq": ((N, K), np.int8), "acc": ((M, N), np.int32),
+              "w_scale": ((N, ng) if group else (N,), np.float32), "wq": ((N, K), np.int8), "acc": ((M, N), np.int32),
               "Yt": ((M, N), np.float64), "Y": ((M, N), np.float64)}
     out = {k: np.empty(s, dtype=d) for k, (s, d) in shapes.items() if k in want}
     g = out.get
     rc = lib().oracle_stamp_linear(_p(X), _p(W), _p(bias), B, L, K, N, int(transform), int(block), int(levels),
                                    int(k_hi), int(bits_hi), int(bits_lo), int(bits_w), _p(g("T")),
                                    _p(g("x_scale")), _p(g("q")), _p(g("w_scale")), _p(g("wq")), _p(g("acc")),
-                                   _p(g("Yt")), _p(g("Y")), int(grid_w), int(bool(asym)), _p(g("x_zero")))
+                                   _p(g("Yt")), _p(g("Y")), int(grid_w), int(bool(asym)), _p(g("x_zero")), int(group))
     _check(rc, "stamp_linear")
     return out

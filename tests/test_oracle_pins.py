@@ -833,3 +833,76 @@ def test_skip_first_layer_keeps_the_massive_token_out_of_the_detail_rows(oracle)
     assert np.max(full["x_scale"][lo]) > 3.0 * np.max(skip["x_scale"][lo])
     err = lambda y: np.linalg.norm(y - plain) / np.linalg.norm(plain)
     assert err(skip["Y"]) < err(full["Y"])
+
+
+# --------------------------------------------------------------------------------------
+# Per-block ("group") scales of 64 features (LVM table: W4A4 per-block quantization, block size 64)
+# --------------------------------------------------------------------------------------
+
+def test_grouped_quantizer_is_the_per_token_quantizer_on_every_group(oracle):
+    """group = K is the per-token quantizer itself; for group < K every group of a row is quantized exactly as if it
+    were a row of its own (codes and scales equal those of the per-token routine run on the reshaped array)."""
+    rng = np.random.default_rng(31)
+    rows, K, group = 24, 256, 64
+    T = rng.standard_normal((rows, K)) * rng.lognormal(0, 1.5, size=(rows, 1))
+    T[:, 7] *= 40.0                                     # an outlier channel: only its group pays for it
+    bits = np.where(np.arange(rows) < 6, 8, 4).astype(np.int32)
+    q_full, s_full = oracle.quantize_rows_grouped(T, bits, K)
+    q_pt, s_pt = oracle.quantize_rows(T, bits)
+    assert np.array_equal(q_full, q_pt) and np.array_equal(s_full[:, 0], s_pt)
+    q, s = oracle.quantize_rows_grouped(T, bits, group)
+    assert s.shape == (rows, K // group)
+    q_ref, s_ref = oracle.quantize_rows(T.reshape(rows * (K // group), group), np.repeat(bits, K // group))
+    assert np.array_equal(q.reshape(-1, group), q_ref) and np.array_equal(s.reshape(-1), s_ref)
+    # error bound per group (Sec. 2.1's rounding bound with the group's own scale) and the gain over one scale per row
+    err = T - np.repeat(s.astype(np.float64), group, axis=1) * q
+    assert np.all(np.abs(err) <= np.repeat(s.astype(np.float64), group, axis=1) / 2 * (1 + 1e-6))
+    err_pt = T - s_pt.astype(np.float64)[:, None] * q_pt
+    assert np.sum(err ** 2) < 0.5 * np.sum(err_pt ** 2)
+    # hand case: two groups of two, scales 1 and 2
+    qh, sh = oracle.quantize_rows_grouped(np.array([[7.0, -3.5, 14.0, 5.0]]), np.array([4], dtype=np.int32), 2)
+    assert sh.tolist() == [[1.0, 2.0]] and qh.tolist() == [[7, -4, 7, 2]]
+
+
+def test_grouped_product_brute_force_and_reduction_to_the_plain_product(oracle):
+    rng = np.random.default_rng(32)
+    M, N, K, group = 9, 7, 128, 32
+    q = rng.integers(-127, 128, size=(M, K), dtype=np.int8)
+    wq = rng.integers(-7, 8, size=(N, K), dtype=np.int8)
+    sx = rng.uniform(0.5, 2.0, size=(M, K // group)).astype(np.float32)
+    sw = rng.uniform(0.01, 0.1, size=(N, K // group)).astype(np.float32)
+    Yt = oracle.gemm_grouped(q, sx, wq, sw, group)
+    # the definition: product of the de-quantized operands
+    A = q.astype(np.float64) * np.repeat(sx.astype(np.float64), group, axis=1)
+    Wd = wq.astype(np.float64) * np.repeat(sw.astype(np.float64), group, axis=1)
+    assert np.max(np.abs(Yt - A @ Wd.T)) <= 1e-12 * np.max(np.abs(Yt))
+    # one group: the plain integer product times the two scales
+    Y1 = oracle.gemm_grouped(q, sx[:, :1], wq, sw[:, :1], K)
+    assert np.array_equal(Y1, oracle.dequant(oracle.gemm_i32(q, wq), sx[:, 0], sw[:, 0]))
+
+
+def test_grouped_layer_exact_codes_and_closer_than_per_token_on_outlier_channels(oracle):
+    """Whole layer with group scales: inputs whose groups are integer multiples of power-of-two scales give the
+    textbook product; on the DiT stand-in (2 % outlier channels x 30) the grouped layer is closer to X W^T than the
+    per-token layer, with and without the sequence transform -- and STaMP still helps on top (LVM table)."""
+    rng = np.random.default_rng(33)
+    nblk, K, N, group = 4, 128, 6, 64
+    P = rng.integers(-127, 128, size=(nblk, K)); P[:, 0] = 127; P[:, 64] = -127
+    Q = rng.integers(-7, 8, size=(nblk, K)); Q[:, 1] = -7; Q[:, 65] = 7
+    P[:, 64:] *= 1                                        # (second group: same construction, own extreme codes)
+    u, v = (P + Q) / 2.0, (P - Q) / 2.0
+    X = np.stack([u, u, v, v], axis=1).reshape(1, 4 * nblk, K).astype(np.float32)
+    Wi = rng.integers(-7, 8, size=(N, K)); Wi[:, 2] = 7; Wi[:, 66] = -7
+    W = (Wi * 2.0 ** -3).astype(np.float32)
+    out = oracle.stamp_linear(X, W, None, transform=T_HAAR, block=4, levels=2, k_hi=1, group=group)
+    assert np.array_equal(out["wq"], Wi) and np.all(out["x_scale"] == 1.0) and np.all(out["w_scale"] == 2.0 ** -3)
+    ref = X[0].astype(np.float64) @ W.astype(np.float64).T
+    assert np.max(np.abs(out["Y"] - ref)) <= 1e-12 * np.max(np.abs(ref))
+    cfg = gen.scaled(gen.config_dit_proj(), B=1, L=256, K=256, N=64, grid=16, levels=4, k_hi=16)
+    Xc, Wc = gen.make_activation(cfg), gen.make_weight(cfg)
+    plain = oracle.matmul_f64(Xc.reshape(-1, cfg.K), Wc)
+    err = lambda **kw: np.linalg.norm(oracle.stamp_linear(Xc, Wc, None, want=("Y",), **kw)["Y"] - plain) / np.linalg.norm(plain)
+    e_pt_id = err(transform=T_ID, k_hi=0)
+    e_g_id = err(transform=T_ID, k_hi=0, group=64)
+    e_g_stamp = err(transform=T_HAAR, levels=4, k_hi=16, group=64)
+    assert e_g_id < e_pt_id and e_g_stamp < e_g_id
