@@ -74,7 +74,7 @@ typedef enum { STAMP_F32 = 0, STAMP_BF16 = 1 } stamp_dtype;
 typedef enum { STAMP_T_IDENTITY = 0, STAMP_T_HAAR = 1, STAMP_T_DCT2 = 2, STAMP_T_HAAR2D = 3, STAMP_T_WHT = 4,
                STAMP_T_HAAR_SKIP1 = 5 } stamp_transform;
 
-typedef enum { STAMP_G_PER_TOKEN = 0, STAMP_G_PER_CHANNEL = 1 } stamp_granularity;
+typedef enum { STAMP_G_PER_TOKEN = 0, STAMP_G_PER_CHANNEL = 1, STAMP_G_GROUP = 2 } stamp_granularity;
 
 /* Weight operand formats accepted by the GEMM entry points. */
 typedef enum {
@@ -105,6 +105,14 @@ typedef struct {
                            the stored code, zc = z - 2^(b-1):  t ~ s * (c - zc).  Every transform is
                            accepted; the layer then runs as separate transform, quantize, GEMM and
                            inverse kernels.                                                       */
+  int32_t group;     /* 0: one scale per transformed token / per output channel (the fields above).
+                        > 0: per-block scales (the LVM table's setting, "W4A4 per-block quantization with block size
+                        64"): every run of `group` consecutive input features of a transformed token, and of a weight
+                        row, has its own scale = absmax / qmax; act_gran and w_gran must both be STAMP_G_GROUP.
+                        group = 64 * 2^i and divides K; symmetric codes only.  x_scale is then [B, L, K / group] and
+                        w_scale [N, K / group], and
+                          Yt[m, n] = sum_g (sum_{k in g} q[m,k] wq[n,k]) * x_scale[m, g] * w_scale[n, g].
+                        The layer runs as separate transform, group quantizer, CUDA-core product and inverse kernels. */
 } stamp_config;
 
 /* Bytes of scratch any call below may need for this problem size (the maximum over the calls). */

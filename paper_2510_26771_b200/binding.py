@@ -15,7 +15,7 @@ from .build import LIB_PATH
 STAMP_OK = 0
 F32, BF16 = 0, 1
 T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT, T_HAAR_SKIP1 = 0, 1, 2, 3, 4, 5
-G_PER_TOKEN, G_PER_CHANNEL = 0, 1
+G_PER_TOKEN, G_PER_CHANNEL, G_GROUP = 0, 1, 2
 W_PACKED4, W_INT8 = 0, 1
 
 EXPORTS = (
@@ -30,15 +30,18 @@ EXPORTS = (
 
 class StampConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("transform", "block", "levels", "k_hi", "bits_hi", "bits_lo",
-                                              "bits_w", "act_gran", "w_gran", "grid_w", "act_zero_point")]
+                                              "bits_w", "act_gran", "w_gran", "grid_w", "act_zero_point", "group")]
 
 
 def make_config(transform: int, block: int = 0, levels: int = 0, k_hi: int = 64, bits_hi: int = 8,
-                bits_lo: int = 4, bits_w: int = 4, grid_w: int = 0, zero_point: bool = False) -> StampConfig:
+                bits_lo: int = 4, bits_w: int = 4, grid_w: int = 0, zero_point: bool = False,
+                group: int = 0) -> StampConfig:
     """grid_w: width of the patch grid for T_HAAR2D (0 for the other transforms); zero_point: activation
-    codes with a per-token zero point and min-max range instead of the symmetric ones."""
-    return StampConfig(transform, block, levels, k_hi, bits_hi, bits_lo, bits_w, G_PER_TOKEN, G_PER_CHANNEL,
-                       grid_w if transform == T_HAAR2D else 0, 1 if zero_point else 0)
+    codes with a per-token zero point and min-max range instead of the symmetric ones; group: features per
+    scale for activations and weights (0: one scale per token / per output channel)."""
+    gran = (G_GROUP, G_GROUP) if group else (G_PER_TOKEN, G_PER_CHANNEL)
+    return StampConfig(transform, block, levels, k_hi, bits_hi, bits_lo, bits_w, gran[0], gran[1],
+                       grid_w if transform == T_HAAR2D else 0, 1 if zero_point else 0, group)
 
 
 class StampError(RuntimeError):
@@ -110,7 +113,7 @@ def alloc_workspace(cfg: StampConfig, B: int, L: int, K: int, N: int, device="cu
 def stamp_quantize_weights(cfg: StampConfig, W: torch.Tensor):
     N, K = W.shape
     wq = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
-    w_scale = torch.empty((N,), dtype=torch.float32, device=W.device)
+    w_scale = torch.empty((N, K // cfg.group) if cfg.group else (N,), dtype=torch.float32, device=W.device)
     _check(lib().stamp_quantize_weights(ctypes.byref(cfg), _ptr(W), _dtype_code(W), N, K, _ptr(wq), _ptr(w_scale),
                                         _stream()), "stamp_quantize_weights")
     return wq, w_scale
@@ -135,7 +138,8 @@ def stamp_quantize(cfg: StampConfig, X: torch.Tensor, ws: torch.Tensor):
     q_hi = torch.empty((max(nh, 1), K), dtype=torch.int8, device=X.device)
     q_lo = torch.empty((max(B * L - nh, 1), K // 2), dtype=torch.uint8, device=X.device)
     # zero-point codes: the scales, then the zero points of the stored codes as int32 words (split_zero_points)
-    x_scale = torch.empty((2, B, L) if cfg.act_zero_point else (B, L), dtype=torch.float32, device=X.device)
+    x_scale = torch.empty((2, B, L) if cfg.act_zero_point else (B, L, K // cfg.group) if cfg.group else (B, L),
+                          dtype=torch.float32, device=X.device)
     wp, wb = _ws_args(ws)
     _check(lib().stamp_quantize(ctypes.byref(cfg), _ptr(X), _dtype_code(X), B, L, K, _ptr(q_hi), _ptr(q_lo),
                                 _ptr(x_scale), wp, wb, _stream()), "stamp_quantize")

@@ -24,6 +24,7 @@ struct Problem {
   int k_hi;        // 8-bit rows per block
   int grid_w;      // 2-D Haar: patch-grid width of a block (0 otherwise)
   int act_zp;      // 1: zero-point activation codes (min-max range), 0: symmetric
+  int group;       // > 0: one scale per `group` features for activations and weights (0: per token / per channel)
   int nseq;        // B * (L / n): independent transform blocks
   long M;          // B * L tokens
   int qmax_hi, qmax_lo, qmax_w;

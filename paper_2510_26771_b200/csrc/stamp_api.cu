@@ -13,6 +13,7 @@
 #include "k_gemm.cuh"
 #include "k_haar2d.cuh"
 #include "k_generic.cuh"
+#include "k_grouped.cuh"
 #include "k_haar_cq.cuh"
 #include "k_haar_tc.cuh"
 #include "k_peak.cuh"
@@ -48,7 +49,14 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
   if (cfg->block < 0 || cfg->levels < 0 || cfg->k_hi < 0 || cfg->grid_w < 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->transform != STAMP_T_HAAR2D && cfg->grid_w != 0) return STAMP_ERR_INVALID_ARG;
   if (cfg->bits_hi != 8 || cfg->bits_lo != 4 || cfg->bits_w != 4) return STAMP_ERR_UNSUPPORTED;
-  if (cfg->act_gran != STAMP_G_PER_TOKEN || cfg->w_gran != STAMP_G_PER_CHANNEL) return STAMP_ERR_UNSUPPORTED;
+  if (cfg->group < 0) return STAMP_ERR_INVALID_ARG;
+  if (cfg->group == 0) {
+    if (cfg->act_gran != STAMP_G_PER_TOKEN || cfg->w_gran != STAMP_G_PER_CHANNEL) return STAMP_ERR_UNSUPPORTED;
+  } else {
+    // per-block scales: both operands, groups of 64 * 2^i features that divide K, symmetric codes
+    if (cfg->act_gran != STAMP_G_GROUP || cfg->w_gran != STAMP_G_GROUP) return STAMP_ERR_INVALID_ARG;
+    if (cfg->group % 64 != 0 || !is_pow2(cfg->group) || K % cfg->group != 0 || cfg->act_zero_point) return STAMP_ERR_UNSUPPORTED;
+  }
   if (cfg->act_zero_point != 0 && cfg->act_zero_point != 1) return STAMP_ERR_INVALID_ARG;
   const int n = cfg->block ? cfg->block : L;
   if (!is_pow2(n) || L % n != 0) return STAMP_ERR_UNSUPPORTED;
@@ -82,6 +90,7 @@ static int resolve(const stamp_config* cfg, int B, int L, int K, int N, bool nee
   out->k_hi = cfg->k_hi;
   out->grid_w = cfg->grid_w;
   out->act_zp = cfg->act_zero_point;
+  out->group = cfg->group;
   out->nseq = B * (L / n);
   out->M = (long)B * L;
   out->qmax_hi = (1 << (cfg->bits_hi - 1)) - 1;
@@ -132,7 +141,7 @@ static Workspace layout(const Problem& pb) {
   w.rowmax = off; off += align256(M * 4);
   // (directly behind the row maxima: one memset clears both before the tensor-core transform+quantize launch)
   w.htc_cnt = off; off += align256((M >> 7) * 4 + 4);
-  w.xscale = off; off += align256(M * 4);
+  w.xscale = off; off += align256(M * 4 * (size_t)(pb.group ? pb.K / pb.group : 1));
   // low-pass band after the first level of the first-token-excluded Haar transform (forward: K wide, inverse: N wide)
   w.skipa = off;  off += align256(pb.transform == STAMP_T_HAAR_SKIP1 ? (M / 2) * KN * 4 : 0);
   w.T = off;      off += align256(M * (size_t)pb.K * 4);
@@ -681,6 +690,23 @@ static int run_quant_rows_zp(const Problem& pb, const float* T, int8_t* a8, void
   return STAMP_OK;
 }
 
+// Per-block scales: quantize materialised rows group by group; the dp4a product that scales every group.
+static int run_quant_rows_grouped(const Problem& pb, const float* T, int8_t* a8, void* q_hi, void* q_lo, float* x_scale,
+                                  cudaStream_t st) {
+  k_quant_rows_grouped<<<(unsigned)pb.M, 256, (size_t)(pb.K / 64) * 4, st>>>(T, pb.K, pb.n, pb.k_hi, pb.qmax_hi, pb.qmax_lo,
+                                                                            pb.group, a8, static_cast<int8_t*>(q_hi),
+                                                                            static_cast<uint8_t*>(q_lo), x_scale);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+static int run_gemm_grouped(const Problem& pb, const int8_t* a8, const int8_t* w8, const float* x_scale,
+                            const float* w_scale, float* Yt, cudaStream_t st) {
+  dim3 grid((unsigned)((pb.N + GG_TILE - 1) / GG_TILE), (unsigned)((pb.M + GG_TILE - 1) / GG_TILE));
+  k_gemm_grouped<<<grid, 256, 0, st>>>(a8, w8, x_scale, w_scale, pb.M, pb.N, pb.K, pb.group, Yt);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
 static int run_weight_row_sums(const int8_t* w8, int N, int K, int* w_sum, cudaStream_t st) {
   k_row_sums_i8<<<(unsigned)((N + 7) / 8), 256, 0, st>>>(w8, N, K, w_sum);
   STAMP_CHECK_LAUNCH();
@@ -1086,6 +1112,10 @@ enum FusedRoute { ROUTE_PATCH2D = 0, ROUTE_ZP_GENERAL = 1, ROUTE_TILED = 2, ROUT
 static FusedRoute fused_route(const Problem& pb, int x_dtype, CqChoice* cc, bool* have_cq) {
   const bool patch_fits = (size_t)64 * pb.K * (x_dtype == STAMP_BF16 ? 2 : 4) <= 224 * 1024;
   *have_cq = (pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, cc);
+  if (pb.group) {   // per-block scales: separate transform, group quantizer, CUDA-core product, inverse
+    *have_cq = false;
+    return ROUTE_GENERAL;
+  }
   if (pb.transform == STAMP_T_HAAR2D && pb.levels == 3 && pb.M % 256 == 0 && (!pb.act_zp || patch_fits)) return ROUTE_PATCH2D;
   if (pb.act_zp) return ROUTE_ZP_GENERAL;
   if (*have_cq && pb.transform == STAMP_T_HAAR && pb.levels >= 5 && pb.n % 256 == 0) return ROUTE_TILED;
@@ -1162,8 +1192,22 @@ int stamp_quantize_weights(const stamp_config* cfg, const void* W, int w_dtype, 
                            float* w_scale, void* stream) {
   t_launches = 0;
   if (!cfg || !W || !wq || !w_scale || N <= 0 || K <= 0 || !dtype_ok(w_dtype)) return STAMP_ERR_INVALID_ARG;
-  if (cfg->bits_w != 4 || cfg->w_gran != STAMP_G_PER_CHANNEL || K % 128 != 0) return STAMP_ERR_UNSUPPORTED;
+  if (cfg->bits_w != 4 || K % 128 != 0) return STAMP_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cfg->group > 0) {
+    if (cfg->w_gran != STAMP_G_GROUP || cfg->group % 64 != 0 || !is_pow2(cfg->group) || K % cfg->group != 0)
+      return STAMP_ERR_UNSUPPORTED;
+    const size_t sm = (size_t)(K / 64) * 4;
+    if (w_dtype == STAMP_BF16)
+      k_quant_weights_grouped<__nv_bfloat16><<<N, 256, sm, st>>>(static_cast<const __nv_bfloat16*>(W), K, 7, cfg->group,
+                                                                 static_cast<uint8_t*>(wq), w_scale);
+    else
+      k_quant_weights_grouped<float><<<N, 256, sm, st>>>(static_cast<const float*>(W), K, 7, cfg->group,
+                                                         static_cast<uint8_t*>(wq), w_scale);
+    STAMP_CHECK_LAUNCH();
+    return STAMP_OK;
+  }
+  if (cfg->w_gran != STAMP_G_PER_CHANNEL) return STAMP_ERR_UNSUPPORTED;
   if (w_dtype == STAMP_BF16)
     k_quant_weights<__nv_bfloat16><<<N, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W), K, 7,
                                                       static_cast<uint8_t*>(wq), w_scale);
@@ -1203,6 +1247,13 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
     if (rc) return rc;
     return run_quant_rows_zp(pb, T, nullptr, q_hi, q_lo, x_scale, reinterpret_cast<int*>(x_scale + pb.M), st);
   }
+  if (pb.group) {
+    rc = run_transform_generic(pb, X, x_dtype, T, nullptr, reinterpret_cast<float*>(base + w.ping),
+                               reinterpret_cast<float*>(base + w.pong), reinterpret_cast<float*>(base + w.dctmat), st,
+                               reinterpret_cast<float*>(base + w.skipa));
+    if (rc) return rc;
+    return run_quant_rows_grouped(pb, T, nullptr, q_hi, q_lo, x_scale, st);
+  }
   CqChoice cc;
   if ((pb.transform == STAMP_T_HAAR || pb.transform == STAMP_T_IDENTITY) && choose_cq(pb.K, &cc))
     return run_quantize_haar(pb, cc, X, x_dtype, nullptr, q_hi, q_lo, x_scale, nullptr, base, w, st);
@@ -1237,6 +1288,7 @@ int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, co
   if ((rc = run_unpack_codes(pb, q_hi, q_lo, a8, st))) return rc;
   const int8_t* w8 = nullptr;
   if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8, st))) return rc;
+  if (pb.group) return run_gemm_grouped(pb, a8, w8, x_scale, w_scale, Yt, st);
   if (pb.act_zp) {
     int* w_sum = reinterpret_cast<int*>(base + wl.wsum);
     if ((rc = run_weight_row_sums(w8, N, K, w_sum, st))) return rc;
@@ -1378,6 +1430,17 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     }
     if ((rc = launch_gemm(a8, w8d, pb.M, N, K, x_scale, w_scale, yt, EPI_DEQUANT_F32, st))) return rc;
     return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st, reinterpret_cast<float*>(base + wl.skipa));
+  }
+  if (pb.group) {
+    if ((rc = run_transform_generic(pb, X, x_dtype, T, nullptr, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st,
+                                    reinterpret_cast<float*>(base + wl.skipa))))
+      return rc;
+    if ((rc = run_quant_rows_grouped(pb, T, a8, nullptr, nullptr, x_scale, st))) return rc;
+    const int8_t* w8g = nullptr;
+    if ((rc = weights_as_int8(pb, w, w_format, reinterpret_cast<int8_t*>(base + wl.w8), &w8g, st))) return rc;
+    if ((rc = run_gemm_grouped(pb, a8, w8g, x_scale, w_scale, yt, st))) return rc;
+    return run_inverse_generic(pb, yt, bias, Y, y_dtype, ping, pong, reinterpret_cast<float*>(base + wl.dctmat), st,
+                               reinterpret_cast<float*>(base + wl.skipa));
   }
   if (have_cq) {
     if ((rc = run_quantize_haar(pb, cc, X, x_dtype, a8, nullptr, nullptr, x_scale, nullptr, base, wl, st))) return rc;

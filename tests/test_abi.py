@@ -36,7 +36,7 @@ def test_status_strings(st):
 
 
 def test_config_struct_matches_header(st):
-    assert ctypes.sizeof(st.StampConfig) == 44      # eleven int32 fields
+    assert ctypes.sizeof(st.StampConfig) == 48      # twelve int32 fields
     header = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "stamp.h")).read()
     body = header[header.index("typedef struct {"):header.index("} stamp_config;")]
     names = re.findall(r"int32_t\s+(\w+);", body)

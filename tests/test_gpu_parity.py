@@ -497,3 +497,80 @@ def test_guard_bands_around_workspace_and_output_stay_intact(st, name):
         assert bool((raw[:guard] == 0xA5).all()) and bool((raw[guard + need:] == 0xA5).all()), "workspace overrun"
         assert bool((yraw[:guard] == 0x5A).all()) and bool((yraw[guard + ybytes:] == 0x5A).all()), "output overrun"
     assert st.stamp_last_device_status() == 0
+
+
+GROUP_CASES = {
+    # the LVM table's setting on the DiT stand-in: 3-level 2-D Haar, 64 low-pass tokens at 8 bits, blocks of 64 features
+    "g64_haar2d": (gen.scaled(gen.config_dit_proj_2d(), B=1, L=1024, K=256, N=136, grid=32, k_hi=16), 64),
+    # 1-D Haar with ragged tiles; a larger block; no transform at all (plain per-block W4A4)
+    "g64_haar": (gen.scaled(gen.config_llm_up(), B=2, L=512, K=384, N=392, k_hi=16), 64),
+    "g128_haar": (gen.scaled(gen.config_llm_up(), B=1, L=256, K=384, N=72, k_hi=8), 128),
+    "g64_identity": (gen.scaled(gen.config_sweep(512, 2048), L=256, K=256, N=128, transform=gen.T_IDENTITY, k_hi=0), 64),
+    # the DiT projection at full size (all 1152 output channels on the GPU, 64 of them through the oracle)
+    "g64_dit_full": (gen.config_dit_proj_2d(), 64),
+}
+
+
+@pytest.mark.parametrize("name", list(GROUP_CASES))
+def test_group_scale_parity(st, oracle, name):
+    """Per-block scales of 64 (128) features for activations and weights against the oracle: weight scales equal,
+    activation scales within the tolerance of T, codes within the tie budget, the product of the oracle's codes and
+    scales within fp32 rounding, the one-call layer within the output tolerance."""
+    import torch
+    cfg, group = GROUP_CASES[name]
+    c = st.make_config(cfg.transform, cfg.block, cfg.levels, cfg.k_hi, grid_w=cfg.grid, group=group)
+    B, L, K, N, M = cfg.B, cfg.L, cfg.K, cfg.N, cfg.M
+    X, bias = gen.make_activation(cfg), gen.make_bias(cfg)
+    cols = np.arange(N) if N <= 512 else np.sort(np.random.default_rng(7).choice(N, size=64, replace=False))
+    W = gen.make_weight(cfg)
+    ref = oracle.stamp_linear(X, W[cols], bias[cols], transform=cfg.transform, block=cfg.block, levels=cfg.levels,
+                              k_hi=cfg.k_hi, grid_w=cfg.grid, group=group, want=("x_scale", "q", "w_scale", "wq", "Yt", "Y"))
+    Xd, Wd, bd = H.to_device(X, cfg.dtype), H.to_device(W, cfg.dtype), torch.from_numpy(bias).cuda()
+    ws = st.alloc_workspace(c, B, L, K, N)
+    # weights
+    wq, wsc = st.stamp_quantize_weights(c, Wd)
+    assert wsc.shape == (N, K // group)
+    assert np.array_equal(wsc.cpu().numpy()[cols], ref["w_scale"])
+    w8 = st.stamp_prepare_weights(c, wq)
+    bad, worst = H.code_mismatch(w8.cpu().numpy()[cols], ref["wq"])
+    assert worst <= 1 and bad <= _allowed(ref["wq"].size), (bad, worst)
+    # activations
+    q_hi, q_lo, xs = st.stamp_quantize(c, Xd, ws)
+    assert xs.shape == (B, L, K // group)
+    assert np.allclose(xs.cpu().numpy().reshape(M, -1), ref["x_scale"], rtol=_scale_rtol(cfg), atol=0)
+    codes = st.stamp_debug_unpack_codes(c, q_hi, q_lo, B, L, K).cpu().numpy().reshape(M, K)
+    bad, worst = H.code_mismatch(codes, ref["q"])
+    print(f"[{name}] group-scaled activation code mismatches: {bad} of {codes.size} (max |diff| {worst})")
+    assert worst <= 1 and bad <= _allowed(codes.size), (bad, worst)
+    # product fed the oracle's codes and scales (all output channels of the oracle's subset)
+    if N <= 512:
+        oq_hi, oq_lo = H.pack_codes(ref["q"], cfg.block_len, cfg.k_hi)
+        Yt = st.stamp_linear(c, torch.from_numpy(oq_hi).cuda(), torch.from_numpy(oq_lo).cuda(),
+                             torch.from_numpy(ref["x_scale"]).cuda().reshape(B, L, -1),
+                             torch.from_numpy(H.pack_nibbles(ref["wq"])).cuda(), st.W_PACKED4,
+                             torch.from_numpy(ref["w_scale"]).cuda(), B, L, K, N, ws).cpu().numpy().reshape(M, N)
+        assert H.rel_fro(Yt, ref["Yt"]) <= 1e-6
+    # the layer: chained calls and the one-call form
+    Yt2 = st.stamp_linear(c, q_hi, q_lo, xs, wq, st.W_PACKED4, wsc, B, L, K, N, ws)
+    Y2 = st.stamp_inverse(c, Yt2, bd, ws).cpu().numpy().reshape(M, N)[:, cols]
+    Y3 = st.stamp_linear_fused(c, Xd, w8, st.W_INT8, wsc, bd, ws).cpu().numpy().reshape(M, N)[:, cols]
+    e2, e3 = H.rel_fro(Y2, ref["Y"]), H.rel_fro(Y3, ref["Y"])
+    print(f"[{name}] output relative Frobenius error: chained {e2:.2e}, one call {e3:.2e}")
+    assert e2 <= (Y_TOL_HAAR if bad == 0 else Y_TOL) and e3 <= (Y_TOL_HAAR if bad == 0 else Y_TOL)
+    assert st.stamp_last_device_status() == 0
+
+
+def test_group_scale_arguments_are_checked(st):
+    import ctypes
+    lib = st.lib()
+    out = ctypes.c_size_t(0)
+    ok = st.make_config(st.T_HAAR, 0, 0, 16, group=64)
+    assert lib.stamp_workspace_bytes(ctypes.byref(ok), 1, 256, 256, 64, ctypes.byref(out)) == 0
+    for bad_group in (48, 96, 192):                      # not 64 * 2^i, or not a divisor of K
+        c = st.make_config(st.T_HAAR, 0, 0, 16, group=bad_group)
+        assert lib.stamp_workspace_bytes(ctypes.byref(c), 1, 256, 384, 64, ctypes.byref(out)) == 2
+    c = st.make_config(st.T_HAAR, 0, 0, 16, group=64, zero_point=True)
+    assert lib.stamp_workspace_bytes(ctypes.byref(c), 1, 256, 256, 64, ctypes.byref(out)) == 2
+    c = st.make_config(st.T_HAAR, 0, 0, 16, group=64)
+    c.w_gran = st.G_PER_CHANNEL                          # group set but the granularity fields disagree
+    assert lib.stamp_workspace_bytes(ctypes.byref(c), 1, 256, 256, 64, ctypes.byref(out)) == 1
