@@ -166,6 +166,19 @@ int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, co
                  void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * De-quantization of stored codes, s (x_int - z) of Sec. 2.1: the transformed activation as the quantizer left it.
+ * With stamp_quantize before and stamp_inverse (N = K, no bias) after it, this is STaMP on a tensor that is stored
+ * rather than multiplied at once -- the KV cache of the LLM experiments (Table "STaMP always improves LLM
+ * quantization": KV cache at 4 bits with the first 64 transformed tokens at 8; App. "Experimental details / LLMs":
+ * scales per token and head).  A cache of H heads of dimension 128 is the activation [B * H, L, 128]: the per-token
+ * scale of every sequence is then a per-token, per-head scale.
+ *   q_hi, q_lo, x_scale : as written by stamp_quantize (zero points and per-block scales included)     in
+ *   T        [B, L, K]   float, transformed-token (logical) order                                      out
+ */
+int stamp_dequantize(const stamp_config* cfg, const void* q_hi, const void* q_lo, const float* x_scale, int B, int L,
+                     int K, float* T, void* stream);
+
+/*
  * Algorithm lines "Y <- L^-1 Y" and "Y <- Y + bias": inverse sequence transform along tokens
  * (L^-1 = L^T, L orthonormal: Theorem 1's premise) and optional bias.
  *   Yt       [B, L, N]   float                                                       in

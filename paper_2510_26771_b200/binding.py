@@ -25,6 +25,7 @@ EXPORTS = (
     "stamp_debug_unpack_codes", "stamp_debug_gemm_i32", "stamp_last_device_status",
     "stamp_last_launch_count", "stamp_status_string", "stamp_inverse_noalloc", "stamp_debug_fused_operand",
     "stamp_measure_i8_mma_issue", "stamp_debug_expire_wait",
+    "stamp_dequantize",
 )
 
 
@@ -159,6 +160,14 @@ def stamp_linear(cfg: StampConfig, q_hi, q_lo, x_scale, w, w_format: int, w_scal
     _check(lib().stamp_linear(ctypes.byref(cfg), _ptr(q_hi), _ptr(q_lo), _ptr(x_scale), _ptr(w), int(w_format),
                               _ptr(w_scale), B, L, K, N, _ptr(Yt), wp, wb, _stream()), "stamp_linear")
     return Yt
+
+
+def stamp_dequantize(cfg: StampConfig, q_hi, q_lo, x_scale, B: int, L: int, K: int) -> torch.Tensor:
+    """Stored codes back to transformed values, s (x_int - z): the read side of a STaMP-quantized cache."""
+    T = torch.empty((B, L, K), dtype=torch.float32, device=x_scale.device)
+    _check(lib().stamp_dequantize(ctypes.byref(cfg), _ptr(q_hi), _ptr(q_lo), _ptr(x_scale), B, L, K, _ptr(T), _stream()),
+           "stamp_dequantize")
+    return T
 
 
 def stamp_inverse(cfg: StampConfig, Yt: torch.Tensor, bias: Optional[torch.Tensor], ws: torch.Tensor,

@@ -447,6 +447,34 @@ __global__ void __launch_bounds__(256) k_pack_codes(const int8_t* __restrict__ c
   }
 }
 
+// De-quantization of stored activation codes back to transformed values (Sec. 2.1: s (x_int - z)): what a reader
+// of a STaMP-quantized KV cache does before the inverse sequence transform.  One CTA per logical row.
+//   T[r, k] = x_scale[r (, k / group)] * (code[r, k] - zero[r])        zero: null for symmetric codes
+__global__ void __launch_bounds__(256) k_dequant_rows(const int8_t* __restrict__ q_hi, const uint8_t* __restrict__ q_lo,
+                                                      const float* __restrict__ x_scale, const int* __restrict__ x_zero,
+                                                      int K, int n, int k_hi, int group, float* __restrict__ T) {
+  const long r = blockIdx.x;
+  const long s = r / n;
+  const int i = static_cast<int>(r - s * n);
+  const int zc = x_zero ? x_zero[r] : 0;
+  const int ng = group ? K / group : 1;
+  const float* sc = x_scale + r * (long)ng;
+  float* dst = T + r * (long)K;
+  if (i < k_hi) {
+    const int8_t* src = q_hi + (s * k_hi + i) * (long)K;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) dst[k] = sc[group ? k / group : 0] * static_cast<float>(src[k] - zc);
+  } else {
+    const uint8_t* src = q_lo + (s * (n - k_hi) + (i - k_hi)) * (long)(K / 2);
+    for (int k2 = threadIdx.x; k2 < K / 2; k2 += blockDim.x) {
+      const uint32_t u = src[k2];
+      const int c0 = static_cast<int>(u << 28) >> 28, c1 = static_cast<int>(u << 24) >> 28;   // sign-extended nibbles
+      const float f = sc[group ? (2 * k2) / group : 0];
+      dst[2 * k2] = f * static_cast<float>(c0 - zc);
+      dst[2 * k2 + 1] = f * static_cast<float>(c1 - zc);
+    }
+  }
+}
+
 // Packed 4-bit rows -> int8 rows (weights). One CTA per row.
 __global__ void __launch_bounds__(256) k_unpack_rows4(const uint8_t* __restrict__ packed, int K, int8_t* __restrict__ out) {
   const long r = blockIdx.x;

@@ -1298,6 +1298,21 @@ int stamp_linear(const stamp_config* cfg, const void* q_hi, const void* q_lo, co
   return launch_gemm(a8, w8, pb.M, N, K, x_scale, w_scale, Yt, EPI_DEQUANT_F32, st);
 }
 
+int stamp_dequantize(const stamp_config* cfg, const void* q_hi, const void* q_lo, const float* x_scale, int B, int L,
+                     int K, float* T, void* stream) {
+  t_launches = 0;
+  Problem pb;
+  int rc = resolve(cfg, B, L, K, 0, false, &pb);
+  if (rc) return rc;
+  if (!x_scale || !T) return STAMP_ERR_INVALID_ARG;
+  if ((pb.n_hi_rows() > 0 && !q_hi) || (pb.n_lo_rows() > 0 && !q_lo)) return STAMP_ERR_INVALID_ARG;
+  const int* zero = pb.act_zp ? reinterpret_cast<const int*>(x_scale + pb.M) : nullptr;
+  k_dequant_rows<<<(unsigned)pb.M, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const int8_t*>(q_hi), static_cast<const uint8_t*>(q_lo), x_scale, zero, K, pb.n, pb.k_hi, pb.group, T);
+  STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
 int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
                   int y_dtype, void* ws, size_t ws_bytes, void* stream) {
   t_launches = 0;
