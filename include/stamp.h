@@ -201,9 +201,14 @@ int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, i
  * Here that scratch is an array compiled into the library, STAMP_NOALLOC_SCRATCH_BYTES per GPU
  * that loads the library, resident until the process exits.  The call performs no cudaMalloc,
  * cudaFree or any other allocating routine.
- *   - Limit: the partial sums of the inverse -- about (B*L/32 + B*L/1024) * N * 4 bytes for a
- *     Haar transform deeper than 5 levels, nothing for 5 levels or fewer -- must fit the array;
- *     otherwise STAMP_ERR_TOO_LARGE is returned before anything is launched.
+ *   - Limit: what the inverse keeps between its launches must fit the array, otherwise
+ *     STAMP_ERR_TOO_LARGE is returned before anything is launched:
+ *       Haar: the partial sums of the coarse-to-fine passes -- nothing up to 5 levels, B*L/32 * N * 4
+ *         bytes for 6 to 10 levels, (B*L/32 + B*L/1024) * N * 4 bytes beyond;
+ *       DCT-II and Walsh-Hadamard: the dense block x block fp32 matrix, block^2 * 4 bytes -- a block of
+ *         1024 tokens fills the 4 MiB exactly, longer blocks are refused;
+ *       2-D Haar and identity: nothing.
+ *     The first-token-excluded Haar transform is not served by this call (STAMP_ERR_UNSUPPORTED).
  *   - The first call on each device looks up the array's device address (with that device
  *     current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array.  Nothing in it has to be cleared between
