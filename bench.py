@@ -265,7 +265,7 @@ def quick_reading(st, cfg, y_t, steps):
     g1.record()
 
     def step(i):
-        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], w_fmt, w_scale, bias, ws, out=Y)
+        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], w_fmt, w_scale, bias, ws, out=Y, n_out=cfg.N)
     ms = time_loop(step, steps, warm=20)
     launches = st.stamp_last_launch_count()
     st.stamp_profile_gemm_events(g0, g1)
@@ -284,8 +284,9 @@ def quick_reading(st, cfg, y_t, steps):
 
 def weight_operand(st, c, wq):
     """The weight operand the benchmark hands to the layer: prepared once, offline (weights are static)."""
-    w8 = st.stamp_prepare_weights(c, wq)
-    return w8, st.W_INT8, "int4 codes, one per int8, prepared offline"
+    both = st.stamp_prepare_weights_both(c, wq)
+    return both, st.W_INT8_AND_PACKED4, ("int4 codes prepared offline: one per int8 for the tensor cores, "
+                                         "packed two per byte for the kernels that only stream them")
 
 
 def main():
@@ -353,7 +354,7 @@ def main():
     ws = st.alloc_workspace(c, B, L, K, N)
 
     def step(i):
-        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], w_fmt, w_scale, bias, ws, out=Y)
+        st.stamp_linear_fused(c, Xs[i % n_x], Ws[i % n_w], w_fmt, w_scale, bias, ws, out=Y, n_out=cfg.N)
 
     if args.quick and args.stage == "quantize":
         def step(i):  # noqa: F811
@@ -462,7 +463,7 @@ def main():
         for i in range(iters):
             stream, ws_h, Y_host = lanes[i % 2]
             with torch.cuda.stream(stream):
-                st.stamp_linear_fused_host(c, X_host, Ws[i % n_w], w_fmt, w_scale, bias, Y_host, ws_h)
+                st.stamp_linear_fused_host(c, X_host, Ws[i % n_w], w_fmt, w_scale, bias, Y_host, ws_h, n_out=N)
         for lane in lanes:
             done = torch.cuda.Event()
             done.record(lane[0])

@@ -80,8 +80,12 @@ typedef enum { STAMP_G_PER_TOKEN = 0, STAMP_G_PER_CHANNEL = 1, STAMP_G_GROUP = 2
 typedef enum {
   STAMP_W_PACKED4 = 0, /* [N, K/2] two's-complement nibbles, low nibble = even k (the output of
                           stamp_quantize_weights); expanded into the workspace on every call  */
-  STAMP_W_INT8 = 1     /* [N, K] one 4-bit code per int8 (the output of stamp_prepare_weights):
+  STAMP_W_INT8 = 1,    /* [N, K] one 4-bit code per int8 (the output of stamp_prepare_weights):
                           the tensor-core operand format, made once for static weights        */
+  STAMP_W_INT8_AND_PACKED4 = 2 /* both: [N, K] int8 directly followed by [N, K/2] packed (the output of
+                          stamp_prepare_weights_both).  The tensor cores read the first part; kernels that only
+                          stream the weights (the product with the few tokens above the GEMM's tiles, for
+                          short sequences) read the packed part and move half the bytes               */
 } stamp_weight_format;
 
 /* The knobs of the paper's problem statement. */
@@ -134,6 +138,10 @@ int stamp_quantize_weights(const stamp_config* cfg, const void* W, int w_dtype, 
  * is a storage choice of this implementation (the int8 MMA consumes one code per byte). */
 int stamp_prepare_weights(const stamp_config* cfg, const void* wq_packed, int N, int K, void* w_int8,
                           void* stream);
+
+/* The same, with the packed codes kept behind the expanded ones (STAMP_W_INT8_AND_PACKED4): w_both holds
+ * N * K + N * K / 2 bytes.  No counterpart in the paper. */
+int stamp_prepare_weights_both(const stamp_config* cfg, const void* wq_packed, int N, int K, void* w_both, void* stream);
 
 /*
  * Algorithm lines "X <- L X" and "x_i <- Q(x_i; b_i)": sequence transform + per-token

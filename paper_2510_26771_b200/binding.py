@@ -16,7 +16,7 @@ STAMP_OK = 0
 F32, BF16 = 0, 1
 T_IDENTITY, T_HAAR, T_DCT2, T_HAAR2D, T_WHT, T_HAAR_SKIP1 = 0, 1, 2, 3, 4, 5
 G_PER_TOKEN, G_PER_CHANNEL, G_GROUP = 0, 1, 2
-W_PACKED4, W_INT8 = 0, 1
+W_PACKED4, W_INT8, W_INT8_AND_PACKED4 = 0, 1, 2
 
 EXPORTS = (
     "stamp_workspace_bytes", "stamp_quantize_weights", "stamp_prepare_weights", "stamp_quantize",
@@ -25,7 +25,7 @@ EXPORTS = (
     "stamp_debug_unpack_codes", "stamp_debug_gemm_i32", "stamp_last_device_status",
     "stamp_last_launch_count", "stamp_status_string", "stamp_inverse_noalloc", "stamp_debug_fused_operand",
     "stamp_measure_i8_mma_issue", "stamp_debug_expire_wait",
-    "stamp_dequantize",
+    "stamp_dequantize", "stamp_prepare_weights_both",
 )
 
 
@@ -128,6 +128,16 @@ def stamp_prepare_weights(cfg: StampConfig, wq: torch.Tensor) -> torch.Tensor:
     return w8
 
 
+def stamp_prepare_weights_both(cfg: StampConfig, wq: torch.Tensor) -> torch.Tensor:
+    """Expanded int8 codes [N, K] followed by the packed ones [N, K/2] in one buffer of N * K * 3 / 2 bytes
+    (weight format W_INT8_AND_PACKED4); pass N to the calls that take it through `n_out`."""
+    N, K2 = wq.shape
+    both = torch.empty((N * 3 * K2,), dtype=torch.int8, device=wq.device)
+    _check(lib().stamp_prepare_weights_both(ctypes.byref(cfg), _ptr(wq), N, 2 * K2, _ptr(both), _stream()),
+           "stamp_prepare_weights_both")
+    return both
+
+
 def n_hi_rows(cfg: StampConfig, B: int, L: int) -> int:
     n = cfg.block if cfg.block else L
     return B * (L // n) * cfg.k_hi
@@ -194,9 +204,9 @@ def stamp_inverse_noalloc(cfg: StampConfig, Yt: torch.Tensor, bias: Optional[tor
 
 def stamp_linear_fused(cfg: StampConfig, X: torch.Tensor, w: torch.Tensor, w_format: int, w_scale: torch.Tensor,
                        bias: Optional[torch.Tensor], ws: torch.Tensor, out_dtype=torch.float32,
-                       out: Optional[torch.Tensor] = None) -> torch.Tensor:
+                       out: Optional[torch.Tensor] = None, n_out: Optional[int] = None) -> torch.Tensor:
     B, L, K = X.shape
-    N = w.shape[0]
+    N = n_out if n_out is not None else w.shape[0]
     Y = out if out is not None else torch.empty((B, L, N), dtype=out_dtype, device=X.device)
     wp, wb = _ws_args(ws)
     _check(lib().stamp_linear_fused(ctypes.byref(cfg), _ptr(X), _dtype_code(X), _ptr(w), int(w_format),
@@ -214,10 +224,10 @@ def stamp_workspace_bytes_host(cfg: StampConfig, B: int, L: int, K: int, N: int,
 
 def stamp_linear_fused_host(cfg: StampConfig, X_host: torch.Tensor, w: torch.Tensor, w_format: int,
                             w_scale: torch.Tensor, bias: Optional[torch.Tensor], Y_host: torch.Tensor,
-                            ws: torch.Tensor) -> torch.Tensor:
+                            ws: torch.Tensor, n_out: Optional[int] = None) -> torch.Tensor:
     """X_host / Y_host are CPU tensors (pinned for asynchronous copies); everything else is on the device."""
     B, L, K = X_host.shape
-    N = w.shape[0]
+    N = n_out if n_out is not None else w.shape[0]
     if X_host.is_cuda or Y_host.is_cuda or not X_host.is_contiguous() or not Y_host.is_contiguous():
         raise ValueError("expected contiguous host tensors")
     wp, wb = _ws_args(ws)

@@ -16,9 +16,20 @@ namespace stamp {
 constexpr int TOPG_THREADS = 256;
 constexpr int TOPG_CH_PER_WARP = 4;
 
+// Eight two's-complement nibbles of a word (nibble 0 = lowest = even feature first) -> eight int8 in two words.
+__device__ __forceinline__ void topg_unpack8(uint32_t w, uint32_t& b0, uint32_t& b1) {
+  uint32_t lo = w & 0x0F0F0F0Fu, hi = (w >> 4) & 0x0F0F0F0Fu;      // features 0, 2, 4, 6 / 1, 3, 5, 7
+  lo |= (lo & 0x08080808u) * 0x1Eu;                                // sign-extend every byte: bit 3 -> bits 4..7
+  hi |= (hi & 0x08080808u) * 0x1Eu;
+  b0 = __byte_perm(lo, hi, 0x5140);
+  b1 = __byte_perm(lo, hi, 0x7362);
+}
+
 // R = total top rows (nseq * rows_per_block), rows_per_block = 2^top_levels.
 //   codes [R, K] int8, x_scale [R], w8 [n_out, K] int8, a8v [R, n_out] float
-template <int R>
+// PACKED: the weights are read as packed 4-bit codes [n_out, K / 2] instead (half the bytes of what is a pure
+// weight stream) and expanded in registers; a lane then covers 32 features per 16-byte load.
+template <int R, bool PACKED = false>
 __global__ void __launch_bounds__(TOPG_THREADS, (R <= 4 ? 3 : (R <= 8 ? 4 : 2))) k_top_gemv(const int8_t* __restrict__ codes,
                                                            const float* __restrict__ x_scale,
                                                            const int8_t* __restrict__ w8, int K, int n_out,
@@ -44,19 +55,46 @@ __global__ void __launch_bounds__(TOPG_THREADS, (R <= 4 ? 3 : (R <= 8 ? 4 : 2)))
   // flight: measured 0.077 -> 0.060 ms per layer step at R = 2, K = 8192); from R = 8 on one step per iteration is
   // as fast or faster (the second set of loads would cost occupancy).
   constexpr int NSTEP = (R <= 4) ? 2 : 1;
-  for (int k0 = lane * 16; k0 < K; k0 += NSTEP * 32 * 16) {
-    const bool second = NSTEP == 2 && k0 + 32 * 16 < K;
+  constexpr int FPL = PACKED ? 32 : 16;     // features per lane and 16-byte load
+  for (int k0 = lane * FPL; k0 < K; k0 += NSTEP * 32 * FPL) {
+    const bool second = NSTEP == 2 && k0 + 32 * FPL < K;
     uint4 w[TOPG_CH_PER_WARP][NSTEP];
 #pragma unroll
     for (int c = 0; c < TOPG_CH_PER_WARP; ++c) {
       const int ch = min(ch0 + c, n_out - 1);   // a ragged last group re-reads the last channel, stores are guarded
-      const uint4* wp = reinterpret_cast<const uint4*>(w8 + (long)ch * K + k0);
+      const uint4* wp = PACKED ? reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(w8) + (long)ch * (K / 2) + k0 / 2)
+                               : reinterpret_cast<const uint4*>(w8 + (long)ch * K + k0);
       w[c][0] = __ldg(wp);
       if (NSTEP == 2) w[c][NSTEP - 1] = second ? __ldg(wp + 32) : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
     for (int u = 0; u < NSTEP; ++u) {
       if (u == 1 && !second) break;
+      if constexpr (PACKED) {
+#pragma unroll
+        for (int c = 0; c < TOPG_CH_PER_WARP; ++c) {
+          uint32_t b[8];
+          topg_unpack8(w[c][u].x, b[0], b[1]);
+          topg_unpack8(w[c][u].y, b[2], b[3]);
+          topg_unpack8(w[c][u].z, b[4], b[5]);
+          topg_unpack8(w[c][u].w, b[6], b[7]);
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            const uint4 a0 = *reinterpret_cast<const uint4*>(topg_smem + r * K + k0 + u * 32 * FPL);
+            const uint4 a1 = *reinterpret_cast<const uint4*>(topg_smem + r * K + k0 + u * 32 * FPL + 16);
+            int s = acc[c][r];
+            s = __dp4a(static_cast<int>(a0.x), static_cast<int>(b[0]), s);
+            s = __dp4a(static_cast<int>(a0.y), static_cast<int>(b[1]), s);
+            s = __dp4a(static_cast<int>(a0.z), static_cast<int>(b[2]), s);
+            s = __dp4a(static_cast<int>(a0.w), static_cast<int>(b[3]), s);
+            s = __dp4a(static_cast<int>(a1.x), static_cast<int>(b[4]), s);
+            s = __dp4a(static_cast<int>(a1.y), static_cast<int>(b[5]), s);
+            s = __dp4a(static_cast<int>(a1.z), static_cast<int>(b[6]), s);
+            s = __dp4a(static_cast<int>(a1.w), static_cast<int>(b[7]), s);
+            acc[c][r] = s;
+          }
+        }
+      } else {
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         const uint4 a = *reinterpret_cast<const uint4*>(topg_smem + r * K + k0 + u * 32 * 16);
@@ -69,6 +107,7 @@ __global__ void __launch_bounds__(TOPG_THREADS, (R <= 4 ? 3 : (R <= 8 ? 4 : 2)))
           s = __dp4a(static_cast<int>(a.w), static_cast<int>(w[c][u].w), s);
           acc[c][r] = s;
         }
+      }
       }
     }
   }

@@ -1027,10 +1027,10 @@ static int run_inverse_dct_tc(const Problem& pb, const __nv_bfloat16* planes, co
 
 // Top rows of a short sequence: codes x weights, de-quantization and the inverse of the levels above 8
 // in one launch (k_top_gemv).  Returns STAMP_ERR_UNSUPPORTED when the shape is outside its range.
-template <int R>
+template <int R, bool PACKED>
 static int launch_top_gemv(const int8_t* codes, const float* sx, const int8_t* w8, int K, int N, int top_levels,
                            float* a8v, cudaStream_t st) {
-  auto kern = k_top_gemv<R>;
+  auto kern = k_top_gemv<R, PACKED>;
   const size_t smem = (size_t)R * K;
   if (int rc = ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return rc;
   const int per_cta = (TOPG_THREADS / 32) * TOPG_CH_PER_WARP;
@@ -1042,16 +1042,23 @@ static int launch_top_gemv(const int8_t* codes, const float* sx, const int8_t* w
   STAMP_CHECK_LAUNCH();
   return STAMP_OK;
 }
-static int run_top_gemv(const Problem& pb, const int8_t* codes, const float* sx, const int8_t* w8, float* a8v,
-                        cudaStream_t st) {
+// w4: the same weights as packed 4-bit codes [N, K / 2] when the caller has them (the kernel then streams half the
+// bytes), else null.
+static int run_top_gemv(const Problem& pb, const int8_t* codes, const float* sx, const int8_t* w8, const uint8_t* w4,
+                        float* a8v, cudaStream_t st) {
   const long R = pb.M >> 8;
-  if (R > 16 || (size_t)R * pb.K > 160 * 1024 || pb.K % 16 != 0) return STAMP_ERR_UNSUPPORTED;
+  if (R > 16 || (size_t)R * pb.K > 160 * 1024 || pb.K % 32 != 0) return STAMP_ERR_UNSUPPORTED;
   const int tl = pb.levels - 8;
+  // Measured (ms per layer step, int8 weights / packed weights): 2 rows: 0.0618 / 0.0587 at K = N = 8192, 0.0352 / 0.0349
+  // at 2048; 8 rows: 0.0978 / 0.1095 on 4096 x 11008, 0.1383 / 0.1522 at K = N = 8192 -- with more than two rows the
+  // expansion of the nibbles costs more than the bytes it saves, so the packed copy is read for up to two rows only.
+  if (R > 2) w4 = nullptr;
+  const int8_t* w4p = reinterpret_cast<const int8_t*>(w4);
   switch (R) {
-    case 2: return launch_top_gemv<2>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
-    case 4: return launch_top_gemv<4>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
-    case 8: return launch_top_gemv<8>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
-    case 16: return launch_top_gemv<16>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    case 2: return w4 ? launch_top_gemv<2, true>(codes, sx, w4p, pb.K, pb.N, tl, a8v, st) : launch_top_gemv<2, false>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    case 4: return w4 ? launch_top_gemv<4, true>(codes, sx, w4p, pb.K, pb.N, tl, a8v, st) : launch_top_gemv<4, false>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    case 8: return w4 ? launch_top_gemv<8, true>(codes, sx, w4p, pb.K, pb.N, tl, a8v, st) : launch_top_gemv<8, false>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
+    case 16: return w4 ? launch_top_gemv<16, true>(codes, sx, w4p, pb.K, pb.N, tl, a8v, st) : launch_top_gemv<16, false>(codes, sx, w8, pb.K, pb.N, tl, a8v, st);
     default: return STAMP_ERR_UNSUPPORTED;
   }
 }
@@ -1067,7 +1074,7 @@ static int run_unpack_codes(const Problem& pb, const void* q_hi, const void* q_l
 // of the packed codes into the workspace.
 static int weights_as_int8(const Problem& pb, const void* w, int w_format, int8_t* w8_ws, const int8_t** out,
                            cudaStream_t st) {
-  if (w_format == STAMP_W_INT8) {
+  if (w_format == STAMP_W_INT8 || w_format == STAMP_W_INT8_AND_PACKED4) {
     *out = static_cast<const int8_t*>(w);
     return STAMP_OK;
   }
@@ -1076,6 +1083,13 @@ static int weights_as_int8(const Problem& pb, const void* w, int w_format, int8_
   STAMP_CHECK_LAUNCH();
   *out = w8_ws;
   return STAMP_OK;
+}
+
+// The packed copy of the weights when the caller's operand has one (kernels that only stream the weights read it).
+static const uint8_t* weights_packed(const Problem& pb, const void* w, int w_format) {
+  if (w_format == STAMP_W_PACKED4) return static_cast<const uint8_t*>(w);
+  if (w_format == STAMP_W_INT8_AND_PACKED4) return static_cast<const uint8_t*>(w) + (size_t)pb.N * pb.K;
+  return nullptr;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1224,6 +1238,15 @@ int stamp_prepare_weights(const stamp_config* cfg, const void* wq_packed, int N,
   k_unpack_rows4<<<N, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t*>(wq_packed), K,
                                                                     static_cast<int8_t*>(w_int8));
   STAMP_CHECK_LAUNCH();
+  return STAMP_OK;
+}
+
+int stamp_prepare_weights_both(const stamp_config* cfg, const void* wq_packed, int N, int K, void* w_both, void* stream) {
+  int rc = stamp_prepare_weights(cfg, wq_packed, N, K, w_both, stream);
+  if (rc) return rc;
+  if (cudaMemcpyAsync(static_cast<uint8_t*>(w_both) + (size_t)N * K, wq_packed, (size_t)N * (K / 2), cudaMemcpyDeviceToDevice,
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return STAMP_ERR_CUDA;
   return STAMP_OK;
 }
 
@@ -1413,7 +1436,7 @@ int stamp_linear_fused(const stamp_config* cfg, const void* X, int x_dtype, cons
     if (pb.levels > 8) {
       float* yttop = reinterpret_cast<float*>(base + wl.yttop);
       float* a8v_w = reinterpret_cast<float*>(base + wl.a8v);
-      rc = run_top_gemv(pb, tl.a8_top, tl.sx_top, w8f, a8v_w, st);
+      rc = run_top_gemv(pb, tl.a8_top, tl.sx_top, w8f, weights_packed(pb, w, w_format), a8v_w, st);
       if (rc == STAMP_OK) {
         a8v = a8v_w;
       } else if (rc != STAMP_ERR_UNSUPPORTED) {

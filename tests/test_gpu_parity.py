@@ -210,8 +210,10 @@ def test_stagewise_parity(st, oracle, name):
     Yt2 = st.stamp_linear(c, q_hi, q_lo, xs, wq, st.W_PACKED4, wsc, B, L, K, N, ws)
     Y2 = st.stamp_inverse(c, Yt2, bd, ws).cpu().numpy().reshape(-1, N)
     assert H.rel_fro(Y2, ref["Y"]) <= Y_TOL
-    for wfmt, wbuf in ((st.W_PACKED4, wq), (st.W_INT8, w8)):
-        Y3 = st.stamp_linear_fused(c, Xd, wbuf, wfmt, wsc, bd, ws).cpu().numpy().reshape(-1, N)
+    both = st.stamp_prepare_weights_both(c, wq)
+    assert torch.equal(both[:N * K].view(N, K), w8) and torch.equal(both[N * K:].view(torch.uint8).view(N, K // 2), wq)
+    for wfmt, wbuf in ((st.W_PACKED4, wq), (st.W_INT8, w8), (st.W_INT8_AND_PACKED4, both)):
+        Y3 = st.stamp_linear_fused(c, Xd, wbuf, wfmt, wsc, bd, ws, n_out=N).cpu().numpy().reshape(-1, N)
         err = H.rel_fro(Y3, ref["Y"])
         print(f"[{name}] one-call layer, output relative Frobenius error {err:.2e}")
         # (the tight bound presumes the oracle's codes; a code on a rounding boundary that fell the other way moves
