@@ -1,5 +1,6 @@
 // Fused Haar transform + per-token mixed-precision quantizer for bf16 activations, one pass over X in HBM
-// (Algorithm lines "X <- L X" and "x_i <- Q(x_i; b_i)"; Sec. "Efficient Energy Concentration").
+// (Algorithm 1: the sequence transform of the activations and their per-token quantizer; Sec. "Efficient Energy
+// Concentration").
 //
 // Why this shape.  The quantizer needs, per transformed token, the maximum over ALL channels before it can
 // code any of them, while a Haar coefficient needs a run of tokens of ONE channel.  On the CUDA cores alone the
@@ -15,20 +16,23 @@
 //     is simply issued again when they are back -- 4 us of tensor time per GB of activations, on a pipe that has
 //     nothing else to do in this pass -- so that no warp parks a coefficient in registers across the exchange
 //     and the ring of six tiles, not the register file, sets how many tiles can be waiting.  Tensor memory
-//     (lane = transformed token, column = channel) only holds the four accumulators in flight.
+//     (lane = transformed token, column = channel) only holds the accumulators in flight.
 // An epilogue thread owns ONE transformed token of the tile: its maximum over the tile's channels is a
 // thread-local reduction, and later its scale, bit width and destination row are per-thread constants.  What
 // is left for the CUDA cores is about 5 instructions per element.
 //
 // Row maxima across the feature axis.  A tile covers 128 channels; the K / 128 tiles of a 128-token row block
 // are consecutive work items, taken at about the same time by neighbouring CTAs of the persistent grid.
-//   job P1(item): product -> the epilogue warps reduce |D| per lane over the tile's columns and combine the
-//                 result into the row block's table in global memory (atomicMax), then count themselves in;
+//   job P1(item): product -> four warps of their own (one per quarter of the accumulator's lanes) reduce |D| per
+//                 lane over the tile's 128 columns and leave the 128 maxima in shared memory; a publisher warp
+//                 combines them into the row block's table in global memory (atomicMax) and, once they are
+//                 delivered, counts the tile in (two publishers alternate);
 //   job P2(item): HTC_LAG items later the MMA thread waits (bounded) until the row block's count is complete,
-//                 issues the product again, and the epilogue warps read the final maxima, derive scale, bit
-//                 width and destination of their row, quantize the accumulator and store the codes.
-// Sending the maxima and counting the tile in is the job of two publisher warps: the fence between the two
-// waits about a microsecond for the atomics to be delivered, which an epilogue warp cannot afford.  A CTA only ever waits for P1 jobs of items that
+//                 issues the product again into the accumulator of one of three sets of quantizing warps, and
+//                 these read the final maxima, derive scale, bit width and destination of their row, quantize
+//                 and store the codes.
+// The warps that take the maxima do nothing else, so a tile's maxima leave the SM a few hundred clocks after its
+// first product and never queue behind a quantizing pass.  A CTA only ever waits for P1 jobs of items that
 // precede or accompany its own in the global item order, and a P1 job needs nothing but a ring stage and an
 // accumulator freed by jobs further back, so the waits cannot form a cycle as long as every CTA of the grid is
 // resident (one CTA per SM, grid <= number of SMs) and a row block has no more tiles than the grid has CTAs.
@@ -39,12 +43,14 @@
 #include "common.cuh"
 #include "k_haar_cq.cuh"
 #include "ptx.cuh"
+#include <type_traits>
 
 namespace stamp {
 
 struct HtcParams {
   int K;             // channels, a multiple of 128
-  int n;             // tokens per transform block (power of two)
+  int n;             // tokens per transform block, a multiple of 128
+  int n_shift;       // log2 n when n is a power of two, else -1
   int lv;            // Haar levels applied here, 1..7 (2^lv <= n)
   int last;          // 1: lv is the transform's depth, the approximation rows are quantized here
                      // 0: (lv == 7) the 128-token sums go to aout, un-normalised, for the next launch
@@ -67,17 +73,20 @@ struct HtcParams {
 
 enum HtcOut { HTC_OUT_A8 = 0, HTC_OUT_PUBLIC = 1, HTC_OUT_T = 2, HTC_OUT_TILED = 3 };
 
-constexpr int HTC_THREADS = 20 * 32;       // TMA warp, MMA warp, two sets of eight epilogue warps, two publisher warps
+// warps: 0 TMA producer, 1 MMA issuer, 2-3 publishers, 4-27 three sets of eight quantizing warps, 28-31 maxima
+constexpr int HTC_THREADS = 32 * 32;
+constexpr int HTC_QSETS = 3;
 constexpr int HTC_STAGES = 6;              // shared-memory ring of activation tiles
-constexpr int HTC_LAG = 4;                 // items between the two products of a tile (even: both jobs go to one warp set)
-constexpr int HTC_NBUF = 4;                // 128-column accumulators in tensor memory
+constexpr int HTC_LAG = 3;                 // items between the two products of a tile (< HTC_STAGES)
+constexpr int HTC_NBUF = 4;                // 128-column accumulators in tensor memory: one for P1 jobs, one per quantizing set
 constexpr int HTC_TILE_BYTES = 128 * 128 * 2;   // [128 tokens x 128 channels] bf16 = two 64-channel atoms
 constexpr int HTC_ATOM_BYTES = 128 * 128;       // [128 tokens x 64 channels] bf16
 constexpr int HTC_A_BYTES = 128 * 128 * 2;      // H: [128 rows x 128 tokens] bf16 = two 64-token atoms
 constexpr int HTC_BAR_OFFSET = HTC_A_BYTES + HTC_STAGES * HTC_TILE_BYTES;
-constexpr int HTC_NUM_BARS = 2 * HTC_STAGES + 2 * HTC_NBUF + 4;   // + pfull[2], pempty[2]
+constexpr int HTC_NUM_BARS = 2 * HTC_STAGES + 2 * HTC_NBUF + 4;   // ring, accumulators (full / empty), pfull[2], pempty[2]
 constexpr int HTC_SLOT_OFFSET = HTC_BAR_OFFSET + HTC_NUM_BARS * 8 + 16;   // [2 sets][128 lanes] maxima on their way out
 constexpr int HTC_DYN_BYTES = HTC_SLOT_OFFSET + 2 * 128 * 4 + 1024;
+constexpr uint32_t HTC_NIB_BIAS = 0x3F400000u;     // sum over i < 8 of 0x4B400000 << 4 i, modulo 2^32 (see the 4-bit packing)
 constexpr long long HTC_WAIT_LIMIT = 4000000000LL;   // SM clocks (~2 s) before a wait gives up
 
 // bf16 A (K-major) x bf16 B (MN-major) -> fp32, M = 128, N = 128
@@ -150,8 +159,10 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const long nitems = p.ntiles * p.nchunks;
-  const long n_local = nitems > blockIdx.x ? (nitems - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;   // this CTA's items
+  // item numbers fit 32 bits (checked by the host): the per-tile index arithmetic below is 32-bit on purpose
+  const unsigned nitems = static_cast<unsigned>(p.ntiles) * static_cast<unsigned>(p.nchunks);
+  const int n_local = nitems > blockIdx.x ? static_cast<int>((nitems - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;   // this CTA's items
+  const unsigned nchunks = static_cast<unsigned>(p.nchunks);
 
   // ---- the analysis matrix, written straight into the K-major 128-byte-swizzled operand layout:
   // element (row r, token t) of atom t / 64 sits in 16-byte chunk ((t % 64) / 8) ^ (r % 8) of row r
@@ -177,7 +188,6 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     const int atom = c16 >> 3, chunk = (c16 & 7) ^ (r & 7);
     *reinterpret_cast<uint4*>(a_sm + atom * HTC_ATOM_BYTES + r * 128 + chunk * 16) = make_uint4(w[0], w[1], w[2], w[3]);
   }
-  if (threadIdx.x < 256) pslot[threadIdx.x] = 0u;
   if (threadIdx.x == 0) {
     for (int s = 0; s < HTC_STAGES; ++s) {
       ptx::mbar_init(&sfull[s], 1);
@@ -185,10 +195,10 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     }
     for (int b = 0; b < HTC_NBUF; ++b) {
       ptx::mbar_init(&tfull[b], 1);
-      ptx::mbar_init(&tempty[b], 8 * 32);   // the eight warps of the set that drains the accumulator
+      ptx::mbar_init(&tempty[b], b == 0 ? 4 * 32 : 8 * 32);   // the four maxima warps / the eight warps of a quantizing set
     }
     for (int q = 0; q < 2; ++q) {
-      ptx::mbar_init(&pfull[q], 8 * 32);
+      ptx::mbar_init(&pfull[q], 4 * 32);
       ptx::mbar_init(&pempty[q], 32);
     }
     *abort_word = 0;
@@ -222,17 +232,17 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
       uint32_t phase = 0;
       uint32_t armed = 0, armed_parity = 0;
       bool ok = true;
-      for (long item = blockIdx.x; item < nitems; item += gridDim.x) {
-        const long rb = item / p.nchunks;
-        const int c = static_cast<int>(item - rb * p.nchunks);
+      for (unsigned item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const unsigned rb = item / nchunks;
+        const int c = static_cast<int>(item - rb * nchunks);
         if (!ptx::mbar_wait_bounded_sleepy(&sempty[stage], phase ^ 1u, abort_word, HTC_WAIT_LIMIT)) {
           ok = false;
           break;
         }
         uint8_t* dst = b_sm + stage * HTC_TILE_BYTES;
         ptx::mbar_arrive_expect_tx(&sfull[stage], HTC_TILE_BYTES);
-        ptx::tma_load_2d(dst, &tmap_x, &sfull[stage], c * 128, static_cast<int>(rb * 128));
-        ptx::tma_load_2d(dst + HTC_ATOM_BYTES, &tmap_x, &sfull[stage], c * 128 + 64, static_cast<int>(rb * 128));
+        ptx::tma_load_2d(dst, &tmap_x, &sfull[stage], c * 128, static_cast<int>(rb * 128u));
+        ptx::tma_load_2d(dst + HTC_ATOM_BYTES, &tmap_x, &sfull[stage], c * 128 + 64, static_cast<int>(rb * 128u));
         armed |= 1u << stage;
         armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
         if (++stage == HTC_STAGES) {
@@ -253,17 +263,15 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
+    // Static order: P1 of item t, then P2 of item t - HTC_LAG.  Accumulator 0 for a P1 job, 1 + i % 3 for the P2
+    // job of item i (the quantizing set i % 3 drains it).
     if (ptx::elect_one()) {
       bool ok = true;
       const uint32_t abase = ptx::smem_u32(a_sm);
-      const unsigned target = static_cast<unsigned>(p.nchunks);
-      long job = 0;
-      // D = H X of the tile in ring stage `stage` into the accumulator of job `job`; the last product of a tile
-      // also hands the stage back to the producer
-      auto product = [&](int stage, bool release_stage) -> bool {
-        const int buf = static_cast<int>(job & (HTC_NBUF - 1));
-        if (!ptx::mbar_wait_bounded_sleepy(&tempty[buf], static_cast<uint32_t>(((job / HTC_NBUF) & 1) ^ 1), abort_word, HTC_WAIT_LIMIT))
-          return false;
+      // D = H X of the tile in ring stage `stage` into accumulator `buf`, whose `use`-th filling this is; the
+      // second product of a tile also hands the stage back to the producer
+      auto product = [&](int stage, int buf, int use, bool release_stage) -> bool {
+        if (!ptx::mbar_wait_bounded_sleepy(&tempty[buf], static_cast<uint32_t>((use & 1) ^ 1), abort_word, HTC_WAIT_LIMIT)) return false;
         ptx::tc_fence_after();
         const uint32_t bbase = ptx::smem_u32(b_sm + stage * HTC_TILE_BYTES);
         const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * 128);
@@ -275,31 +283,30 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
         }
         if (release_stage) ptx::tc_commit(&sempty[stage]);
         ptx::tc_commit(&tfull[buf]);
-        ++job;
         return true;
       };
-      for (long t = 0; t < n_local + HTC_LAG && ok; ++t) {
+      for (int t = 0; t < n_local + HTC_LAG && ok; ++t) {
         if (t < n_local) {   // P1 of item t
-          const int stage = static_cast<int>(t % HTC_STAGES);
+          const int stage = t % HTC_STAGES;
           if (!ptx::mbar_wait_bounded_sleepy(&sfull[stage], static_cast<uint32_t>((t / HTC_STAGES) & 1), abort_word, HTC_WAIT_LIMIT) ||
-              !product(stage, false)) {
+              !product(stage, 0, t, false)) {
             ok = false;
             break;
           }
         }
         if (t >= HTC_LAG) {  // P2 of item t - HTC_LAG: its row block's maxima must be complete
-          const long i = t - HTC_LAG;
-          const long rb = (blockIdx.x + i * gridDim.x) / p.nchunks;
+          const int i = t - HTC_LAG;
+          const unsigned rb = (blockIdx.x + static_cast<unsigned>(i) * gridDim.x) / nchunks;
           const long long t0 = clock64();
           unsigned spins = 0;
-          while (ld_acquire_gpu(p.cnt + rb) < target) {
+          while (ld_acquire_gpu(p.cnt + rb) < nchunks) {
             if ((++spins & 15u) == 0u && (*abort_word != 0u || clock64() - t0 > HTC_WAIT_LIMIT)) {
               ok = false;
               break;
             }
             __nanosleep(20);
           }
-          if (!ok || !product(static_cast<int>(i % HTC_STAGES), true)) {
+          if (!ok || !product(i % HTC_STAGES, 1 + i % HTC_QSETS, i / HTC_QSETS, true)) {
             ok = false;
             break;
           }
@@ -310,44 +317,83 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
         raise_device_status(STAMP_ERR_TIMEOUT);
       }
     }
-  } else if (warp >= 18) {
-    // ------------------------------------------------------------------ publisher warps (one per epilogue set)
-    // Takes the lane maxima a set has gathered for a tile out of shared memory, sends them to the row block's
-    // table and, once they are delivered (the fence), counts the tile in.  The wait for the delivery -- about a
-    // microsecond under load -- is all this warp does, so it stalls nobody.
-    const int set = warp - 18;
+  } else if (warp < 4) {
+    // ------------------------------------------------------------------ publisher warps (items of one parity each)
+    // Takes a tile's 128 lane maxima out of shared memory, sends them to the row block's table and, once they
+    // are delivered, counts the tile in.
+    const int set = warp - 2;
     bool ok = true;
-    long k = 0;
-    for (long i = set; i < n_local; i += 2, ++k) {
-      const long rb = (blockIdx.x + i * gridDim.x) / p.nchunks;
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&pfull[set], static_cast<uint32_t>(k & 1), abort_word, HTC_WAIT_LIMIT))) {
+    for (int i = set; i < n_local; i += 2) {
+      const unsigned rb = (blockIdx.x + static_cast<unsigned>(i) * gridDim.x) / nchunks;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&pfull[set], static_cast<uint32_t>((i >> 1) & 1), abort_word, HTC_WAIT_LIMIT))) {
         ok = false;
         break;
       }
       unsigned m[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        m[q] = pslot[set * 128 + q * 32 + lane];
-        pslot[set * 128 + q * 32 + lane] = 0u;
-      }
-      ptx::mbar_arrive(&pempty[set]);      // the slot is clear again
+      for (int q = 0; q < 4; ++q) m[q] = pslot[set * 128 + q * 32 + lane];
+      ptx::mbar_arrive(&pempty[set]);      // the slot may be written again
 #pragma unroll
-      for (int q = 0; q < 4; ++q) atomicMax(p.rowmax + rb * 128 + q * 32 + lane, m[q]);
-      __threadfence();
+      for (int q = 0; q < 4; ++q) atomicMax(p.rowmax + (size_t)rb * 128 + q * 32 + lane, m[q]);
+      // Counting the tile in is a release at GPU scope: whoever reads the complete count with an acquire load also
+      // sees the maxima (the other lanes' atomics are ordered before lane 0's release by the warp barrier).  The
+      // release costs less than a full fence between the atomics and a relaxed count (164 against 168 us on
+      // 32768 x 8192 tokens x channels).
       __syncwarp();
-      if (lane == 0) atomicAdd(p.cnt + rb, 1u);
+      if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt + rb) : "memory");
+    }
+    if (!ok) {
+      *abort_word = 1;
+      raise_device_status(STAMP_ERR_TIMEOUT);
+    }
+  } else if (warp >= 28) {
+    // ------------------------------------------------------------------ maxima warps: one per quarter of the lanes
+    // P1 of every item: |D| of this thread's lane over the tile's 128 columns, left in the slot of the item's
+    // parity for the publisher.  The accumulator is released as soon as its values are in registers.
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;
+    bool ok = true;
+    for (int i = 0; i < n_local; ++i) {
+      const int slot = i & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&tfull[0], static_cast<uint32_t>(i & 1), abort_word, HTC_WAIT_LIMIT))) {
+        ok = false;
+        break;
+      }
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+      uint32_t v[2][16];
+      float m0 = 0.f, m1 = 0.f;
+      ptx::tmem_ld_32x32b_x16(taddr, v[0]);
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        ptx::tmem_ld_wait();
+        if (ch < 7) ptx::tmem_ld_32x32b_x16(taddr + 16 * (ch + 1), v[(ch + 1) & 1]);
+        const uint32_t(&x)[16] = v[ch & 1];
+#pragma unroll
+        for (int q = 0; q < 16; q += 2) {
+          m0 = fmaxf(m0, fabsf(__uint_as_float(x[q])));
+          m1 = fmaxf(m1, fabsf(__uint_as_float(x[q + 1])));
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&tempty[0]);
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&pempty[slot], static_cast<uint32_t>(((i >> 1) & 1) ^ 1), abort_word, HTC_WAIT_LIMIT))) {
+        ok = false;
+        break;
+      }
+      pslot[slot * 128 + r] = __float_as_uint(fmaxf(m0, m1));
+      ptx::mbar_arrive(&pfull[slot]);
     }
     if (!ok) {
       *abort_word = 1;
       raise_device_status(STAMP_ERR_TIMEOUT);
     }
   } else {
-    // ------------------------------------------------------------------ epilogue warps
-    // Two sets of eight warps take the CTA's items alternately (both jobs of an item go to the same set); inside
-    // a set a warp owns the 32 lanes of its quarter (warp % 4) and 64 of the tile's 128 columns.  A warp's jobs
-    // alternate: P1 of item i (lane maxima of its columns, handed to the set's publisher warp), then P2 of item
-    // i - HTC_LAG (scale, codes, stores) -- each waits for the accumulator the MMA thread fills for it.
-    const int e = warp - 2;
+    // ------------------------------------------------------------------ quantizing warps
+    // Three sets of eight warps take the CTA's items in turn; inside a set a warp owns the 32 lanes of its
+    // quarter (warp % 4) and 64 of the tile's 128 columns, a thread ONE transformed token: scale, bit width and
+    // destination row are per-thread scalars, and a thread's 64 codes are 32 or 64 contiguous bytes of its row.
+    const int e = warp - 4;
     const int set = e >> 3;
     const int quarter = warp & 3;
     const int half = (e >> 2) & 1;
@@ -357,178 +403,203 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     htc_lane_row(p.lv, r, j, idx, approx);
     const bool raw = approx && !p.last;        // the 128-token sum: handed on un-normalised
     const bool odd = (j & 1) != 0;
+    const bool warp_has_odd = __any_sync(0xffffffffu, odd);   // false: no lane of the warp needs the 1/sqrt 2 factor
     const float pw = __int_as_float((127 - (j >> 1)) << 23);      // 2^(-(j >> 1))
     const float2 nhi = odd ? make_float2(CQ_RSQRT2_HI, CQ_RSQRT2_HI) : make_float2(1.f, 1.f);
     const float2 nlo = odd ? make_float2(CQ_RSQRT2_LO, CQ_RSQRT2_LO) : make_float2(0.f, 0.f);
-    const int K = p.K;
-    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(half * 64);
+    const unsigned K = static_cast<unsigned>(p.K);
+    const unsigned n = static_cast<unsigned>(p.n);
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>((1 + set) * 128 + half * 64);
     bool ok = true;
+    // (row block, tile inside it) of the set's items, advanced without a division per item
+    const unsigned item0 = blockIdx.x + static_cast<unsigned>(set) * gridDim.x;
+    unsigned rb = item0 / nchunks;
+    unsigned cu = item0 - rb * nchunks;
+    const unsigned step_rb = (HTC_QSETS * gridDim.x) / nchunks, step_c = HTC_QSETS * gridDim.x - step_rb * nchunks;
 
-    // job index of the two products of local item i in the MMA thread's issue order
-    auto job_p1 = [&](long i) -> long { return i + (i > HTC_LAG ? i - HTC_LAG : 0); };
-    auto job_p2 = [&](long i) -> long { return i + HTC_LAG < n_local ? 2 * i + HTC_LAG + 1 : n_local + i; };
-    auto wait_acc = [&](long jb) -> bool {
-      const int buf = static_cast<int>(jb & (HTC_NBUF - 1));
-      const bool got = __all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&tfull[buf], static_cast<uint32_t>((jb / HTC_NBUF) & 1),
-                                                                      abort_word, HTC_WAIT_LIMIT));
-      ptx::tc_fence_after();
-      return got;
-    };
-
-    // P2 of local item i
-    auto pass2 = [&](long i) -> bool {
-      const long item = blockIdx.x + i * gridDim.x;
-      const long rb = item / p.nchunks;
-      const int c = static_cast<int>(item - rb * p.nchunks);
-      const long jb = job_p2(i);
-      const int buf = static_cast<int>(jb & (HTC_NBUF - 1));
-      // where this lane's row goes (all per-thread scalars; the tile's tokens are [128 rb, 128 rb + 128))
-      const long tok0 = rb * 128;
-      const long blk = tok0 / p.n;
-      const int off = static_cast<int>(tok0 - blk * p.n);
-      const int ib = (off >> j) + idx;                          // index inside the block at level j
-      const int i_in_blk = approx ? ib : (p.n >> j) + ib;        // logical row inside the block
-      const bool hi = i_in_blk < p.k_hi;
+    for (int i = set; i < n_local && ok; i += HTC_QSETS, rb += step_rb, cu += step_c) {
+      if (cu >= nchunks) {
+        cu -= nchunks;
+        ++rb;
+      }
+      // where this lane's row goes (the tile's tokens are [128 rb, 128 rb + 128)); rows and row pitches fit 32 bits
+      const unsigned tok0 = rb * 128u;
+      const unsigned blk = p.n_shift >= 0 ? tok0 >> p.n_shift : tok0 / n;
+      const unsigned off = tok0 - blk * n;
+      const unsigned ib = (off >> j) + idx;                         // index inside the block at level j
+      const unsigned i_in_blk = approx ? ib : (n >> j) + ib;        // logical row inside the block
+      const bool hi = i_in_blk < static_cast<unsigned>(p.k_hi);
       const float qmax = hi ? p.qmax_hi : p.qmax_lo;
+      const unsigned row = blk * n + i_in_blk;
+      const unsigned col0 = cu * 128u + half * 64u;
+      uint8_t* dst = nullptr;       // this lane's 64 channels of its row
+      bool four_bit = false;
+      size_t scale_at = 0;          // where this lane reports its scale (one lane of the row block's first tile)
+      float* scale_to = p.x_scale;
+      if (raw) {
+        dst = reinterpret_cast<uint8_t*>(p.aout) + ((size_t)rb * K + col0) * 4;
+      } else if (OUT == HTC_OUT_T) {
+        dst = reinterpret_cast<uint8_t*>(p.T_out) + ((size_t)row * K + col0) * 4;
+      } else if (OUT == HTC_OUT_PUBLIC) {
+        if (hi) {
+          dst = reinterpret_cast<uint8_t*>(p.q_hi) + (size_t)(blk * p.k_hi + i_in_blk) * K + col0;
+        } else {
+          dst = p.q_lo + (size_t)(blk * (n - p.k_hi) + (i_in_blk - p.k_hi)) * (K >> 1) + (col0 >> 1);
+          four_bit = true;
+        }
+        scale_at = row;
+      } else if (OUT == HTC_OUT_A8) {
+        dst = reinterpret_cast<uint8_t*>(p.a8) + (size_t)row * K + col0;
+        scale_at = row;
+      } else {
+        // tile order of the GEMM's fused inverse (see k_haar_cq.cuh): 256-token tiles
+        const unsigned tile = (blk * n + (ib << j)) >> 8;
+        const int i_loc = static_cast<int>(ib & ((256u >> j) - 1u));
+        const int tcol = approx ? 32 * i_loc : cq_tile_col_detail(j, i_loc);
+        const unsigned prow = tile * 256u + tcol;
+        dst = reinterpret_cast<uint8_t*>(p.a8) + (size_t)prow * K + col0;
+        scale_at = prow;
+        scale_to = p.sx_epi;
+      }
+      // a warp whose 32 rows all take 4-bit codes (the common case) packs nibbles only
+      const bool all_four = __all_sync(0xffffffffu, four_bit && !raw);
       // the MMA thread issued this product after it saw the row block's count complete: the table is final
-      if (!wait_acc(jb)) return false;
-      const float u = __uint_as_float(ld_relaxed_gpu(p.rowmax + rb * 128 + r));
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&tfull[1 + set], static_cast<uint32_t>((i / HTC_QSETS) & 1), abort_word, HTC_WAIT_LIMIT))) {
+        ok = false;
+        break;
+      }
+      ptx::tc_fence_after();
+      uint32_t v[2][16];
+      ptx::tmem_ld_32x32b_x16(taddr, v[0]);
+      const float u = __uint_as_float(ld_relaxed_gpu(p.rowmax + (size_t)rb * 128 + r));
       const float amax = odd ? fmaf(u, CQ_RSQRT2_HI, u * CQ_RSQRT2_LO) : u;      // in units of 2^(-(j >> 1))
       const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
       const float inv = __fdiv_rn(1.0f, scale);
       const float true_scale = (amax > 0.f) ? scale * pw : 1.0f;
       const float2 inv2 = make_float2(inv, inv), ns2 = make_float2(-scale, -scale);
-      const long row = blk * p.n + i_in_blk;
-      const int col0 = c * 128 + half * 64;
-      uint8_t* dst = nullptr;       // this lane's 64 channels of its row
-      bool four_bit = false;
-      if (raw) {
-        dst = reinterpret_cast<uint8_t*>(p.aout + rb * (long)K + col0);
-      } else if (OUT == HTC_OUT_T) {
-        dst = reinterpret_cast<uint8_t*>(p.T_out + row * (long)K + col0);
-      } else if (OUT == HTC_OUT_PUBLIC) {
-        if (hi) {
-          dst = reinterpret_cast<uint8_t*>(p.q_hi + (blk * p.k_hi + i_in_blk) * (long)K + col0);
-        } else {
-          dst = p.q_lo + (blk * (p.n - p.k_hi) + (i_in_blk - p.k_hi)) * (long)(K >> 1) + (col0 >> 1);
-          four_bit = true;
+      // Rounding by adding 1.5 * 2^23: the sum's low mantissa bits are the two's complement code.  A 4-bit row adds 8
+      // more, so that its low nibble is the code + 8 in [1, 15] and nothing above it changes: eight such words
+      // combine into eight nibbles with shifts and adds alone, and one XOR takes the 8 out of every nibble again.
+      const float magic = four_bit ? CQ_MAGIC + 8.0f : CQ_MAGIC;
+      const float2 magic2 = make_float2(magic, magic);
+      if (cu == 0 && half == 0 && !raw && OUT != HTC_OUT_T)
+        scale_to[scale_at] = (OUT == HTC_OUT_TILED) ? true_scale * (odd ? pw * CQ_RSQRT2_HI : pw) : true_scale;
+
+      // One chunk of 16 columns: x -> 16 codes (or values).  Codes collect in `pend` until they fill a 32-byte
+      // sector of the row (64 four-bit codes: the whole pass; 32 eight-bit codes: two chunks), which then leaves
+      // in one store: a warp's store touches 32 different rows, so the fewer pieces per row the better.
+      // MIXED: the warp's rows differ in kind (raw sum, 8-bit, 4-bit).  Every lane then runs the same
+      // instructions -- both packings, selected per lane, and predicated stores -- instead of the kinds taking
+      // turns through the whole chunk.
+      uint32_t pend[8];
+      auto chunk = [&](const uint32_t(&x)[16], auto ch_tag, auto norm_tag, auto mixed_tag) {
+        constexpr int ch = decltype(ch_tag)::value;
+        constexpr bool NORM = decltype(norm_tag)::value;
+        constexpr bool MIXED = decltype(mixed_tag)::value;
+        if (MIXED && raw) {
+          ptx::st_global_v8(dst + ch * 64, x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
+          ptx::st_global_v8(dst + ch * 64 + 32, x[8], x[9], x[10], x[11], x[12], x[13], x[14], x[15]);
         }
-        if (c == 0 && half == 0) p.x_scale[row] = true_scale;
-      } else if (OUT == HTC_OUT_A8) {
-        dst = reinterpret_cast<uint8_t*>(p.a8 + row * (long)K + col0);
-        if (c == 0 && half == 0) p.x_scale[row] = true_scale;
-      } else {
-        // tile order of the GEMM's fused inverse (see k_haar_cq.cuh): 256-token tiles
-        const long tile = (blk * p.n + ((long)ib << j)) >> 8;
-        const int i_loc = ib & ((256 >> j) - 1);
-        const int tcol = approx ? 32 * i_loc : cq_tile_col_detail(j, i_loc);
-        const long prow = tile * 256 + tcol;
-        dst = reinterpret_cast<uint8_t*>(p.a8 + prow * (long)K + col0);
-        if (c == 0 && half == 0) p.sx_epi[prow] = true_scale * (odd ? pw * CQ_RSQRT2_HI : pw);
-      }
-      const uint32_t taddr = lane_base + static_cast<uint32_t>(buf * 128);
-      uint32_t v[2][32];
-      ptx::tmem_ld_32x32b_x32(taddr, v[0]);
-#pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        ptx::tmem_ld_wait();
-        if (ch == 0) ptx::tmem_ld_32x32b_x32(taddr + 32, v[1]);
-        const uint32_t(&x)[32] = v[ch];
-        if (raw) {
-          float4* o = reinterpret_cast<float4*>(dst) + ch * 8;
-#pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4)
-            o[q4] = make_float4(__uint_as_float(x[4 * q4]), __uint_as_float(x[4 * q4 + 1]), __uint_as_float(x[4 * q4 + 2]),
-                                __uint_as_float(x[4 * q4 + 3]));
-          continue;
-        }
-        uint32_t w[8];
+        uint32_t bits[16];
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
-          uint32_t bits[4];
+          const float2 raw2 = make_float2(__uint_as_float(x[2 * g]), __uint_as_float(x[2 * g + 1]));
+          // 2^(-j/2) = c * 2^(-(j >> 1)): only c touches the data, head + tail so the product is rounded once
+          const float2 t = NORM ? __ffma2_rn(raw2, nhi, __fmul2_rn(raw2, nlo)) : raw2;
+          if (OUT == HTC_OUT_T) {
+            bits[2 * g] = __float_as_uint(t.x * pw);
+            bits[2 * g + 1] = __float_as_uint(t.y * pw);
+          } else {
+            const float2 q0 = __fmul2_rn(t, inv2);
+            const float2 rem = __ffma2_rn(q0, ns2, t);
+            const float2 q = __fadd2_rn(__ffma2_rn(rem, inv2, q0), magic2);
+            bits[2 * g] = __float_as_uint(q.x);
+            bits[2 * g + 1] = __float_as_uint(q.y);
+          }
+        }
+        if (OUT == HTC_OUT_T) {
+          if (!raw) {
+            ptx::st_global_v8(dst + ch * 64, bits[0], bits[1], bits[2], bits[3], bits[4], bits[5], bits[6], bits[7]);
+            ptx::st_global_v8(dst + ch * 64 + 32, bits[8], bits[9], bits[10], bits[11], bits[12], bits[13], bits[14], bits[15]);
+          }
+          return;
+        }
+        // 4-bit: word = sum_i (0x4B400000 | u_i) << 4 i  (mod 2^32), u_i the code + 8; the constant part of the sum
+        // is HTC_NIB_BIAS; low nibble = even channel.  Two interleaved chains (even / odd nibbles).
+        uint32_t w4[2];
+        if (OUT == HTC_OUT_PUBLIC) {
 #pragma unroll
           for (int h2 = 0; h2 < 2; ++h2) {
-            const float2 raw2 = make_float2(__uint_as_float(x[4 * g + 2 * h2]), __uint_as_float(x[4 * g + 2 * h2 + 1]));
-            // 2^(-j/2) = c * 2^(-(j >> 1)): only c touches the data, head + tail so the product is rounded once
-            const float2 t = __ffma2_rn(raw2, nhi, __fmul2_rn(raw2, nlo));
-            if (OUT == HTC_OUT_T) {
-              bits[2 * h2] = __float_as_uint(t.x * pw);
-              bits[2 * h2 + 1] = __float_as_uint(t.y * pw);
-            } else {
-              const float2 q0 = __fmul2_rn(t, inv2);
-              const float2 rem = __ffma2_rn(q0, ns2, t);
-              const float2 q = __fadd2_rn(__ffma2_rn(rem, inv2, q0), make_float2(CQ_MAGIC, CQ_MAGIC));
-              bits[2 * h2] = __float_as_uint(q.x);
-              bits[2 * h2 + 1] = __float_as_uint(q.y);
+            uint32_t ev = bits[8 * h2 + 6], od = bits[8 * h2 + 7];
+#pragma unroll
+            for (int k = 2; k >= 0; --k) {
+              ev = (ev << 8) + bits[8 * h2 + 2 * k];
+              od = (od << 8) + bits[8 * h2 + 2 * k + 1];
             }
+            w4[h2] = ((od << 4) + ev - HTC_NIB_BIAS) ^ 0x88888888u;
           }
-          if (OUT == HTC_OUT_T) {
-            reinterpret_cast<uint4*>(dst)[ch * 8 + g] = make_uint4(bits[0], bits[1], bits[2], bits[3]);
+        }
+        if (OUT == HTC_OUT_PUBLIC && !MIXED) {
+          pend[2 * ch] = w4[0];
+          pend[2 * ch + 1] = w4[1];
+          if (ch == 3) ptx::st_global_v8(dst, pend[0], pend[1], pend[2], pend[3], pend[4], pend[5], pend[6], pend[7]);
+          return;
+        }
+        // 8-bit: the low byte of each word is the two's complement code
+        uint32_t w8[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+          w8[g] = __byte_perm(__byte_perm(bits[4 * g], bits[4 * g + 1], 0x0040), __byte_perm(bits[4 * g + 2], bits[4 * g + 3], 0x0040), 0x5410);
+        if (OUT != HTC_OUT_PUBLIC) {   // GEMM operand: every row one code per byte
+          if (ch & 1) {
+            if (!raw) ptx::st_global_v8(dst + 32 * (ch >> 1), pend[0], pend[1], pend[2], pend[3], w8[0], w8[1], w8[2], w8[3]);
           } else {
-            // the low byte of each word is the two's complement code
-            w[g] = __byte_perm(__byte_perm(bits[0], bits[1], 0x0040), __byte_perm(bits[2], bits[3], 0x0040), 0x5410);
-          }
-        }
-        if (OUT == HTC_OUT_T) continue;
-        if (four_bit) {
-          uint32_t n4[4];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const uint32_t na = w[2 * g] & 0x0F0F0F0Fu, nb = w[2 * g + 1] & 0x0F0F0F0Fu;
-            const uint32_t ta = (na | (na >> 4)) & 0x00FF00FFu, tb = (nb | (nb >> 4)) & 0x00FF00FFu;   // bytes 0, 2
-            n4[g] = __byte_perm(ta, tb, 0x6420);
+            for (int g = 0; g < 4; ++g) pend[g] = w8[g];
           }
-          reinterpret_cast<uint4*>(dst)[ch] = make_uint4(n4[0], n4[1], n4[2], n4[3]);
+          return;
+        }
+        // public format, mixed warp: an 8-bit lane fills pend[0..3], then stores with this chunk's words at odd
+        // chunks; a 4-bit lane fills pend[2 ch], pend[2 ch + 1] and stores after the last chunk
+        if (ch & 1) {
+          if (!raw && !four_bit) ptx::st_global_v8(dst + 32 * (ch >> 1), pend[0], pend[1], pend[2], pend[3], w8[0], w8[1], w8[2], w8[3]);
+          pend[2 * ch] = w4[0];
+          pend[2 * ch + 1] = w4[1];
         } else {
-          reinterpret_cast<uint4*>(dst)[2 * ch] = make_uint4(w[0], w[1], w[2], w[3]);
-          reinterpret_cast<uint4*>(dst)[2 * ch + 1] = make_uint4(w[4], w[5], w[6], w[7]);
-        }
-      }
-      ptx::tc_fence_before();
-      ptx::mbar_arrive(&tempty[buf]);
-      return true;
-    };
-
-    long i = set;
-    for (; i < n_local && ok; i += 2) {
-      const long item = blockIdx.x + i * gridDim.x;
-      const long rb = item / p.nchunks;
-      // ---- P1: maxima of this warp's 64 columns
-      const long jb = job_p1(i);
-      const int buf = static_cast<int>(jb & (HTC_NBUF - 1));
-      if (!wait_acc(jb)) {
-        ok = false;
-        break;
-      }
-      {
-        const uint32_t taddr = lane_base + static_cast<uint32_t>(buf * 128);
-        uint32_t v[2][32];
-        ptx::tmem_ld_32x32b_x32(taddr, v[0]);
-        ptx::tmem_ld_32x32b_x32(taddr + 32, v[1]);
-        ptx::tmem_ld_wait();
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(&tempty[buf]);     // the values are in registers: the accumulator may be refilled
-        float m0 = 0.f, m1 = 0.f;
+          if (ch == 0) {
 #pragma unroll
-        for (int q4 = 0; q4 < 32; ++q4) {
-          m0 = fmaxf(m0, fabsf(__uint_as_float(v[0][q4])));
-          m1 = fmaxf(m1, fabsf(__uint_as_float(v[1][q4])));
+            for (int g = 0; g < 4; ++g) pend[g] = four_bit ? (g < 2 ? w4[g] : 0u) : w8[g];
+          } else {   // ch == 2: a 4-bit lane keeps pend[0..3] (chunks 0, 1) and adds pend[4..5]; an 8-bit lane restarts
+            pend[4] = w4[0];
+            pend[5] = w4[1];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) pend[g] = four_bit ? pend[g] : w8[g];
+          }
         }
-        // hand the maxima to the set's publisher warp (its slot is clear once it has taken the previous tile's)
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&pempty[set], static_cast<uint32_t>(((i >> 1) & 1) ^ 1), abort_word,
-                                                            HTC_WAIT_LIMIT))) {
-          ok = false;
-          break;
+        if (ch == 3 && !raw && four_bit) ptx::st_global_v8(dst, pend[0], pend[1], pend[2], pend[3], pend[4], pend[5], pend[6], pend[7]);
+      };
+      const bool mixed = (OUT == HTC_OUT_PUBLIC) ? !all_four : __any_sync(0xffffffffu, raw);
+      auto step = [&](auto ch_tag) {
+        constexpr int ch = decltype(ch_tag)::value;
+        ptx::tmem_ld_wait();
+        if (ch < 3) {
+          ptx::tmem_ld_32x32b_x16(taddr + 16 * (ch + 1), v[(ch + 1) & 1]);
+        } else {
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(&tempty[1 + set]);   // every value of the accumulator is in registers: it may be refilled
         }
-        atomicMax(&pslot[set * 128 + r], __float_as_uint(fmaxf(m0, m1)));
-        ptx::mbar_arrive(&pfull[set]);
-      }
-      // ---- P2 of the item HTC_LAG back
-      if (i >= HTC_LAG && !pass2(i - HTC_LAG)) ok = false;
+        if (mixed)
+          chunk(v[ch & 1], ch_tag, std::true_type{}, std::true_type{});
+        else if (warp_has_odd)
+          chunk(v[ch & 1], ch_tag, std::true_type{}, std::false_type{});
+        else
+          chunk(v[ch & 1], ch_tag, std::false_type{}, std::false_type{});
+      };
+      step(std::integral_constant<int, 0>{});
+      step(std::integral_constant<int, 1>{});
+      step(std::integral_constant<int, 2>{});
+      step(std::integral_constant<int, 3>{});
     }
-    // the last HTC_LAG items of the CTA: their second products come after its last first product
-    for (long i2 = i - HTC_LAG; i2 < n_local && ok; i2 += 2)
-      if (i2 >= 0 && !pass2(i2)) ok = false;
     if (!ok) {
       *abort_word = 1;
       raise_device_status(STAMP_ERR_TIMEOUT);

@@ -901,8 +901,9 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
 // 128-token sums.
 // ------------------------------------------------------------------------------------------
 static bool htc_ok(const Problem& pb, int x_dtype) {
+  // the kernel's per-tile index arithmetic is 32-bit: tokens and work items must fit
   return pb.transform == STAMP_T_HAAR && x_dtype == STAMP_BF16 && pb.levels >= 1 && pb.n % 128 == 0 && !pb.act_zp &&
-         pb.K / 128 <= sm_count();
+         pb.K % 128 == 0 && pb.K / 128 <= sm_count() && pb.M < (1L << 31) && (pb.M >> 7) * (long)(pb.K / 128) < (1L << 31);
 }
 
 template <int OUT>
@@ -929,6 +930,9 @@ static int run_quantize_haar(const Problem& pb, const CqChoice& c, const void* X
   HtcParams hp{};
   hp.K = pb.K;
   hp.n = pb.n;
+  hp.n_shift = -1;
+  for (int sh = 7; sh < 31; ++sh)
+    if ((1 << sh) == pb.n) hp.n_shift = sh;
   hp.lv = lv;
   hp.last = (lv == pb.levels) ? 1 : 0;
   hp.k_hi = pb.k_hi;
