@@ -38,7 +38,13 @@ SECONDARY_WORKLOAD = "llm_mlp_up"         # read as well (extra.secondary): the 
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture of the kernel as it stands (see profiles/);
 # a workload is listed only while that capture is current.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # k_gemm_i8<256, 6, EPI_HAAR_BF16, pair>: dram__bytes_read.sum 736.34 MB + dram__bytes_write.sum 519.52 MB, one
+    # launch, single-pass capture at full size (profiles/k_gemm_i8_pair_dram_sweep_L32768_D8192.txt)
+    "sweep_L32768_D8192": 1255860000,
+    # the same kernel on the small case: 54.27 MB + 16.40 MB
+    "llm_mlp_up": 70661376,
+}
 
 
 def workloads():
