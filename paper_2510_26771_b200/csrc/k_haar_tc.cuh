@@ -10,13 +10,15 @@
 // that load:
 //   * the tensor cores apply up to seven Haar levels to a tile of 128 tokens x 128 channels as ONE product
 //     D = H X, where H (128 x 128, entries 0 / +1 / -1: the un-normalised Haar analysis matrix) is exact in
-//     bf16, X is bf16 as it lies in HBM (TMA, consumed as an MN-major operand: nothing is transposed), and the
-//     accumulation is fp32.  The 2^(-j/2) factors are applied afterwards exactly as the butterfly kernel does;
+//     bf16 and lives in tensor memory (64 columns: the product reads it as a tensor-memory operand, which leaves
+//     the whole shared memory to the activation tiles), X is bf16 as it lies in HBM (TMA, consumed as an MN-major
+//     operand: nothing is transposed), and the accumulation is fp32.  The 2^(-j/2) factors are applied afterwards
+//     exactly as the butterfly kernel does;
 //   * the activation tile stays in shared memory (32 KB of bf16) while the row maxima travel, and the product
 //     is simply issued again when they are back -- 4 us of tensor time per GB of activations, on a pipe that has
 //     nothing else to do in this pass -- so that no warp parks a coefficient in registers across the exchange
-//     and the ring of six tiles, not the register file, sets how many tiles can be waiting.  Tensor memory
-//     (lane = transformed token, column = channel) only holds the accumulators in flight.
+//     and the ring of seven tiles, not the register file, sets how many tiles can be waiting.  Tensor memory
+//     (lane = transformed token, column = channel) holds H and the three accumulators in flight.
 // An epilogue thread owns ONE transformed token of the tile: its maximum over the tile's channels is a
 // thread-local reduction, and later its scale, bit width and destination row are per-thread constants.  What
 // is left for the CUDA cores is about 5 instructions per element.
@@ -28,7 +30,7 @@
 //                 combines them into the row block's table in global memory (atomicMax) and, once they are
 //                 delivered, counts the tile in (two publishers alternate);
 //   job P2(item): HTC_LAG items later the MMA thread waits (bounded) until the row block's count is complete,
-//                 issues the product again into the accumulator of one of three sets of quantizing warps, and
+//                 issues the product again into the accumulator of one of two sets of quantizing warps, and
 //                 these read the final maxima, derive scale, bit width and destination of their row, quantize
 //                 and store the codes.
 // The warps that take the maxima do nothing else, so a tile's maxima leave the SM a few hundred clocks after its
@@ -73,16 +75,17 @@ struct HtcParams {
 
 enum HtcOut { HTC_OUT_A8 = 0, HTC_OUT_PUBLIC = 1, HTC_OUT_T = 2, HTC_OUT_TILED = 3 };
 
-// warps: 0 TMA producer, 1 MMA issuer, 2-3 publishers, 4-27 three sets of eight quantizing warps, 28-31 maxima
-constexpr int HTC_THREADS = 32 * 32;
-constexpr int HTC_QSETS = 3;
-constexpr int HTC_STAGES = 6;              // shared-memory ring of activation tiles
-constexpr int HTC_LAG = 3;                 // items between the two products of a tile (< HTC_STAGES)
+// warps: 0 TMA producer, 1 MMA issuer, 2-3 publishers, then HTC_QSETS sets of eight quantizing warps, then 4 maxima warps
+constexpr int HTC_QSETS = 2;
+constexpr int HTC_MAXW0 = 4 + 8 * HTC_QSETS;          // first maxima warp
+constexpr int HTC_THREADS = (HTC_MAXW0 + 4) * 32;
+constexpr int HTC_STAGES = 7;                         // shared-memory ring of activation tiles
+constexpr int HTC_H_COL = 128 * (1 + HTC_QSETS);      // H as a tensor-memory operand: 64 columns after the accumulators
+constexpr int HTC_LAG = 4;                 // items between the two products of a tile (< HTC_STAGES)
 constexpr int HTC_NBUF = 4;                // 128-column accumulators in tensor memory: one for P1 jobs, one per quantizing set
 constexpr int HTC_TILE_BYTES = 128 * 128 * 2;   // [128 tokens x 128 channels] bf16 = two 64-channel atoms
 constexpr int HTC_ATOM_BYTES = 128 * 128;       // [128 tokens x 64 channels] bf16
-constexpr int HTC_A_BYTES = 128 * 128 * 2;      // H: [128 rows x 128 tokens] bf16 = two 64-token atoms
-constexpr int HTC_BAR_OFFSET = HTC_A_BYTES + HTC_STAGES * HTC_TILE_BYTES;
+constexpr int HTC_BAR_OFFSET = HTC_STAGES * HTC_TILE_BYTES;
 constexpr int HTC_NUM_BARS = 2 * HTC_STAGES + 2 * HTC_NBUF + 4;   // ring, accumulators (full / empty), pfull[2], pempty[2]
 constexpr int HTC_SLOT_OFFSET = HTC_BAR_OFFSET + HTC_NUM_BARS * 8 + 16;   // [2 sets][128 lanes] maxima on their way out
 constexpr int HTC_DYN_BYTES = HTC_SLOT_OFFSET + 2 * 128 * 4 + 1024;
@@ -95,12 +98,13 @@ __host__ __device__ constexpr uint32_t htc_idesc() {
          (static_cast<uint32_t>(128 >> 4) << 24);
 }
 
-__device__ __forceinline__ void htc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+// D (+)= A B with A read from tensor memory (lane = row of A, two bf16 per 32-bit column: 16 tokens = 8 columns)
+__device__ __forceinline__ void htc_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(htc_idesc()), "r"(accumulate)
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(htc_idesc()), "r"(accumulate)
       : "memory");
 }
 
@@ -145,8 +149,7 @@ template <int OUT>
 __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constant__ CUtensorMap tmap_x, const HtcParams p) {
   extern __shared__ uint8_t htc_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(htc_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* a_sm = smem;                              // H
-  uint8_t* b_sm = smem + HTC_A_BYTES;                // ring of activation tiles
+  uint8_t* b_sm = smem;                              // ring of activation tiles
   uint64_t* sfull = reinterpret_cast<uint64_t*>(smem + HTC_BAR_OFFSET);
   uint64_t* sempty = sfull + HTC_STAGES;
   uint64_t* tfull = sempty + HTC_STAGES;
@@ -164,30 +167,6 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
   const int n_local = nitems > blockIdx.x ? static_cast<int>((nitems - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;   // this CTA's items
   const unsigned nchunks = static_cast<unsigned>(p.nchunks);
 
-  // ---- the analysis matrix, written straight into the K-major 128-byte-swizzled operand layout:
-  // element (row r, token t) of atom t / 64 sits in 16-byte chunk ((t % 64) / 8) ^ (r % 8) of row r
-  for (int e = threadIdx.x; e < 128 * 16; e += HTC_THREADS) {
-    const int r = e >> 4, c16 = e & 15;              // row, 8-token group
-    int j, idx;
-    bool approx;
-    htc_lane_row(p.lv, r, j, idx, approx);
-    const int first = idx << j, mid = first + (1 << j) / 2, end = first + (1 << j);
-    uint32_t w[4];
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      uint32_t pair = 0;
-#pragma unroll
-      for (int s = 0; s < 2; ++s) {
-        const int t = c16 * 8 + 2 * h + s;
-        uint32_t v = 0;
-        if (t >= first && t < end) v = (approx || t < mid) ? 0x3F80u : 0xBF80u;   // +1.0 / -1.0 in bf16
-        pair |= v << (16 * s);
-      }
-      w[h] = pair;
-    }
-    const int atom = c16 >> 3, chunk = (c16 & 7) ^ (r & 7);
-    *reinterpret_cast<uint4*>(a_sm + atom * HTC_ATOM_BYTES + r * 128 + chunk * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < HTC_STAGES; ++s) {
       ptx::mbar_init(&sfull[s], 1);
@@ -205,7 +184,6 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmap_x);
   }
-  ptx::fence_proxy_async_smem();   // H was written with ordinary stores; the tensor cores read it through the async proxy
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, 512);
     ptx::tmem_relinquish();
@@ -214,6 +192,36 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // H into tensor memory: thread = row r of H (its lane), column c = tokens 2 c (low half) and 2 c + 1 (high half)
+  if (warp >= 4 && warp < 8) {
+    const int r = (warp & 3) * 32 + lane;
+    int j, idx;
+    bool approx;
+    htc_lane_row(p.lv, r, j, idx, approx);
+    const int first = idx << j, mid = first + (1 << j) / 2, end = first + (1 << j);
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + HTC_H_COL;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      uint32_t w[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        uint32_t pair = 0;
+#pragma unroll
+        for (int s2 = 0; s2 < 2; ++s2) {
+          const int t = 2 * (16 * g + c) + s2;
+          uint32_t v = 0;
+          if (t >= first && t < end) v = (approx || t < mid) ? 0x3F80u : 0xBF80u;   // +1.0 / -1.0 in bf16
+          pair |= v << (16 * s2);
+        }
+        w[c] = pair;
+      }
+      ptx::tmem_st_32x32b_x16(taddr + 16 * g, w);
+    }
+    ptx::tmem_st_wait();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
   if (warp == 0 && p.pf_bytes > 0) {   // fire-and-forget hints, 8 KB each
     constexpr long PF_CHUNK = 8192;
     const long nchunk = (p.pf_bytes + PF_CHUNK - 1) / PF_CHUNK;
@@ -263,11 +271,10 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    // Static order: P1 of item t, then P2 of item t - HTC_LAG.  Accumulator 0 for a P1 job, 1 + i % 3 for the P2
-    // job of item i (the quantizing set i % 3 drains it).
+    // Static order: P1 of item t, then P2 of item t - HTC_LAG.  Accumulator 0 for a P1 job, 1 + i % HTC_QSETS for
+    // the P2 job of item i (the quantizing set i % HTC_QSETS drains it).
     if (ptx::elect_one()) {
       bool ok = true;
-      const uint32_t abase = ptx::smem_u32(a_sm);
       // D = H X of the tile in ring stage `stage` into accumulator `buf`, whose `use`-th filling this is; the
       // second product of a tile also hands the stage back to the producer
       auto product = [&](int stage, int buf, int use, bool release_stage) -> bool {
@@ -277,9 +284,8 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
         const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * 128);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {   // 16 tokens per instruction
-          const uint64_t adesc = ptx::make_kmajor_sw128_desc(abase + (k >> 2) * HTC_ATOM_BYTES + (k & 3) * 32);
           const uint64_t bdesc = htc_bdesc(bbase + k * 16 * 128);
-          htc_mma(tmem_d, adesc, bdesc, k != 0 ? 1u : 0u);
+          htc_mma_ts(tmem_d, tmem_base + HTC_H_COL + 8 * k, bdesc, k != 0 ? 1u : 0u);   // 16 tokens = 8 columns of H
         }
         if (release_stage) ptx::tc_commit(&sempty[stage]);
         ptx::tc_commit(&tfull[buf]);
@@ -346,7 +352,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
       *abort_word = 1;
       raise_device_status(STAMP_ERR_TIMEOUT);
     }
-  } else if (warp >= 28) {
+  } else if (warp >= HTC_MAXW0) {
     // ------------------------------------------------------------------ maxima warps: one per quarter of the lanes
     // P1 of every item: |D| of this thread's lane over the tile's 128 columns, left in the slot of the item's
     // parity for the publisher.  The accumulator is released as soon as its values are in registers.
@@ -390,7 +396,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     }
   } else {
     // ------------------------------------------------------------------ quantizing warps
-    // Three sets of eight warps take the CTA's items in turn; inside a set a warp owns the 32 lanes of its
+    // Two sets of eight warps take the CTA's items in turn; inside a set a warp owns the 32 lanes of its
     // quarter (warp % 4) and 64 of the tile's 128 columns, a thread ONE transformed token: scale, bit width and
     // destination row are per-thread scalars, and a thread's 64 codes are 32 or 64 contiguous bytes of its row.
     const int e = warp - 4;
