@@ -162,7 +162,8 @@ __global__ void __launch_bounds__(512, 1) k_haar_cq(const CqParams p) {
       ptx::prefetch_l2_bulk(p.pf_base + off, static_cast<uint32_t>(left < PF_CHUNK ? left : PF_CHUNK));
     }
   }
-  ptx::grid_dependency_wait();   // the input rows may come from the previous launch
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();   // the next kernel may set itself up on SMs as they fall free; it still waits for this grid to finish   // the input rows may come from the previous launch
 
   // warp 0 brings one group's rows of this strip into a ring stage: lane r copies token row r
   auto issue_load = [&](long grp, int stage) {

@@ -145,6 +145,16 @@ __device__ __forceinline__ void htc_lane_row(int lv, int r, int& j, int& idx, bo
   }
 }
 
+// Clears the row-maximum table and the tile counts before k_haar_tc.  A kernel rather than a memset, so that both
+// launches can be programmatic dependents: this one's launch overlaps the tail of whatever ran before (it waits for
+// that to complete before it writes), and k_haar_tc sets up its barriers, tensor memory and H while this one runs.
+__global__ void __launch_bounds__(256) k_htc_clear(uint4* __restrict__ words16, long n16) {
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+  for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (long)gridDim.x * blockDim.x)
+    words16[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
 template <int OUT>
 __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constant__ CUtensorMap tmap_x, const HtcParams p) {
   extern __shared__ uint8_t htc_raw[];
@@ -232,6 +242,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     }
   }
   ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();   // the next kernel may set itself up on SMs as they fall free; it still waits for this grid to finish
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer

@@ -36,6 +36,7 @@ __global__ void __launch_bounds__(TOPG_THREADS, (R <= 4 ? 3 : (R <= 8 ? 4 : 2)))
                                                            int top_levels, float* __restrict__ a8v) {
   extern __shared__ __align__(16) uint8_t topg_smem[];   // [R, K] codes
   ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();   // the next kernel may set itself up on SMs as they fall free; it still waits for this grid to finish
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   {
     const uint4* src = reinterpret_cast<const uint4*>(codes);

@@ -313,6 +313,9 @@ __device__ __forceinline__ void prefetch_l2_bulk(const void* gptr, uint32_t byte
 }
 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream (a programmatic dependent) be scheduled now; its own griddepcontrol.wait still
+// waits until this grid has completed and its writes are visible.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---------------------------------------------------------------- clusters
 __device__ __forceinline__ uint32_t cluster_ctarank() {

@@ -954,8 +954,17 @@ static int run_quantize_haar(const Problem& pb, const CqChoice& c, const void* X
     hp.pf_bytes = tiled->pf_bytes;
   }
   // row maxima and tile counts start from zero (the two regions are adjacent)
-  if (cudaMemsetAsync(base + wl.rowmax, 0, (wl.htc_cnt - wl.rowmax) + (size_t)(pb.M >> 7) * 4, st) != cudaSuccess)
-    return STAMP_ERR_CUDA;
+  {
+    const size_t bytes = (wl.htc_cnt - wl.rowmax) + (size_t)(pb.M >> 7) * 4;
+    const long n16 = (long)((bytes + 15) / 16);   // both regions are 256-byte aligned and padded in the workspace
+    const int grid = (int)std::min<long>((n16 + 255) / 256, 64);
+    if (launch_pdl(k_htc_clear, dim3((unsigned)grid), dim3(256), 0, st, reinterpret_cast<uint4*>(base + wl.rowmax), n16) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return STAMP_ERR_CUDA;
+    }
+    STAMP_CHECK_LAUNCH();
+  }
   CUtensorMap tx;
   int rc = make_tmap_bf16(X, pb.M, pb.K, &tx, 128);
   if (rc) return rc;
