@@ -69,6 +69,13 @@ struct HtcParams {
   float* x_scale;    // [M] logical order (A8, PUBLIC)
   float* T_out;      // HTC_OUT_T: [M, K] transformed values, fp32 (debug export)
   float* sx_epi;     // HTC_OUT_TILED: [M] scale * 2^(-j/2) of every tile row, indexed like a8
+  // fold != 0: the levels above the seventh are finished by this kernel's tail (logical-order outputs only)
+  int fold;
+  int levels;        // depth of the whole transform (fold)
+  int nseq;          // transform blocks: M / n (fold)
+  unsigned* done;    // [1] zero on entry: CTAs whose 128-token sums are written
+  unsigned* rowmax2; // [M / 128] zero on entry: maxima of the coarse rows, block * (n / 128) + logical row
+  unsigned* cnt2;    // [nseq] zero on entry: strips of a block whose coarse maxima have been sent
   const uint8_t* pf_base;   // optional region to pull towards L2 (the layer's weight codes), pf_bytes % 16 == 0
   long pf_bytes;
 };
@@ -620,6 +627,159 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     if (!ok) {
       *abort_word = 1;
       raise_device_status(STAMP_ERR_TIMEOUT);
+    }
+  }
+
+  // ------------------------------------------------------------------ tail: the levels above the seventh
+  // The 128-token sums of a block (n / 128 rows x K, fp32, 1 / 128 of the data) are what the deeper levels work on.
+  // When they fit the shared memory that the ring no longer needs, the CTAs finish the transform themselves
+  // instead of leaving it to one or two more launches: a CTA takes (block, 128-channel strip) items, loads the
+  // strip's sums, runs the remaining levels in place (after level l the sums sit at rows that are multiples of
+  // 2^(l+1), the details of that level at the odd multiples of 2^l: every pair writes back to the two rows it
+  // read), exchanges the maxima of the coarse rows exactly as above (table, release count, bounded acquire
+  // wait) and quantizes them with the arithmetic of the quantizing warps.
+  if (p.fold) {
+    __syncthreads();   // every role is through: this CTA's sums are written
+    float* S = reinterpret_cast<float*>(b_sm);
+    volatile uint32_t* tail_ok = abort_word + 1;
+    const int R = p.n >> 7, lr = p.levels - 7;
+    if (threadIdx.x == 0) {
+      asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.done) : "memory");
+      bool ok = (*abort_word == 0u);
+      const long long t0 = clock64();
+      unsigned spins = 0;
+      while (ok && ld_acquire_gpu(p.done) < gridDim.x) {
+        if ((++spins & 15u) == 0u && clock64() - t0 > HTC_WAIT_LIMIT) ok = false;
+        __nanosleep(100);
+      }
+      if (!ok) raise_device_status(STAMP_ERR_TIMEOUT);
+      *tail_ok = ok ? 1u : 0u;
+    }
+    __syncthreads();
+    bool ok = (*tail_ok != 0u);
+    const unsigned ntail = static_cast<unsigned>(p.nseq) * nchunks;
+    const int K = p.K;
+    for (unsigned it = blockIdx.x; it < ntail && ok; it += gridDim.x) {
+      const unsigned blk = it / nchunks;
+      const unsigned c = it - blk * nchunks;
+      // (1) the strip's sums: R rows x 128 channels
+      for (int e0 = threadIdx.x; e0 < R * 32; e0 += 4 * HTC_THREADS) {   // four loads in flight per thread
+        float4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int e = e0 + k * HTC_THREADS;
+          if (e < R * 32)   // other CTAs wrote the sums: read past L1
+            v[k] = __ldcg(reinterpret_cast<const float4*>(p.aout + ((size_t)blk * R + (e >> 5)) * K + c * 128u + 4 * (e & 31)));
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int e = e0 + k * HTC_THREADS;
+          if (e < R * 32) reinterpret_cast<float4*>(S)[e] = v[k];
+        }
+      }
+      __syncthreads();
+      // (2) remaining levels on un-normalised sums, in place
+      for (int l = 0; l < lr; ++l) {
+        const int npairs = R >> (l + 1);
+        for (int e = threadIdx.x; e < npairs * 32; e += HTC_THREADS) {   // four channels at a time
+          const int i = e >> 5, q = e & 31;
+          float4* a = reinterpret_cast<float4*>(S) + (i << (l + 1)) * 32 + q;
+          float4* b = a + (32 << l);
+          const float4 x0 = *a, x1 = *b;
+          *a = make_float4(x0.x + x1.x, x0.y + x1.y, x0.z + x1.z, x0.w + x1.w);
+          *b = make_float4(x0.x - x1.x, x0.y - x1.y, x0.z - x1.z, x0.w - x1.w);
+        }
+        __syncthreads();
+      }
+      // (3) maxima of the strip's rows (un-normalised, as in the main loop), one warp per row
+      for (int row = warp; row < R; row += HTC_THREADS / 32) {
+        const float4 v = reinterpret_cast<const float4*>(S)[row * 32 + lane];
+        float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+        m = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(m)));
+        if (lane == 0) atomicMax(p.rowmax2 + (size_t)blk * R + row, __float_as_uint(m));   // indexed by the row in S
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt2 + blk) : "memory");
+        const long long t0 = clock64();
+        unsigned spins = 0;
+        bool got = true;
+        while (ld_acquire_gpu(p.cnt2 + blk) < nchunks) {
+          if ((++spins & 15u) == 0u && clock64() - t0 > HTC_WAIT_LIMIT) {
+            got = false;
+            break;
+          }
+          __nanosleep(100);
+        }
+        if (!got) raise_device_status(STAMP_ERR_TIMEOUT);
+        *tail_ok = got ? 1u : 0u;
+      }
+      __syncthreads();
+      ok = (*tail_ok != 0u);
+      if (!ok) break;
+      // the block's final maxima, once, behind the strip (one load per row here instead of one round trip per row below)
+      // every row's level, destination, scale and reciprocal, one thread per row (the two divisions of all rows run
+      // side by side here instead of one after the other in the loop below)
+      float4* srow = reinterpret_cast<float4*>(S + (size_t)R * 128);   // {scale, 1 / scale, scale as stored, level | hi << 8}
+      for (int row = threadIdx.x; row < R; row += HTC_THREADS) {
+        int j, lrow;
+        if ((row & ((1 << lr) - 1)) == 0) {
+          j = p.levels;
+          lrow = row >> lr;
+        } else {
+          const int tz = __ffs(row) - 1;
+          j = 8 + tz;
+          lrow = (p.n >> j) + (row >> (tz + 1));
+        }
+        const bool hi = lrow < p.k_hi;
+        const float qmax = hi ? p.qmax_hi : p.qmax_lo;
+        const float u = __uint_as_float(ld_relaxed_gpu(p.rowmax2 + (size_t)blk * R + row));
+        const float amax = (j & 1) ? fmaf(u, CQ_RSQRT2_HI, u * CQ_RSQRT2_LO) : u;
+        const float scale = (amax > 0.f) ? __fdiv_rn(amax, qmax) : 1.0f;
+        const float pw = __int_as_float((127 - (j >> 1)) << 23);      // 2^(-(j >> 1))
+        srow[row] = make_float4(scale, __fdiv_rn(1.0f, scale), (amax > 0.f) ? scale * pw : 1.0f,
+                                __int_as_float(j | (hi ? 256 : 0) | (lrow << 9)));
+      }
+      __syncthreads();
+      // (4) quantize, one warp per row, a lane four channels
+      for (int row = warp; row < R; row += HTC_THREADS / 32) {
+        const float4 sr = srow[row];
+        const float scale = sr.x, inv = sr.y, true_scale = sr.z;
+        const int tag = __float_as_int(sr.w);
+        const int j = tag & 255, lrow = tag >> 9;
+        const bool hi = (tag & 256) != 0, odd = (j & 1) != 0;
+        const float pw = __int_as_float((127 - (j >> 1)) << 23);      // 2^(-(j >> 1))
+        const float4 v = reinterpret_cast<const float4*>(S)[row * 32 + lane];
+        const float raw4[4] = {v.x, v.y, v.z, v.w};
+        const size_t grow = (size_t)blk * p.n + lrow;     // logical row of the whole problem
+        const unsigned col = c * 128u + 4u * lane;
+        if (OUT == HTC_OUT_T) {
+          float o[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) o[k] = (odd ? fmaf(raw4[k], CQ_RSQRT2_HI, raw4[k] * CQ_RSQRT2_LO) : raw4[k]) * pw;
+          *reinterpret_cast<float4*>(p.T_out + grow * K + col) = make_float4(o[0], o[1], o[2], o[3]);
+          continue;
+        }
+        uint32_t code[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float t = odd ? fmaf(raw4[k], CQ_RSQRT2_HI, raw4[k] * CQ_RSQRT2_LO) : raw4[k];
+          const float q0 = t * inv;
+          const float rem = fmaf(q0, -scale, t);
+          code[k] = __float_as_uint(fmaf(rem, inv, q0) + CQ_MAGIC);   // low byte: the two's complement code
+        }
+        if (OUT == HTC_OUT_PUBLIC && !hi) {
+          const uint32_t b0 = (code[0] & 0xFu) | ((code[1] & 0xFu) << 4), b1 = (code[2] & 0xFu) | ((code[3] & 0xFu) << 4);
+          *reinterpret_cast<uint16_t*>(p.q_lo + ((size_t)blk * (p.n - p.k_hi) + (lrow - p.k_hi)) * (size_t)(K >> 1) + (col >> 1)) =
+              static_cast<uint16_t>(b0 | (b1 << 8));
+        } else {
+          const uint32_t w = (code[0] & 0xFFu) | ((code[1] & 0xFFu) << 8) | ((code[2] & 0xFFu) << 16) | (code[3] << 24);
+          int8_t* base8 = (OUT == HTC_OUT_PUBLIC) ? p.q_hi + ((size_t)blk * p.k_hi + lrow) * (size_t)K : p.a8 + grow * (size_t)K;
+          *reinterpret_cast<uint32_t*>(base8 + col) = w;
+        }
+        if (c == 0 && lane == 0) p.x_scale[grow] = true_scale;
+      }
+      __syncthreads();   // S is loaded again for the CTA's next item
     }
   }
 

@@ -140,7 +140,8 @@ static Workspace layout(const Problem& pb) {
   size_t off = 0;
   w.rowmax = off; off += align256(M * 4);
   // (directly behind the row maxima: one memset clears both before the tensor-core transform+quantize launch)
-  w.htc_cnt = off; off += align256((M >> 7) * 4 + 4);
+  // tile counts [M / 128], CTA count [4 words], coarse-row maxima [M / 128], strip counts per block [nseq]
+  w.htc_cnt = off; off += align256(((M >> 7) * 2 + 4 + (size_t)pb.nseq) * 4 + 16);
   w.xscale = off; off += align256(M * 4 * (size_t)(pb.group ? pb.K / pb.group : 1));
   // low-pass band after the first level of the first-token-excluded Haar transform (forward: K wide, inverse: N wide)
   w.skipa = off;  off += align256(pb.transform == STAMP_T_HAAR_SKIP1 ? (M / 2) * KN * 4 : 0);
@@ -954,8 +955,19 @@ static int run_quantize_haar(const Problem& pb, const CqChoice& c, const void* X
     hp.pf_bytes = tiled->pf_bytes;
   }
   // row maxima and tile counts start from zero (the two regions are adjacent)
+  // The kernel's tail finishes the levels above the seventh itself when the outputs are in logical order and a
+  // block has at most 64 rows of 128-token sums (blocks of up to 8192 tokens).  Measured, whole call, tail against
+  // continuation launches: 31 against 35 us at 2048 tokens x 4096 channels, 54.6 against 55.5 us at 8192 x 8192;
+  // with 256 rows per block (32768 tokens) one CTA per 128-channel strip is too few hands (164 against 154 us).
+  const int coarse_rows = pb.n >> 7;
+  hp.fold = (!tiled && !hp.last && coarse_rows <= 64) ? 1 : 0;
+  hp.levels = pb.levels;
+  hp.nseq = pb.nseq;
+  hp.done = hp.cnt + (pb.M >> 7);
+  hp.rowmax2 = hp.done + 4;
+  hp.cnt2 = hp.rowmax2 + (pb.M >> 7);
   {
-    const size_t bytes = (wl.htc_cnt - wl.rowmax) + (size_t)(pb.M >> 7) * 4;
+    const size_t bytes = (wl.htc_cnt - wl.rowmax) + ((size_t)(pb.M >> 7) * 2 + 4 + (size_t)pb.nseq) * 4;
     const long n16 = (long)((bytes + 15) / 16);   // both regions are 256-byte aligned and padded in the workspace
     const int grid = (int)std::min<long>((n16 + 255) / 256, 64);
     if (launch_pdl(k_htc_clear, dim3((unsigned)grid), dim3(256), 0, st, reinterpret_cast<uint4*>(base + wl.rowmax), n16) !=
@@ -972,7 +984,7 @@ static int run_quantize_haar(const Problem& pb, const CqChoice& c, const void* X
        : a8  ? launch_htc<HTC_OUT_A8>(tx, hp, st)
         : T_out ? launch_htc<HTC_OUT_T>(tx, hp, st)
                 : launch_htc<HTC_OUT_PUBLIC>(tx, hp, st);
-  if (rc || hp.last) return rc;
+  if (rc || hp.last || hp.fold) return rc;
   CqTiled rest;
   if (tiled) {
     rest = *tiled;
