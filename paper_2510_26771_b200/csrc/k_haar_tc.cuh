@@ -69,7 +69,8 @@ struct HtcParams {
   float* x_scale;    // [M] logical order (A8, PUBLIC)
   float* T_out;      // HTC_OUT_T: [M, K] transformed values, fp32 (debug export)
   float* sx_epi;     // HTC_OUT_TILED: [M] scale * 2^(-j/2) of every tile row, indexed like a8
-  // fold != 0: the levels above the seventh are finished by this kernel's tail (logical-order outputs only)
+  // fold != 0: the levels above the seventh are finished by this kernel's tail (logical-order outputs only), in
+  // strips of 128 channels (1) or 64 channels (2)
   int fold;
   int levels;        // depth of the whole transform (fold)
   int nseq;          // transform blocks: M / n (fold)
@@ -643,6 +644,9 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     float* S = reinterpret_cast<float*>(b_sm);
     volatile uint32_t* tail_ok = abort_word + 1;
     const int R = p.n >> 7, lr = p.levels - 7;
+    // strips of 128 channels, or of 64 when that gives more CTAs something to do (sh = log2 of float4 per strip row)
+    const int sh = p.fold == 2 ? 4 : 5, sw4 = 1 << sh;
+    const unsigned nstrips = static_cast<unsigned>(p.K >> (sh + 2));
     if (threadIdx.x == 0) {
       asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.done) : "memory");
       bool ok = (*abort_word == 0u);
@@ -657,34 +661,34 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
     }
     __syncthreads();
     bool ok = (*tail_ok != 0u);
-    const unsigned ntail = static_cast<unsigned>(p.nseq) * nchunks;
+    const unsigned ntail = static_cast<unsigned>(p.nseq) * nstrips;
     const int K = p.K;
     for (unsigned it = blockIdx.x; it < ntail && ok; it += gridDim.x) {
-      const unsigned blk = it / nchunks;
-      const unsigned c = it - blk * nchunks;
-      // (1) the strip's sums: R rows x 128 channels
-      for (int e0 = threadIdx.x; e0 < R * 32; e0 += 4 * HTC_THREADS) {   // four loads in flight per thread
+      const unsigned blk = it / nstrips;
+      const unsigned c = it - blk * nstrips;
+      // (1) the strip's sums: R rows x 4 sw4 channels
+      for (int e0 = threadIdx.x; e0 < (R << sh); e0 += 4 * HTC_THREADS) {   // four loads in flight per thread
         float4 v[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int e = e0 + k * HTC_THREADS;
-          if (e < R * 32)   // other CTAs wrote the sums: read past L1
-            v[k] = __ldcg(reinterpret_cast<const float4*>(p.aout + ((size_t)blk * R + (e >> 5)) * K + c * 128u + 4 * (e & 31)));
+          if (e < (R << sh))   // other CTAs wrote the sums: read past L1
+            v[k] = __ldcg(reinterpret_cast<const float4*>(p.aout + ((size_t)blk * R + (e >> sh)) * K + ((c << sh) + (e & (sw4 - 1))) * 4u));
         }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int e = e0 + k * HTC_THREADS;
-          if (e < R * 32) reinterpret_cast<float4*>(S)[e] = v[k];
+          if (e < (R << sh)) reinterpret_cast<float4*>(S)[e] = v[k];
         }
       }
       __syncthreads();
       // (2) remaining levels on un-normalised sums, in place
       for (int l = 0; l < lr; ++l) {
         const int npairs = R >> (l + 1);
-        for (int e = threadIdx.x; e < npairs * 32; e += HTC_THREADS) {   // four channels at a time
-          const int i = e >> 5, q = e & 31;
-          float4* a = reinterpret_cast<float4*>(S) + (i << (l + 1)) * 32 + q;
-          float4* b = a + (32 << l);
+        for (int e = threadIdx.x; e < (npairs << sh); e += HTC_THREADS) {   // four channels at a time
+          const int i = e >> sh, q = e & (sw4 - 1);
+          float4* a = reinterpret_cast<float4*>(S) + ((i << (l + 1)) << sh) + q;
+          float4* b = a + (sw4 << l);
           const float4 x0 = *a, x1 = *b;
           *a = make_float4(x0.x + x1.x, x0.y + x1.y, x0.z + x1.z, x0.w + x1.w);
           *b = make_float4(x0.x - x1.x, x0.y - x1.y, x0.z - x1.z, x0.w - x1.w);
@@ -692,11 +696,15 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
         __syncthreads();
       }
       // (3) maxima of the strip's rows (un-normalised, as in the main loop), one warp per row
-      for (int row = warp; row < R; row += HTC_THREADS / 32) {
-        const float4 v = reinterpret_cast<const float4*>(S)[row * 32 + lane];
-        float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
-        m = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(m)));
-        if (lane == 0) atomicMax(p.rowmax2 + (size_t)blk * R + row, __float_as_uint(m));   // indexed by the row in S
+      // (a warp takes one row of 128 channels or two rows of 64: R is even)
+      const int rpw = 32 >> sh, sub = lane >> sh, ln = lane & (sw4 - 1);
+      const unsigned submask = sh == 5 ? 0xffffffffu : (0xffffu << (16 * sub));
+      for (int row0 = warp * rpw; row0 < R; row0 += (HTC_THREADS / 32) * rpw) {
+        const int row = row0 + sub;
+        const float4 v = reinterpret_cast<const float4*>(S)[(row << sh) + ln];
+        const float m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+        const unsigned mm = __reduce_max_sync(submask, __float_as_uint(m));
+        if (ln == 0) atomicMax(p.rowmax2 + (size_t)blk * R + row, mm);   // indexed by the row in S
       }
       __syncthreads();
       if (threadIdx.x == 0) {
@@ -704,7 +712,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
         const long long t0 = clock64();
         unsigned spins = 0;
         bool got = true;
-        while (ld_acquire_gpu(p.cnt2 + blk) < nchunks) {
+        while (ld_acquire_gpu(p.cnt2 + blk) < nstrips) {
           if ((++spins & 15u) == 0u && clock64() - t0 > HTC_WAIT_LIMIT) {
             got = false;
             break;
@@ -720,7 +728,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
       // the block's final maxima, once, behind the strip (one load per row here instead of one round trip per row below)
       // every row's level, destination, scale and reciprocal, one thread per row (the two divisions of all rows run
       // side by side here instead of one after the other in the loop below)
-      float4* srow = reinterpret_cast<float4*>(S + (size_t)R * 128);   // {scale, 1 / scale, scale as stored, level | hi << 8}
+      float4* srow = reinterpret_cast<float4*>(S) + ((size_t)R << sh);   // {scale, 1 / scale, scale as stored, level | hi << 8}
       for (int row = threadIdx.x; row < R; row += HTC_THREADS) {
         int j, lrow;
         if ((row & ((1 << lr) - 1)) == 0) {
@@ -742,17 +750,18 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
       }
       __syncthreads();
       // (4) quantize, one warp per row, a lane four channels
-      for (int row = warp; row < R; row += HTC_THREADS / 32) {
+      for (int row0 = warp * rpw; row0 < R; row0 += (HTC_THREADS / 32) * rpw) {
+        const int row = row0 + sub;
         const float4 sr = srow[row];
         const float scale = sr.x, inv = sr.y, true_scale = sr.z;
         const int tag = __float_as_int(sr.w);
         const int j = tag & 255, lrow = tag >> 9;
         const bool hi = (tag & 256) != 0, odd = (j & 1) != 0;
         const float pw = __int_as_float((127 - (j >> 1)) << 23);      // 2^(-(j >> 1))
-        const float4 v = reinterpret_cast<const float4*>(S)[row * 32 + lane];
+        const float4 v = reinterpret_cast<const float4*>(S)[(row << sh) + ln];
         const float raw4[4] = {v.x, v.y, v.z, v.w};
         const size_t grow = (size_t)blk * p.n + lrow;     // logical row of the whole problem
-        const unsigned col = c * 128u + 4u * lane;
+        const unsigned col = ((c << sh) + ln) * 4u;
         if (OUT == HTC_OUT_T) {
           float o[4];
 #pragma unroll
@@ -777,7 +786,7 @@ __global__ void __launch_bounds__(HTC_THREADS, 1) k_haar_tc(const __grid_constan
           int8_t* base8 = (OUT == HTC_OUT_PUBLIC) ? p.q_hi + ((size_t)blk * p.k_hi + lrow) * (size_t)K : p.a8 + grow * (size_t)K;
           *reinterpret_cast<uint32_t*>(base8 + col) = w;
         }
-        if (c == 0 && lane == 0) p.x_scale[grow] = true_scale;
+        if (c == 0 && ln == 0) p.x_scale[grow] = true_scale;
       }
       __syncthreads();   // S is loaded again for the CTA's next item
     }

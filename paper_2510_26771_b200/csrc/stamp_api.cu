@@ -901,6 +901,9 @@ static int run_quantize_cq(const Problem& pb, const CqChoice& c, const void* X, 
 // coefficients resident in tensor memory (k_haar_tc), deeper levels by the butterfly kernel on the
 // 128-token sums.
 // ------------------------------------------------------------------------------------------
+#ifndef HTC_FOLD_ROWS
+#define HTC_FOLD_ROWS 64
+#endif
 static bool htc_ok(const Problem& pb, int x_dtype) {
   // the kernel's per-tile index arithmetic is 32-bit: tokens and work items must fit
   return pb.transform == STAMP_T_HAAR && x_dtype == STAMP_BF16 && pb.levels >= 1 && pb.n % 128 == 0 && !pb.act_zp &&
@@ -960,7 +963,8 @@ static int run_quantize_haar(const Problem& pb, const CqChoice& c, const void* X
   // continuation launches: 31 against 35 us at 2048 tokens x 4096 channels, 54.6 against 55.5 us at 8192 x 8192;
   // with 256 rows per block (32768 tokens) one CTA per 128-channel strip is too few hands (164 against 154 us).
   const int coarse_rows = pb.n >> 7;
-  hp.fold = (!tiled && !hp.last && coarse_rows <= 64) ? 1 : 0;
+  hp.fold = (!tiled && !hp.last && coarse_rows <= HTC_FOLD_ROWS) ? 1 : 0;
+  if (hp.fold && (long)pb.nseq * (pb.K / 64) <= sm_count()) hp.fold = 2;   // 64-channel strips: twice as many CTAs at work
   hp.levels = pb.levels;
   hp.nseq = pb.nseq;
   hp.done = hp.cnt + (pb.M >> 7);

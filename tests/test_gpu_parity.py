@@ -119,6 +119,8 @@ CASES = {
     # twelve levels over two sequences: the five levels above the tensor-core tile are finished by the transform
     # kernel's own tail, and most of their 32 rows per sequence take 4-bit codes (k_hi below the row count)
     "deep_tail_4bit": gen.scaled(gen.config_llm_up(), B=2, L=4096, K=256, N=64, k_hi=8),
+    # the same tail with more (sequence, 64-channel strip) items than the GPU has SMs: it then takes 128-channel strips
+    "tail_wide_strips": gen.scaled(gen.config_llm_up(), B=8, L=512, K=1280, N=64, k_hi=2),
     # 2-D Haar over the patch grid: square and oblong grids, one to three levels
     "haar2d_3": gen.scaled(gen.config_dit_proj_2d(), B=2, L=1024, K=256, N=136, grid=32, levels=3, k_hi=16),
     "haar2d_1": gen.scaled(gen.config_dit_proj_2d(), B=1, L=256, K=128, N=64, grid=16, levels=1, k_hi=64),
@@ -144,7 +146,7 @@ CASES = {
 
 
 # cases whose one-call route writes the GEMM operand in tile or patch order
-FUSED_ORDER_CASES = {"ragged", "blocked", "wide_k4096", "tile_depth5", "tile_depth7", "deep_tail_4bit", "haar2d_3",
+FUSED_ORDER_CASES = {"ragged", "blocked", "wide_k4096", "tile_depth5", "tile_depth7", "deep_tail_4bit", "tail_wide_strips", "haar2d_3",
                      "haar2d_oblong", "haar2d_max_bf16", "haar2d_max_fp32", "haar2d_wide_k"}
 
 
