@@ -144,7 +144,7 @@ int stamp_prepare_weights(const stamp_config* cfg, const void* wq_packed, int N,
 int stamp_prepare_weights_both(const stamp_config* cfg, const void* wq_packed, int N, int K, void* w_both, void* stream);
 
 /*
- * Algorithm lines "X <- L X" and "x_i <- Q(x_i; b_i)": sequence transform + per-token
+ * Algorithm 1 ("STaMP linear layer"), its first two steps: sequence transform + per-token
  * mixed-precision quantization of one activation tensor.
  *   X        [B, L, K]   x_dtype                                                    in
  *   q_hi     [B * n_hi, K]        int8, the 8-bit tokens in logical order, where
@@ -159,7 +159,7 @@ int stamp_quantize(const stamp_config* cfg, const void* X, int x_dtype, int B, i
                    void* q_lo, float* x_scale, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * Algorithm line "Y <- X W^T" on the integer codes plus de-quantization (Sec. 2.1):
+ * Algorithm 1, the product step, on the integer codes, plus de-quantization (Sec. 2.1):
  *   Yt[m, n] = (sum_k q[m,k] * wq[n,k]) * x_scale[m] * w_scale[n],   int32 accumulation on the
  * tensor cores.  Output stays in the transformed token domain.
  *   q_hi, q_lo, x_scale : as written by stamp_quantize                               in
@@ -187,7 +187,7 @@ int stamp_dequantize(const stamp_config* cfg, const void* q_hi, const void* q_lo
                      int K, float* T, void* stream);
 
 /*
- * Algorithm lines "Y <- L^-1 Y" and "Y <- Y + bias": inverse sequence transform along tokens
+ * Algorithm 1, its last two steps: inverse sequence transform along tokens
  * (L^-1 = L^T, L orthonormal: Theorem 1's premise) and optional bias.
  *   Yt       [B, L, N]   float                                                       in
  *   bias     [N] float or NULL                                                       in

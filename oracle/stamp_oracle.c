@@ -316,8 +316,8 @@ int oracle_haar_matrix_csr(int n, int levels, int64_t* row_ptr, int32_t* col, do
 }
 
 /* ------------------------------------------------------------------------------------------
- * Applying the transform along the token axis: T_b = blockdiag(Lmat) * X_b  (Algorithm line
- * "X <- L X"), or its transpose (line "Y <- L^{-1} Y" with L^{-1} = L^T).
+ * Applying the transform along the token axis: T_b = blockdiag(Lmat) * X_b  (the transform step of
+ * Algorithm 1), or its transpose (the inverse-transform step, with L^{-1} = L^T).
  * X: [B, L, K] row-major.  Lmat: n x n, n divides L.  Plain triple loop; exact zeros of the
  * matrix are skipped (they contribute nothing).
  * ------------------------------------------------------------------------------------------ */
@@ -636,7 +636,7 @@ int oracle_gemm_grouped(const int8_t* q, const float* sx, const int8_t* wq, cons
 }
 
 /* ------------------------------------------------------------------------------------------
- * Integer matmul (Algorithm line "Y <- X W^T" on the integer codes): naive triple loop,
+ * Integer matmul (the product step of Algorithm 1, on the integer codes): naive triple loop,
  * acc[m][n] = sum_k q[m][k] * wq[n][k], accumulated in int64 and checked to fit int32.
  * Returns 5 if any accumulator would overflow int32.
  * ------------------------------------------------------------------------------------------ */

@@ -1,5 +1,5 @@
-// Integer GEMM of the STaMP linear layer on the 5th-generation tensor cores (Algorithm line
-// "Y <- X W^T" evaluated on the integer codes, followed by the de-quantization of Sec. 2.1).
+// Integer GEMM of the STaMP linear layer on the 5th-generation tensor cores (the product step of
+// Algorithm 1 evaluated on the integer codes, followed by the de-quantization of Sec. 2.1).
 //
 //   acc[tok, ch] = sum_k a8[tok, k] * w8[ch, k]            int8 x int8 -> int32
 //
@@ -50,7 +50,7 @@ struct GemmParams {
   int group;               // channel tiles per raster band
   // EPI_HAAR_*: the token operand is in the tiled row order of the transform+quantize kernel, x_scale
   // holds scale * 2^(-j/2) per tile row, and the epilogue applies the inverse Haar transform of the
-  // tile's 256 tokens (Algorithm line "Y <- L^-1 Y"), w_scale and the bias before storing Y.
+  // tile's 256 tokens (the inverse-transform step of Algorithm 1), w_scale and the bias before storing Y.
   int depth;               // Haar levels closed inside a tile, 5..8
   const float* a8v;        // [m_tok / 256, n_out] level-8 approximation of every tile when the transform
                            // has more than 8 levels (orthonormal scaling), else nullptr

@@ -1,5 +1,5 @@
-// Fused Haar transform + per-token mixed-precision quantizer (Algorithm lines "X <- L X" and
-// "x_i <- Q(x_i; b_i)"): one pass over the activation in HBM, up to four Haar levels per launch.
+// Fused Haar transform + per-token mixed-precision quantizer (Algorithm 1, "STaMP
+// linear layer": its sequence transform and its per-token quantizer): one pass over the activation in HBM, up to four Haar levels per launch.
 //
 // The two axes pull in different directions: a transformed token's scale needs the maximum over
 // ALL K channels of its row, while a Haar coefficient of level l needs 2^l consecutive tokens of

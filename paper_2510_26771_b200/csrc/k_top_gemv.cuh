@@ -2,7 +2,7 @@
 // sequences: when a layer has at most 16 such rows, their product with the weights is a skinny
 // GEMV-like contraction bound by reading the weights once, not worth a tensor-core launch plus a
 // separate inverse pass.  One kernel does, per output channel:
-//   acc[r] = sum_k top_codes[r, k] * w8[ch, k]          (dp4a, int32: Algorithm line "Y <- X W^T")
+//   acc[r] = sum_k top_codes[r, k] * w8[ch, k]          (dp4a, int32: the product step of Algorithm 1)
 //   yt[r]  = acc[r] * x_scale[r]                        (weight scales are applied by the main GEMM)
 //   a8[.]  = inverse Haar of the (levels - 8) top levels over each block's rows (orthonormal)
 // and writes a8v [R, n_out]: the level-8 approximation coefficient of every 256-token tile, which
