@@ -3,9 +3,9 @@
 // features of a row has its own scale = absmax / qmax and is quantized with the symmetric round-to-nearest
 // quantizer of Sec. 2.1; the product is de-quantized group by group:
 //     Yt[m, n] = sum_g ( sum_{k in g} q[m, k] wq[n, k] ) * sx[m, g] * sw[n, g].
-// General-shape kernels, correct before fast: quantizers that read materialised rows, and a CUDA-core dp4a product
-// that scales its integer partial sums after every group.  (On the tensor cores the accumulator would have to be
-// drained after every two K32 instructions; that design is not built.)  group = 64 * 2^i, K a multiple of group.
+// General-shape kernels: quantizers that read materialised rows, and a CUDA-core dp4a product
+// that scales its integer partial sums after every group (the tensor-core product of k_gemm_grouped_tc.cuh takes the
+// shapes it can; this one the rest).  group = 64 * 2^i, K a multiple of group.
 #pragma once
 #include "common.cuh"
 #include "k_generic.cuh"

@@ -14,6 +14,7 @@
 #include "k_haar2d.cuh"
 #include "k_generic.cuh"
 #include "k_grouped.cuh"
+#include "k_gemm_grouped_tc.cuh"
 #include "k_haar_cq.cuh"
 #include "k_haar_tc.cuh"
 #include "k_peak.cuh"
@@ -702,6 +703,29 @@ static int run_quant_rows_grouped(const Problem& pb, const float* T, int8_t* a8,
 }
 static int run_gemm_grouped(const Problem& pb, const int8_t* a8, const int8_t* w8, const float* x_scale,
                             const float* w_scale, float* Yt, cudaStream_t st) {
+  // tensor cores when a ring stage (128 features) holds whole groups or is part of one, a group's partial sum
+  // converts exactly (at most 4096 features) and a tile's token scales fit the shared-memory table
+  if (pb.K % GGT_BK == 0 && pb.group >= 64 && pb.group <= 4096 && (pb.group == 64 || pb.group % 128 == 0) &&
+      pb.K / pb.group <= GGT_MAX_GROUPS && pb.M < (1L << 31)) {
+    GgtParams gp{};
+    gp.n_out = pb.N;
+    gp.m_tok = (int)pb.M;
+    gp.k = pb.K;
+    gp.group = pb.group;
+    gp.x_scale = x_scale;
+    gp.w_scale = w_scale;
+    gp.out = Yt;
+    CUtensorMap tw, tx;
+    int rc = make_tmap_i8(w8, pb.N, pb.K, GGT_BM, &tw);
+    if (rc) return rc;
+    if ((rc = make_tmap_i8(a8, pb.M, pb.K, GGT_BN, &tx))) return rc;
+    if ((rc = ensure_dyn_smem(reinterpret_cast<const void*>(k_gemm_grouped_tc), GGT_DYN_BYTES))) return rc;
+    const long tiles = ((pb.N + GGT_BM - 1) / GGT_BM) * ((pb.M + GGT_BN - 1) / GGT_BN);
+    const int grid = (int)std::min<long>(tiles, sm_count());
+    k_gemm_grouped_tc<<<grid, GGT_THREADS, GGT_DYN_BYTES, st>>>(tw, tx, gp);
+    STAMP_CHECK_LAUNCH();
+    return STAMP_OK;
+  }
   dim3 grid((unsigned)((pb.N + GG_TILE - 1) / GG_TILE), (unsigned)((pb.M + GG_TILE - 1) / GG_TILE));
   k_gemm_grouped<<<grid, 256, 0, st>>>(a8, w8, x_scale, w_scale, pb.M, pb.N, pb.K, pb.group, Yt);
   STAMP_CHECK_LAUNCH();
@@ -1365,12 +1389,14 @@ int stamp_dequantize(const stamp_config* cfg, const void* q_hi, const void* q_lo
   return STAMP_OK;
 }
 
+static int inverse_stand_in_k(const stamp_config* cfg) { return (cfg && cfg->group > 128) ? cfg->group : 128; }
+
 int stamp_inverse(const stamp_config* cfg, const float* Yt, const float* bias, int B, int L, int N, void* Y,
                   int y_dtype, void* ws, size_t ws_bytes, void* stream) {
   t_launches = 0;
   Problem pb;
-  // the inverse does not touch K: validate with a stand-in that satisfies the K rule
-  int rc = resolve(cfg, B, L, 128, N, true, &pb);
+  // the inverse does not touch K: validate with a stand-in that satisfies the K rules (a multiple of the scale group too)
+  int rc = resolve(cfg, B, L, inverse_stand_in_k(cfg), N, true, &pb);
   if (rc) return rc;
   if (!Yt || !Y || !dtype_ok(y_dtype)) return STAMP_ERR_INVALID_ARG;
   const Workspace wl = layout(pb);
@@ -1385,7 +1411,7 @@ int stamp_inverse_noalloc(const stamp_config* cfg, const float* Yt, const float*
                           int y_dtype, void* stream) {
   t_launches = 0;
   Problem pb;
-  int rc = resolve(cfg, B, L, 128, N, true, &pb);
+  int rc = resolve(cfg, B, L, inverse_stand_in_k(cfg), N, true, &pb);
   if (rc) return rc;
   if (!Yt || !Y || !dtype_ok(y_dtype)) return STAMP_ERR_INVALID_ARG;
   if (pb.transform == STAMP_T_HAAR_SKIP1) return STAMP_ERR_UNSUPPORTED;   // (its low-pass band would need half of Yt again)

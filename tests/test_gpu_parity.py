@@ -513,6 +513,10 @@ GROUP_CASES = {
     "g64_haar": (gen.scaled(gen.config_llm_up(), B=2, L=512, K=384, N=392, k_hi=16), 64),
     "g128_haar": (gen.scaled(gen.config_llm_up(), B=1, L=256, K=384, N=72, k_hi=8), 128),
     "g64_identity": (gen.scaled(gen.config_sweep(512, 2048), L=256, K=256, N=128, transform=gen.T_IDENTITY, k_hi=0), 64),
+    # more than 128 groups per row (the tensor-core product's scale table holds 128): the CUDA-core product
+    "g64_long_k": (gen.scaled(gen.config_llm_up(), B=1, L=128, K=8320, N=64, k_hi=8), 64),
+    # blocks of 256 features: a ring stage of the tensor-core product is part of one group
+    "g256_haar": (gen.scaled(gen.config_llm_up(), B=1, L=512, K=1024, N=256, k_hi=8), 256),
     # the DiT projection at full size (all 1152 output channels on the GPU, 64 of them through the oracle)
     "g64_dit_full": (gen.config_dit_proj_2d(), 64),
 }
