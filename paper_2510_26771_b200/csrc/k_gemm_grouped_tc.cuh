@@ -3,9 +3,9 @@
 //     Yt[m, n] = sum_g ( sum_{k in g} q[m, k] wq[n, k] ) * sx[m, g] * sw[n, g] ).
 // The integer partial sum of every group has to be scaled on its own, so the accumulator cannot run over all of K:
 // the MMA thread accumulates ONE group (group / 32 instructions of kind::i8, 128 channels x 128 tokens) into one of
-// two tensor-memory accumulators and commits it; the epilogue warps drain that accumulator, scale it by
+// four tensor-memory accumulators and commits it; the epilogue warps drain that accumulator, scale it by
 // sx[token, g] * sw[channel, g] and add it to fp32 sums they keep in registers (32 per thread) while the next group
-// fills the other accumulator.  The drain is the longer of the two (4 CUDA-core instructions per product of a
+// fills the next accumulator.  The drain is the longer of the two (4 CUDA-core instructions per product of a
 // 64-feature group against 1 / 64 of a tensor instruction), so this kernel runs at a fraction of the int8 rate by
 // construction -- and an order of magnitude above the CUDA-core dp4a product it replaces (k_grouped.cuh, kept for
 // the shapes this kernel does not take).
@@ -28,12 +28,13 @@ struct GgtParams {
 };
 
 constexpr int GGT_BM = 128, GGT_BN = 128, GGT_BK = 128, GGT_STAGES = 4;
+constexpr int GGT_NACC = 4;            // TMEM accumulators (all 512 columns): groups in flight between MMA and drain
 constexpr int GGT_EPI_THREADS = 512;   // sixteen epilogue warps: four per quarter of the TMEM lanes, 32 columns each
 constexpr int GGT_THREADS = 64 + GGT_EPI_THREADS;
 constexpr int GGT_MAX_GROUPS = 128;   // token scales of a tile staged in shared memory: [groups][128 tokens]
 constexpr int GGT_STAGE_BYTES = (GGT_BM + GGT_BN) * GGT_BK;
 constexpr int GGT_BAR_OFFSET = GGT_STAGES * GGT_STAGE_BYTES;
-constexpr int GGT_NUM_BARS = 2 * GGT_STAGES + 4;   // full, empty, gfull[2], gempty[2]
+constexpr int GGT_NUM_BARS = 2 * GGT_STAGES + 2 * GGT_NACC;   // full, empty, gfull, gempty
 constexpr int GGT_SX_OFFSET = GGT_BAR_OFFSET + GGT_NUM_BARS * 8 + 16;
 constexpr int GGT_DYN_BYTES = GGT_SX_OFFSET + GGT_MAX_GROUPS * GGT_BN * 4 + 1024;
 constexpr long long GGT_WAIT_LIMIT = 4000000000LL;
@@ -45,8 +46,8 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + GGT_BAR_OFFSET);
   uint64_t* empty = full + GGT_STAGES;
   uint64_t* gfull = empty + GGT_STAGES;
-  uint64_t* gempty = gfull + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gempty + 2);
+  uint64_t* gempty = gfull + GGT_NACC;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gempty + GGT_NACC);
   volatile uint32_t* abort_word = tmem_slot + 1;
   float* sxs = reinterpret_cast<float*>(smem + GGT_SX_OFFSET);
 
@@ -64,7 +65,7 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
     }
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < GGT_NACC; ++a) {
       ptx::mbar_init(&gfull[a], 1);
       ptx::mbar_init(&gempty[a], GGT_EPI_THREADS);
     }
@@ -74,7 +75,7 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
     ptx::prefetch_tensormap(&tmap_x);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, 2 * GGT_BN);
+    ptx::tmem_alloc(tmem_slot, GGT_NACC * GGT_BN);
     ptx::tmem_relinquish();
   }
   ptx::tc_fence_before();
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         const int tok_t = tile / ch_tiles, ch_t = tile - tok_t * ch_tiles;   // channel tiles fastest: CTAs share token tiles
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!ptx::mbar_wait_bounded(&empty[stage], phase ^ 1u, abort_word, GGT_WAIT_LIMIT)) {
+          if (!ptx::mbar_wait_bounded_sleepy(&empty[stage], phase ^ 1u, abort_word, GGT_WAIT_LIMIT)) {
             ok = false;
             break;
           }
@@ -125,12 +126,12 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
       constexpr uint32_t idesc = ptx::make_i8_idesc(GGT_BM, GGT_BN);
       int stage = 0;
       uint32_t phase = 0;
-      unsigned gcount = 0;   // groups issued so far: accumulator gcount & 1, its (gcount >> 1)-th filling
+      unsigned gcount = 0;   // groups issued so far: accumulator gcount % GGT_NACC, its (gcount / GGT_NACC)-th filling
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int in_group = 0;    // instructions issued into the current group
         for (int kb = 0; kb < num_kb && ok; ++kb) {
-          if (!ptx::mbar_wait_bounded(&full[stage], phase, abort_word, GGT_WAIT_LIMIT)) {
+          if (!ptx::mbar_wait_bounded_sleepy(&full[stage], phase, abort_word, GGT_WAIT_LIMIT)) {
             ok = false;
             break;
           }
@@ -138,9 +139,9 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
           const uint32_t wa = ptx::smem_u32(smem + stage * GGT_STAGE_BYTES);
           const uint32_t xa = wa + GGT_BM * GGT_BK;
           for (int k = 0; k < GGT_BK / 32; ++k) {
-            const int a = static_cast<int>(gcount & 1u);
+            const int a = static_cast<int>(gcount % GGT_NACC);
             if (in_group == 0) {   // a new group: its accumulator must have been drained
-              if (!ptx::mbar_wait_bounded(&gempty[a], ((gcount >> 1) & 1u) ^ 1u, abort_word, GGT_WAIT_LIMIT)) {
+              if (!ptx::mbar_wait_bounded_sleepy(&gempty[a], ((gcount / GGT_NACC) & 1u) ^ 1u, abort_word, GGT_WAIT_LIMIT)) {
                 ok = false;
                 break;
               }
@@ -193,16 +194,16 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
       asm volatile("bar.sync 1, %0;" ::"n"(GGT_EPI_THREADS) : "memory");
       if (*abort_word != 0u) ok = false;
       if (!ok) continue;
-      float acc[32];
+      float2 acc[16];   // column pairs, as the packed fp32 instructions take them
 #pragma unroll
-      for (int c = 0; c < 32; ++c) acc[c] = 0.f;
+      for (int c = 0; c < 16; ++c) acc[c] = make_float2(0.f, 0.f);
       const float* swp = p.w_scale + (size_t)(ch_ok ? ch : 0) * ng;
       float sw_next = ch_ok ? __ldg(swp) : 0.f;
       for (int g = 0; g < ng; ++g, ++gcount) {
-        const int a = static_cast<int>(gcount & 1u);
+        const int a = static_cast<int>(gcount % GGT_NACC);
         const float sw = sw_next;
         if (g + 1 < ng) sw_next = ch_ok ? __ldg(swp + g + 1) : 0.f;
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(&gfull[a], (gcount >> 1) & 1u, abort_word, GGT_WAIT_LIMIT))) {
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded_sleepy(&gfull[a], (gcount / GGT_NACC) & 1u, abort_word, GGT_WAIT_LIMIT))) {
           ok = false;
           *abort_word = 1;
           break;
@@ -229,17 +230,14 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             const float4 s4 = sxg[4 * q + v];
-            const int c = 16 * q + 4 * v;
-            const float2 f01 = __fadd2_rn(make_float2(__int_as_float(static_cast<int>(x[4 * v]) + 0x4B400000),
-                                                      __int_as_float(static_cast<int>(x[4 * v + 1]) + 0x4B400000)), off2);
-            const float2 f23 = __fadd2_rn(make_float2(__int_as_float(static_cast<int>(x[4 * v + 2]) + 0x4B400000),
-                                                      __int_as_float(static_cast<int>(x[4 * v + 3]) + 0x4B400000)), off2);
-            const float2 a01 = __ffma2_rn(f01, __fmul2_rn(make_float2(s4.x, s4.y), sw2), make_float2(acc[c], acc[c + 1]));
-            const float2 a23 = __ffma2_rn(f23, __fmul2_rn(make_float2(s4.z, s4.w), sw2), make_float2(acc[c + 2], acc[c + 3]));
-            acc[c] = a01.x;
-            acc[c + 1] = a01.y;
-            acc[c + 2] = a23.x;
-            acc[c + 3] = a23.y;
+            const int c2 = 8 * q + 2 * v;
+            float2 f01, f23;
+            f01.x = __int_as_float(static_cast<int>(x[4 * v]) + 0x4B400000);
+            f01.y = __int_as_float(static_cast<int>(x[4 * v + 1]) + 0x4B400000);
+            f23.x = __int_as_float(static_cast<int>(x[4 * v + 2]) + 0x4B400000);
+            f23.y = __int_as_float(static_cast<int>(x[4 * v + 3]) + 0x4B400000);
+            acc[c2] = __ffma2_rn(__fadd2_rn(f01, off2), __fmul2_rn(make_float2(s4.x, s4.y), sw2), acc[c2]);
+            acc[c2 + 1] = __ffma2_rn(__fadd2_rn(f23, off2), __fmul2_rn(make_float2(s4.z, s4.w), sw2), acc[c2 + 1]);
           }
         }
       }
@@ -247,7 +245,7 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
         float* out = p.out + (size_t)(tok0 + colq * 32) * p.n_out + ch;
 #pragma unroll
         for (int c = 0; c < 32; ++c)
-          if (tok0 + colq * 32 + c < p.m_tok) out[(size_t)c * p.n_out] = acc[c];
+          if (tok0 + colq * 32 + c < p.m_tok) out[(size_t)c * p.n_out] = (c & 1) ? acc[c >> 1].y : acc[c >> 1].x;
       }
     }
     if (!ok) {
@@ -260,7 +258,7 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
   __syncthreads();
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, 2 * GGT_BN);
+    ptx::tmem_dealloc(tmem_base, GGT_NACC * GGT_BN);
   }
 }
 
