@@ -21,7 +21,7 @@ struct GgtParams {
   int n_out;             // N output channels
   int m_tok;             // M tokens
   int k;                 // K features, a multiple of 128
-  int group;             // features per scale: 64 * 2^i, at most 4096 (a group's partial sum stays below 2^22)
+  int group;             // features per scale: 64 * 2^i, at most 4096
   const float* x_scale;  // [m_tok, k / group]
   const float* w_scale;  // [n_out, k / group]
   float* out;            // [m_tok, n_out]
@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
     }
     for (int a = 0; a < GGT_NACC; ++a) {
       ptx::mbar_init(&gfull[a], 1);
-      ptx::mbar_init(&gempty[a], GGT_EPI_THREADS);
+      ptx::mbar_init(&gempty[a], GGT_EPI_THREADS / 32);   // one arrival per epilogue warp
     }
     *abort_word = 0;
     ptx::fence_mbar_init();
@@ -210,11 +210,11 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
         }
         ptx::tc_fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(a * GGT_BN + colq * 32);
-        // two chunks of 16 columns, the next chunk's load in flight while this one is scaled.  int32 -> float by the
-        // 1.5 * 2^23 offset (exact below 2^22: a group's partial sum is), then, two columns at a time on packed
-        // fp32 instructions, one multiply for the scale pair and one fused multiply-add per product.
+        // two chunks of 16 columns, the next chunk's load in flight while this one is scaled: int32 -> float, then,
+        // two columns at a time on packed fp32 instructions, one multiply for the scale pair and one fused
+        // multiply-add per product.
         const float4* sxg = reinterpret_cast<const float4*>(sxs + g * GGT_BN + colq * 32);
-        const float2 sw2 = make_float2(sw, sw), off2 = make_float2(-12582912.0f, -12582912.0f);
+        const float2 sw2 = make_float2(sw, sw);
         uint32_t r[2][16];
         ptx::tmem_ld_32x32b_x16(taddr, r[0]);
 #pragma unroll
@@ -223,21 +223,21 @@ __global__ void __launch_bounds__(GGT_THREADS, 1)
           if (q < 1) {
             ptx::tmem_ld_32x32b_x16(taddr + 16 * (q + 1), r[(q + 1) & 1]);
           } else {
+            // the partial sums are in registers (the wait above is warp-wide): the accumulator may take a new group;
+            // one arrival per warp
             ptx::tc_fence_before();
-            ptx::mbar_arrive(&gempty[a]);   // the partial sums are in registers: the accumulator may take a new group
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&gempty[a]);
           }
           const uint32_t(&x)[16] = r[q & 1];
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             const float4 s4 = sxg[4 * q + v];
             const int c2 = 8 * q + 2 * v;
-            float2 f01, f23;
-            f01.x = __int_as_float(static_cast<int>(x[4 * v]) + 0x4B400000);
-            f01.y = __int_as_float(static_cast<int>(x[4 * v + 1]) + 0x4B400000);
-            f23.x = __int_as_float(static_cast<int>(x[4 * v + 2]) + 0x4B400000);
-            f23.y = __int_as_float(static_cast<int>(x[4 * v + 3]) + 0x4B400000);
-            acc[c2] = __ffma2_rn(__fadd2_rn(f01, off2), __fmul2_rn(make_float2(s4.x, s4.y), sw2), acc[c2]);
-            acc[c2 + 1] = __ffma2_rn(__fadd2_rn(f23, off2), __fmul2_rn(make_float2(s4.z, s4.w), sw2), acc[c2 + 1]);
+            const float2 f01 = make_float2(static_cast<float>(static_cast<int>(x[4 * v])), static_cast<float>(static_cast<int>(x[4 * v + 1])));
+            const float2 f23 = make_float2(static_cast<float>(static_cast<int>(x[4 * v + 2])), static_cast<float>(static_cast<int>(x[4 * v + 3])));
+            acc[c2] = __ffma2_rn(f01, __fmul2_rn(make_float2(s4.x, s4.y), sw2), acc[c2]);
+            acc[c2 + 1] = __ffma2_rn(f23, __fmul2_rn(make_float2(s4.z, s4.w), sw2), acc[c2 + 1]);
           }
         }
       }

@@ -703,8 +703,8 @@ static int run_quant_rows_grouped(const Problem& pb, const float* T, int8_t* a8,
 }
 static int run_gemm_grouped(const Problem& pb, const int8_t* a8, const int8_t* w8, const float* x_scale,
                             const float* w_scale, float* Yt, cudaStream_t st) {
-  // tensor cores when a ring stage (128 features) holds whole groups or is part of one, a group's partial sum
-  // converts exactly (at most 4096 features) and a tile's token scales fit the shared-memory table
+  // tensor cores when a ring stage (128 features) holds whole groups or is part of one (groups of up to 4096
+  // features) and a tile's token scales fit the shared-memory table
   if (pb.K % GGT_BK == 0 && pb.group >= 64 && pb.group <= 4096 && (pb.group == 64 || pb.group % 128 == 0) &&
       pb.K / pb.group <= GGT_MAX_GROUPS && pb.M < (1L << 31)) {
     GgtParams gp{};
